@@ -1,0 +1,386 @@
+// CPU oracle for the AQ-SGD boundary codec.
+//
+// TEST INFRASTRUCTURE ONLY.  This file is the slow, plain statement of what the
+// codec computes, written from the paper (Algorithm 1, Algorithm 2 of the
+// distributed-view appendix, and the quantizer paragraph of Section 4.1
+// "Baselines").  Only the tests, the smoke check and the benchmark's
+// cpu_baseline / reference arm may build, load or call it.  It shares no code,
+// header, table or constant generator with the CUDA library and neither side
+// includes the other.
+//
+// Arithmetic contract: every floating-point step is ONE IEEE-754 binary32
+// operation with round-to-nearest-even (compile with -ffp-contract=off, no
+// fast-math).  The 16-bit activation types (IEEE binary16 "fp16", and
+// bfloat16 "bf16") are converted by the bit-level routines below, not by a
+// compiler extension.
+//
+// Pins (tests/test_oracle_*.py): conversions against numpy/torch tables,
+// hand-derived code vectors, exact-rational brute force of the interval index,
+// the error bound Delta/2, sender/receiver buffer identity, first-visit
+// identity, zero-delta fixed point, step-change decay, bitstream length, and
+// published splitmix64 vectors for the checksum mixer.
+//
+// Parity with the paper authors' own implementation is UNPINNED: the paper
+// prints no codes, scales or bit layout; mid-rise reconstruction, the fp32
+// step as the transmitted scale and the little-endian two's-complement
+// bitstream are readings stated here and in the design notes.
+
+#include <cfloat>
+#include <cmath>
+#include <cstdint>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+namespace {
+
+// ---------------------------------------------------------------------------
+// 16-bit float types, bit level (IEEE 754-2008 binary16; bfloat16 = upper half
+// of binary32).
+// ---------------------------------------------------------------------------
+
+inline uint32_t f32_bits(float f) { uint32_t u; std::memcpy(&u, &f, 4); return u; }
+inline float bits_f32(uint32_t u) { float f; std::memcpy(&f, &u, 4); return f; }
+
+// binary16 -> binary32, exact for every input.
+float half_to_float(uint16_t h) {
+  const uint32_t sign = (uint32_t)(h & 0x8000u) << 16;
+  const uint32_t expo = (h >> 10) & 0x1Fu;
+  const uint32_t frac = h & 0x3FFu;
+  if (expo == 0x1Fu) return bits_f32(sign | 0x7F800000u | (frac << 13));  // inf / nan
+  if (expo == 0) {
+    // subnormal (or zero): value = frac * 2^-24, exactly representable in binary32
+    float mag = (float)frac * 5.9604644775390625e-08f;  // 2^-24
+    return (sign != 0) ? -mag : mag;
+  }
+  return bits_f32(sign | ((expo + 112u) << 23) | (frac << 13));
+}
+
+// binary32 -> binary16, round to nearest, ties to even; overflow gives inf.
+uint16_t float_to_half(float f) {
+  const uint32_t x = f32_bits(f);
+  const uint16_t sign = (uint16_t)((x >> 16) & 0x8000u);
+  const uint32_t mag = x & 0x7FFFFFFFu;
+  if (mag >= 0x7F800000u) {                       // inf or nan
+    return (mag == 0x7F800000u) ? (uint16_t)(sign | 0x7C00u) : (uint16_t)(sign | 0x7E00u);
+  }
+  const uint32_t e32 = mag >> 23;                 // biased binary32 exponent
+  if (e32 >= 143u) return (uint16_t)(sign | 0x7C00u);   // |f| >= 2^16: beyond every finite half
+  if (e32 >= 113u) {                              // result is a normal half (before rounding)
+    uint32_t r = ((e32 - 112u) << 10) | ((mag & 0x7FFFFFu) >> 13);
+    const uint32_t rem = mag & 0x1FFFu;
+    if (rem > 0x1000u || (rem == 0x1000u && (r & 1u))) r += 1;  // carry may reach 0x7C00 = inf
+    return (uint16_t)(sign | r);
+  }
+  // result is a subnormal half (or zero): integer r = RNE(|f| * 2^24)
+  if (e32 < 102u) return sign;                    // |f| < 2^-25 rounds to zero (2^-25 itself ties to even = 0)
+  const uint32_t m = (mag & 0x7FFFFFu) | 0x800000u;   // 24-bit significand, value = m * 2^(e32-150)
+  const uint32_t shift = 126u - e32;              // 14 .. 24
+  uint32_t r = m >> shift;
+  const uint32_t rem = m & ((1u << shift) - 1u);
+  const uint32_t halfway = 1u << (shift - 1u);
+  if (rem > halfway || (rem == halfway && (r & 1u))) r += 1;    // may become 0x400 = smallest normal
+  return (uint16_t)(sign | r);
+}
+
+float bf16_to_float(uint16_t b) { return bits_f32((uint32_t)b << 16); }
+
+// binary32 -> bfloat16, round to nearest, ties to even; overflow gives inf.
+uint16_t float_to_bf16(float f) {
+  const uint32_t x = f32_bits(f);
+  if ((x & 0x7FFFFFFFu) > 0x7F800000u) return (uint16_t)((x >> 16) | 0x0040u);  // quiet nan
+  uint32_t r = x >> 16;
+  const uint32_t rem = x & 0xFFFFu;
+  if (rem > 0x8000u || (rem == 0x8000u && (r & 1u))) r += 1;
+  return (uint16_t)r;
+}
+
+enum { DT_FP16 = 0, DT_BF16 = 1 };
+
+inline float t_to_float(uint16_t v, int dtype) {
+  return dtype == DT_FP16 ? half_to_float(v) : bf16_to_float(v);
+}
+inline uint16_t float_to_t(float v, int dtype) {
+  return dtype == DT_FP16 ? float_to_half(v) : float_to_bf16(v);
+}
+
+// ---------------------------------------------------------------------------
+// The quantizer Q (Section 4.1, "Baselines": normalise the vector into [-1,1],
+// partition [-1,1] uniformly into 2^b intervals, send the b-bit interval
+// number).  One "vector" is a group of G consecutive hidden elements.
+//
+//   s     = max_j |d_j|                          (normaliser: sup-norm)
+//   Delta = s * 2^(1-b)                          (width of one interval, un-normalised)
+//   k_j   = floor(d_j / Delta), clamped to [-2^(b-1), 2^(b-1)-1]
+//           (interval number, counted from the interval whose left edge is 0;
+//            d_j = +s lies on the right edge of the last interval and is
+//            clamped into it)
+//   Q(d)_j = (k_j + 1/2) * Delta                 (interval centre)
+//
+// Readings fixed here: the quotient is formed as d_j * (1/Delta) with one
+// division per group; a group with Delta < FLT_MIN (all-zero or vanishing) has
+// Delta = 0 and all codes 0.
+// ---------------------------------------------------------------------------
+
+void quantize_group(const float* d, int G, int bits, int32_t* k, float* delta_out) {
+  float s = 0.0f;
+  for (int j = 0; j < G; ++j) {
+    const float a = std::fabs(d[j]);
+    if (a > s) s = a;
+  }
+  const float two_pow = 1.0f / (float)(1 << (bits - 1));   // 2^(1-b), exact
+  float delta = s * two_pow;
+  if (!(delta >= FLT_MIN)) {
+    *delta_out = 0.0f;
+    for (int j = 0; j < G; ++j) k[j] = 0;
+    return;
+  }
+  const float inv = 1.0f / delta;
+  const float kmin = -(float)(1 << (bits - 1));
+  const float kmax = (float)((1 << (bits - 1)) - 1);
+  for (int j = 0; j < G; ++j) {
+    const float u = d[j] * inv;
+    float kf = std::floor(u);
+    if (kf < kmin) kf = kmin;
+    if (kf > kmax) kf = kmax;
+    k[j] = (int32_t)kf;
+  }
+  *delta_out = delta;
+}
+
+inline float reconstruct(int32_t k, float delta) {
+  const float centre = (float)k + 0.5f;    // exact
+  return centre * delta;
+}
+
+// ---------------------------------------------------------------------------
+// Bitstream: element j of a stream owns bits [j*b, (j+1)*b); bit t of the
+// stream is bit (t mod 8) of byte (t div 8).  The field is the low b bits of
+// the two's-complement code.
+// ---------------------------------------------------------------------------
+
+void put_code(uint8_t* stream, int64_t j, int bits, int32_t k) {
+  const uint32_t field = (uint32_t)k & ((1u << bits) - 1u);
+  const int64_t t0 = j * bits;
+  for (int i = 0; i < bits; ++i) {
+    const int64_t t = t0 + i;
+    const uint8_t bit = (uint8_t)((field >> i) & 1u);
+    uint8_t& byte = stream[t >> 3];
+    byte = (uint8_t)((byte & ~(1u << (t & 7))) | (bit << (t & 7)));
+  }
+}
+
+int32_t get_code(const uint8_t* stream, int64_t j, int bits) {
+  uint32_t field = 0;
+  const int64_t t0 = j * bits;
+  for (int i = 0; i < bits; ++i) {
+    const int64_t t = t0 + i;
+    field |= (uint32_t)((stream[t >> 3] >> (t & 7)) & 1u) << i;
+  }
+  if (field & (1u << (bits - 1))) field |= ~((1u << bits) - 1u);   // sign-extend
+  return (int32_t)field;
+}
+
+// ---------------------------------------------------------------------------
+// State of one side of one boundary: the array m of previous messages, indexed
+// by sample (Algorithm 1, "array of previous messages m initialized to 0"),
+// and the "seen before" set.
+// ---------------------------------------------------------------------------
+
+struct Side {
+  int64_t n_samples;
+  int seq, hidden, bits, group, dtype;
+  std::vector<uint16_t> m;       // [n_samples][seq][hidden], activation dtype
+  std::vector<uint8_t> seen;     // [n_samples]
+  uint32_t status;               // sticky: 1 id out of range, 2 duplicate id in a call, 4 first visit at decode with no raw message
+};
+
+enum { ST_BAD_ID = 1, ST_DUP_ID = 2, ST_NO_RAW = 4 };
+
+// 0 = steady (delta) visit, 1 = first visit, 2 = skipped (bad or repeated id)
+int resolve(Side* S, const int32_t* ids, int y) {
+  const int64_t id = ids[y];
+  if (id < 0 || id >= S->n_samples) { S->status |= ST_BAD_ID; return 2; }
+  for (int p = 0; p < y; ++p)
+    if (ids[p] == ids[y]) { S->status |= ST_DUP_ID; return 2; }
+  return S->seen[id] ? 0 : 1;
+}
+
+uint64_t mix64(uint64_t index, uint64_t word) {
+  // splitmix64 output function (Steele, Lea, Flood 2014; Vigna's constants)
+  uint64_t z = index * 0x9E3779B97F4A7C15ull + word;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+
+}  // namespace
+
+extern "C" {
+
+// ---- conversions and the bare quantizer, exported so the pins can reach them
+
+float aqo_half_to_float(uint16_t h) { return half_to_float(h); }
+uint16_t aqo_float_to_half(float f) { return float_to_half(f); }
+float aqo_bf16_to_float(uint16_t h) { return bf16_to_float(h); }
+uint16_t aqo_float_to_bf16(float f) { return float_to_bf16(f); }
+uint64_t aqo_mix64(uint64_t index, uint64_t word) { return mix64(index, word); }
+
+void aqo_quantize_group(const float* d, int G, int bits, int32_t* k, float* delta) {
+  quantize_group(d, G, bits, k, delta);
+}
+float aqo_reconstruct(int32_t k, float delta) { return reconstruct(k, delta); }
+void aqo_put_code(uint8_t* stream, int64_t j, int bits, int32_t k) { put_code(stream, j, bits, k); }
+int32_t aqo_get_code(const uint8_t* stream, int64_t j, int bits) { return get_code(stream, j, bits); }
+
+// ---- one side of one boundary
+
+void* aqo_create(int64_t n_samples, int seq, int hidden, int bits, int group, int dtype) {
+  if (n_samples <= 0 || seq <= 0 || hidden <= 0 || bits < 1 || bits > 8 || group <= 0) return nullptr;
+  if (hidden % group != 0 || (dtype != DT_FP16 && dtype != DT_BF16)) return nullptr;
+  if (((int64_t)seq * hidden * bits) % 8 != 0) return nullptr;
+  Side* S = new (std::nothrow) Side();
+  if (!S) return nullptr;
+  S->n_samples = n_samples; S->seq = seq; S->hidden = hidden;
+  S->bits = bits; S->group = group; S->dtype = dtype; S->status = 0;
+  S->m.assign((size_t)n_samples * seq * hidden, 0);     // "initialized to 0"
+  S->seen.assign((size_t)n_samples, 0);
+  return S;
+}
+
+void aqo_destroy(void* h) { delete (Side*)h; }
+
+const uint16_t* aqo_m(void* h) { return ((Side*)h)->m.data(); }
+const uint8_t* aqo_seen(void* h) { return ((Side*)h)->seen.data(); }
+uint32_t aqo_status(void* h) { Side* S = (Side*)h; uint32_t s = S->status; S->status = 0; return s; }
+
+// Sender (Algorithm 2, "on network a"; Algorithm 1 lines 4-9).
+//   act     [n_batch][seq][hidden]  activation a(xi)
+//   ids     [n_batch]               sample ids xi
+//   packed  [n_batch][seq*hidden*bits/8]   out: bitstream of codes
+//   scales  [n_batch][seq][hidden/group]   out: Delta of every group
+//   first   [n_batch] or null       out: 1 where the sample was a first visit
+// First visit: m(xi) = a(xi) (the full-precision activation is the message),
+// codes and scales of that sample are zero.  Otherwise
+//   Delta_m = Q(a - m),  m <- m + Delta_m,  codes/scales describe Delta_m.
+void aqo_encode(void* h, const uint16_t* act, const int32_t* ids, int n_batch,
+                uint8_t* packed, float* scales, uint8_t* first) {
+  Side* S = (Side*)h;
+  const int64_t E = (int64_t)S->seq * S->hidden;
+  const int64_t pbytes = E * S->bits / 8;
+  const int64_t ngroups = E / S->group;
+  std::vector<float> d(S->group);
+  std::vector<int32_t> k(S->group);
+  for (int y = 0; y < n_batch; ++y) {
+    const uint16_t* a = act + (int64_t)y * E;
+    uint8_t* P = packed + (int64_t)y * pbytes;
+    float* SC = scales + (int64_t)y * ngroups;
+    std::memset(P, 0, (size_t)pbytes);
+    for (int64_t g = 0; g < ngroups; ++g) SC[g] = 0.0f;
+    const int mode = resolve(S, ids, y);
+    if (first) first[y] = (uint8_t)(mode == 1);
+    if (mode == 2) continue;
+    uint16_t* M = S->m.data() + (int64_t)ids[y] * E;
+    if (mode == 1) {
+      for (int64_t i = 0; i < E; ++i) M[i] = a[i];
+      S->seen[ids[y]] = 1;
+      continue;
+    }
+    for (int64_t g = 0; g < ngroups; ++g) {          // groups never straddle token rows: hidden % group == 0
+      const int64_t base = g * S->group;
+      for (int j = 0; j < S->group; ++j)
+        d[j] = t_to_float(a[base + j], S->dtype) - t_to_float(M[base + j], S->dtype);
+      float delta;
+      quantize_group(d.data(), S->group, S->bits, k.data(), &delta);
+      SC[g] = delta;
+      for (int j = 0; j < S->group; ++j) {
+        put_code(P, base + j, S->bits, k[j]);
+        const float qhat = reconstruct(k[j], delta);        // (0 + 1/2) * 0 = 0 for a zero group
+        const float sum = t_to_float(M[base + j], S->dtype) + qhat;
+        M[base + j] = float_to_t(sum, S->dtype);
+      }
+    }
+  }
+}
+
+// Receiver (Algorithm 2, "on network b": m <- m + Delta_m, then m is the
+// forward activation).
+//   raw  [n_batch][seq][hidden] or null: the uncompressed message of first-visit samples
+//   out  [n_batch][seq][hidden]: the activation handed to network b
+// A skipped sample (bad id, repeated id, first visit with raw == null) gets an
+// all-zero out block and no state change.
+void aqo_decode(void* h, const uint8_t* packed, const float* scales, const uint16_t* raw,
+                const int32_t* ids, int n_batch, uint16_t* out, uint8_t* first) {
+  Side* S = (Side*)h;
+  const int64_t E = (int64_t)S->seq * S->hidden;
+  const int64_t pbytes = E * S->bits / 8;
+  const int64_t ngroups = E / S->group;
+  for (int y = 0; y < n_batch; ++y) {
+    uint16_t* O = out + (int64_t)y * E;
+    int mode = resolve(S, ids, y);
+    if (mode == 1 && raw == nullptr) { S->status |= ST_NO_RAW; mode = 2; }
+    if (first) first[y] = (uint8_t)(mode == 1);
+    if (mode == 2) { for (int64_t i = 0; i < E; ++i) O[i] = 0; continue; }
+    uint16_t* M = S->m.data() + (int64_t)ids[y] * E;
+    if (mode == 1) {
+      const uint16_t* R = raw + (int64_t)y * E;
+      for (int64_t i = 0; i < E; ++i) { M[i] = R[i]; O[i] = R[i]; }
+      S->seen[ids[y]] = 1;
+      continue;
+    }
+    const uint8_t* P = packed + (int64_t)y * pbytes;
+    const float* SC = scales + (int64_t)y * ngroups;
+    for (int64_t i = 0; i < E; ++i) {
+      const float delta = SC[i / S->group];
+      const int32_t k = get_code(P, i, S->bits);
+      const float qhat = reconstruct(k, delta);
+      const float sum = t_to_float(M[i], S->dtype) + qhat;
+      M[i] = float_to_t(sum, S->dtype);
+      O[i] = M[i];
+    }
+  }
+}
+
+// Direct quantization of the backward activation-gradient (Algorithm 1,
+// "Machine b sends Q(grad_a (f o b)|_m)"): same Q, no buffer, no delta.
+void aqo_quant_grad(const uint16_t* grad, int64_t n_elems, int bits, int group, int dtype,
+                    uint8_t* packed, float* scales) {
+  std::vector<float> d(group);
+  std::vector<int32_t> k(group);
+  std::memset(packed, 0, (size_t)(n_elems * bits / 8));
+  for (int64_t g = 0; g < n_elems / group; ++g) {
+    const int64_t base = g * group;
+    for (int j = 0; j < group; ++j) d[j] = t_to_float(grad[base + j], dtype);
+    float delta;
+    quantize_group(d.data(), group, bits, k.data(), &delta);
+    scales[g] = delta;
+    for (int j = 0; j < group; ++j) put_code(packed, base + j, bits, k[j]);
+  }
+}
+
+void aqo_dequant_grad(const uint8_t* packed, const float* scales, int64_t n_elems, int bits,
+                      int group, int dtype, uint16_t* out) {
+  for (int64_t i = 0; i < n_elems; ++i) {
+    const float delta = scales[i / group];
+    const float v = reconstruct(get_code(packed, i, bits), delta);
+    out[i] = float_to_t(v, dtype);
+  }
+}
+
+// Order-independent 64-bit digest of the whole state: the m array read as
+// little-endian 32-bit words (word i = elements 2i, 2i+1), plus the seen set.
+uint64_t aqo_state_checksum(void* h) {
+  Side* S = (Side*)h;
+  uint64_t sum = 0;
+  const int64_t nwords = (int64_t)S->m.size() / 2;
+  for (int64_t i = 0; i < nwords; ++i) {
+    const uint32_t w = (uint32_t)S->m[2 * i] | ((uint32_t)S->m[2 * i + 1] << 16);
+    sum += mix64((uint64_t)i, w);
+  }
+  for (int64_t x = 0; x < S->n_samples; ++x)
+    sum += mix64((1ull << 40) + (uint64_t)x, S->seen[x]);
+  return sum;
+}
+
+}  // extern "C"
