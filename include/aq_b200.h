@@ -1,0 +1,179 @@
+/*
+ * aq_b200 -- AQ-SGD activation-delta codec for one NVIDIA B200 (sm_100a).
+ *
+ * C ABI of the boundary codec that AQ-SGD (Algorithm 1; two-machine form:
+ * Algorithm 2 of the appendix "Distributed View") runs where one pipeline
+ * stage hands its activations to the next:
+ *
+ *   sender    Delta_m = Q(a(xi) - m(xi));  m(xi) <- m(xi) + Delta_m;  send Delta_m
+ *   receiver  m(xi) <- m(xi) + Delta_m;    use m(xi) as the forward activation
+ *   backward  send Q(gradient) -- plain quantization, no buffer
+ *
+ * Q is the uniform b-bit quantizer of Section 4.1 ("Baselines"): a vector is
+ * normalised into [-1,1] by its largest magnitude, [-1,1] is cut into 2^b equal
+ * intervals and each number is sent as the b-bit number of its interval.  Here
+ * a "vector" is a group of `group` consecutive hidden elements of one token:
+ *
+ *   s = max|d|,  Delta = s * 2^(1-b),  k = clamp(floor(d * (1/Delta)), -2^(b-1), 2^(b-1)-1),
+ *   Q(d) = (k + 1/2) * Delta;   Delta < FLT_MIN  =>  Delta = 0, k = 0.
+ *
+ * All arithmetic is IEEE binary32, one rounding per operation (no fused
+ * multiply-add), so results are reproducible bit for bit.
+ *
+ * One handle is ONE copy of the previous-message array m (Algorithm 1: "array
+ * of previous messages m initialized to 0"): the sender's or the receiver's
+ * side of one stage boundary.  A pipeline with K stages uses K-1 independent
+ * pairs of handles (appendix A.1).
+ *
+ * Layouts (all row-major, densely packed):
+ *   activations / gradients  T[n_batch][seq][hidden], T = fp16 or bf16 (2 bytes)
+ *   m                        T[n_samples][seq][hidden], owned by the handle
+ *   packed                   uint8[n_batch][seq*hidden*bits/8]; per sample a little-endian
+ *                            bitstream: element j owns stream bits [j*bits, (j+1)*bits),
+ *                            stream bit t is bit (t mod 8) of byte (t div 8); the field is
+ *                            the two's-complement code k truncated to `bits` bits
+ *   scales                   float[n_batch][seq][hidden/group], holds Delta of each group
+ *
+ * Pointers: unless a function says "host", every data pointer is a DEVICE
+ * pointer (or any pointer the GPU can read, e.g. pinned host memory for
+ * sample_ids), 16-byte aligned, owned by the caller, and must stay valid until
+ * the work queued on the handle's stream has finished.  The functions only
+ * enqueue work on that stream and return; they do not synchronise unless they
+ * say so.  Calls on one handle must not overlap on the GPU (use one stream per
+ * handle, or order the streams).
+ *
+ * Errors: functions returning int give AQ_OK or a negative AQ_E* code and leave
+ * a message for aq_last_error().  Conditions only the GPU can see (a sample id
+ * out of range, an id repeated inside one call, a first visit at the receiver
+ * with no raw message) never fault: that sample is skipped -- no state change,
+ * its outputs zero-filled -- and a sticky bit is set that aq_status() returns.
+ * Preconditions that are not checked: finite inputs; both sides of a boundary
+ * are fed the same sequence of sample ids.
+ */
+#ifndef AQ_B200_H
+#define AQ_B200_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct aq_handle aq_handle;
+
+enum {
+  AQ_OK = 0,
+  AQ_EINVAL = -1,        /* null / misaligned pointer, size or setting out of range */
+  AQ_ENOMEM = -2,        /* device or host allocation failed */
+  AQ_ECUDA = -3,         /* a CUDA runtime call failed; aq_last_error() names it */
+  AQ_EUNSUPPORTED = -4   /* valid request that this build has no kernel for */
+};
+
+/* keys of aq_configure */
+enum {
+  AQ_DTYPE = 1,          /* AQ_FP16 (default) or AQ_BF16: type T of activations, gradients and m */
+  AQ_BATCH = 2,          /* n_batch: sequences per aq_encode / aq_decode call, 0..65535 (default 1) */
+  AQ_STREAM = 3,         /* cudaStream_t as an integer (default 0, the legacy default stream) */
+  AQ_RAW = 4,            /* device pointer T[n_batch][seq][hidden]: the uncompressed message that
+                            aq_decode stores for first-visit samples; 0 = none (default) */
+  AQ_FIRST_FLAGS = 5     /* device pointer uint8[n_batch] or 0: aq_encode / aq_decode write 1 for
+                            each sample that took the first-visit path, else 0 */
+};
+enum { AQ_FP16 = 0, AQ_BF16 = 1 };
+
+/* sticky bits of aq_status */
+enum {
+  AQ_ST_BAD_ID = 1,      /* a sample id was < 0 or >= n_samples */
+  AQ_ST_DUP_ID = 2,      /* an id appeared twice in one call; every occurrence after the first is skipped */
+  AQ_ST_NO_RAW = 4       /* aq_decode met a first-visit sample while AQ_RAW was 0 */
+};
+
+/*
+ * Algorithm 1, "Initialize": allocates m (n_samples*seq*hidden*2 bytes of device
+ * memory on the current device) filled with zeros, and an empty "seen before"
+ * set.  bits in 1..8 is b of the forward quantizer; group in {8,16,32,64,128,256}
+ * must divide hidden.  Returns NULL on failure; aq_last_error(NULL) says why.
+ */
+aq_handle* aq_create(int64_t n_samples, int seq, int hidden, int bits, int group);
+
+/* Waits for the handle's stream, frees everything the handle owns.  NULL is allowed. */
+void aq_destroy(aq_handle* h);
+
+int aq_configure(aq_handle* h, int key, int64_t value);
+
+/*
+ * Sender side (Algorithm 2, "on network a"; Algorithm 1 lines 4-9).  For each
+ * of the n_batch samples, in one fused pass over the data:
+ *   first visit  m(xi) <- act (bit copy; the full-precision activation itself is the
+ *                message, the caller forwards `act`), codes and scales of the sample = 0;
+ *   otherwise    d = act - m(xi); per group: Delta, codes k; m(xi) <- T(m(xi) + (k+1/2)*Delta).
+ * act T[n_batch][seq][hidden] (in), sample_ids int32[n_batch] (in),
+ * packed and scales (out, layouts above).
+ */
+int aq_encode(aq_handle* h, const void* act, const int32_t* sample_ids, void* packed, float* scales);
+
+/*
+ * Receiver side (Algorithm 2, "on network b"): m(xi) <- T(m(xi) + (k+1/2)*Delta) on this
+ * handle's own copy of m, and out <- the new m(xi), which network b uses as its forward
+ * activation.  First visit: m(xi) <- raw, out <- raw (AQ_RAW).
+ * packed, scales (in), sample_ids int32[n_batch] (in), out T[n_batch][seq][hidden] (out).
+ */
+int aq_decode(aq_handle* h, const void* packed, const float* scales, const int32_t* sample_ids, void* out);
+
+/*
+ * Backward direction (Algorithm 1: "Machine b sends Q(gradient of f o b w.r.t. a)"):
+ * the same Q applied directly to the gradient; touches no state.  n_elems must be a
+ * multiple of the handle's group; bits in 1..8 may differ from the handle's forward b.
+ * grad T[n_elems] (in); packed uint8[n_elems*bits/8], scales float[n_elems/group] (out).
+ * n_elems == 0 is a no-op.
+ */
+int aq_quant_grad(aq_handle* h, const void* grad, int64_t n_elems, int bits, void* packed, float* scales);
+
+/* Inverse: out[j] = T((k_j + 1/2) * Delta).  packed, scales (in); out T[n_elems] (out). */
+int aq_dequant_grad(aq_handle* h, const void* packed, const float* scales, int64_t n_elems, int bits, void* out);
+
+/*
+ * 64-bit digest of the whole state, independent of summation order:
+ *   sum_i mix(i, word_i) + sum_xi mix(2^40 + xi, seen[xi])   (mod 2^64),
+ * word_i = the i-th little-endian 32-bit word of m, mix(i, w) = the splitmix64 output
+ * function applied to i*0x9E3779B97F4A7C15 + w.  Two handles fed the same id sequence
+ * (the two sides of a boundary, Algorithm 2: "networks a and b each maintain a copy")
+ * must give the same digest.  Synchronises the stream; *out_host is host memory.
+ */
+int aq_state_checksum(aq_handle* h, uint64_t* out_host);
+
+/* Synchronises the stream, returns the sticky AQ_ST_* bits in *bits_host (host) and clears them. */
+int aq_status(aq_handle* h, uint32_t* bits_host);
+
+/* Message of the last failed call on this handle; with h == NULL, of the last failed
+ * aq_create on this thread.  Never NULL.  The string is owned by the library. */
+const char* aq_last_error(aq_handle* h);
+
+/* Bytes of `packed` and floats of `scales` per sample for this handle's forward settings. */
+int64_t aq_packed_bytes_per_sample(aq_handle* h);
+int64_t aq_scales_per_sample(aq_handle* h);
+
+/*
+ * Host-buffer forms: same operations, but every pointer is HOST memory (pinned memory
+ * makes the copies asynchronous to the CPU; pageable works).  The call copies the inputs
+ * to device staging buffers owned by the handle (allocated on first use, sized for the
+ * current AQ_BATCH), runs the same kernel, copies the results back and returns after the
+ * stream has finished.  raw_host may be NULL (then first visits at the receiver are
+ * skipped and reported, as with AQ_RAW = 0).
+ */
+int aq_encode_host(aq_handle* h, const void* act_host, const int32_t* sample_ids_host,
+                   void* packed_host, float* scales_host);
+int aq_decode_host(aq_handle* h, const void* packed_host, const float* scales_host,
+                   const void* raw_host, const int32_t* sample_ids_host, void* out_host);
+
+/*
+ * State access for checkpoints and tests.  Copies one sample's m block (seq*hidden*2
+ * bytes) and its seen flag between the handle and HOST memory; synchronises the stream.
+ */
+int aq_export_sample(aq_handle* h, int64_t sample_id, void* m_host, uint8_t* seen_host);
+int aq_import_sample(aq_handle* h, int64_t sample_id, const void* m_host, uint8_t seen);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AQ_B200_H */

@@ -1,0 +1,329 @@
+// C ABI of the codec: handle, argument checks, stream plumbing.  All arithmetic lives in
+// aq_kernels.cu; nothing here computes on the CPU and there is no CPU fallback.
+
+#include "../../include/aq_b200.h"
+#include "aq_internal.h"
+
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+struct aq_handle {
+  aq::State st{};
+  int seq = 0, hidden = 0, bits = 0, group = 0;
+  int dtype = AQ_FP16;
+  int n_batch = 1;
+  int device = 0;
+  cudaStream_t stream = nullptr;
+  const void* raw = nullptr;
+  uint8_t* first_flags = nullptr;
+  unsigned long long* sum_dev = nullptr;     // scratch of aq_state_checksum
+  // staging for the host-buffer entry points, sized for staged_batch samples
+  int staged_batch = 0;
+  void* d_act = nullptr;      // also raw / out
+  int32_t* d_ids = nullptr;
+  uint8_t* d_packed = nullptr;
+  float* d_scales = nullptr;
+  char err[256] = {0};
+};
+
+namespace {
+
+thread_local char g_create_err[256] = "";
+
+int fail(aq_handle* h, int code, const char* fmt, ...) {
+  char* dst = h ? h->err : g_create_err;
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(dst, 256, fmt, ap);
+  va_end(ap);
+  return code;
+}
+
+int cuda_fail(aq_handle* h, cudaError_t e, const char* what) {
+  return fail(h, e == cudaErrorMemoryAllocation ? AQ_ENOMEM : AQ_ECUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+#define AQ_CUDA(h, call)                                   \
+  do {                                                     \
+    cudaError_t e_ = (call);                               \
+    if (e_ != cudaSuccess) return cuda_fail(h, e_, #call); \
+  } while (0)
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int lanes_for_group(int group) {
+  switch (group) {
+    case 8: case 16: case 32: case 64: case 128: case 256: return group / 8;
+    default: return 0;
+  }
+}
+
+// The handle's device must be current for launches on its stream; restore on exit.
+struct DeviceGuard {
+  int prev = -1;
+  explicit DeviceGuard(int dev) {
+    cudaGetDevice(&prev);
+    if (prev != dev) cudaSetDevice(dev);
+    else prev = -1;
+  }
+  ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+void free_staging(aq_handle* h) {
+  cudaFree(h->d_act); cudaFree(h->d_ids); cudaFree(h->d_packed); cudaFree(h->d_scales);
+  h->d_act = nullptr; h->d_ids = nullptr; h->d_packed = nullptr; h->d_scales = nullptr;
+  h->staged_batch = 0;
+}
+
+int ensure_staging(aq_handle* h) {
+  if (h->staged_batch >= h->n_batch && h->d_act) return AQ_OK;
+  AQ_CUDA(h, cudaStreamSynchronize(h->stream));
+  free_staging(h);
+  const size_t nb = (size_t)(h->n_batch > 0 ? h->n_batch : 1);
+  AQ_CUDA(h, cudaMalloc(&h->d_act, nb * (size_t)h->st.elems * 2));
+  AQ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&h->d_ids), nb * sizeof(int32_t)));
+  AQ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&h->d_packed), nb * (size_t)h->st.packed_bytes));
+  AQ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&h->d_scales), nb * (size_t)h->st.groups * sizeof(float)));
+  h->staged_batch = (int)nb;
+  return AQ_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+aq_handle* aq_create(int64_t n_samples, int seq, int hidden, int bits, int group) {
+  g_create_err[0] = 0;
+  const int lanes = lanes_for_group(group);
+  if (n_samples <= 0 || seq <= 0 || hidden <= 0) { fail(nullptr, AQ_EINVAL, "n_samples, seq and hidden must be positive"); return nullptr; }
+  if (bits < 1 || bits > 8) { fail(nullptr, AQ_EINVAL, "bits must be in 1..8 (got %d)", bits); return nullptr; }
+  if (!lanes) { fail(nullptr, AQ_EINVAL, "group must be one of 8,16,32,64,128,256 (got %d)", group); return nullptr; }
+  if (hidden % group) { fail(nullptr, AQ_EINVAL, "group %d does not divide hidden %d", group, hidden); return nullptr; }
+  aq_handle* h = new (std::nothrow) aq_handle();
+  if (!h) { fail(nullptr, AQ_ENOMEM, "host allocation failed"); return nullptr; }
+  h->seq = seq; h->hidden = hidden; h->bits = bits; h->group = group;
+  aq::State& st = h->st;
+  st.n_samples = n_samples;
+  st.elems = (long long)seq * hidden;
+  st.chunks = st.elems / aq::kChunk;
+  st.packed_bytes = st.elems * bits / 8;
+  st.groups = st.elems / group;
+  st.lanes_per_group = lanes;
+  st.lg_shift = __builtin_ctz((unsigned)lanes);
+  cudaError_t e = cudaGetDevice(&h->device);
+  const size_t m_bytes = (size_t)n_samples * (size_t)st.elems * 2;
+  if (e == cudaSuccess) e = cudaMalloc(&st.m, m_bytes);
+  if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&st.seen), (size_t)n_samples);
+  if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&st.status), 2 * sizeof(uint32_t));
+  if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&h->sum_dev), sizeof(unsigned long long));
+  if (e == cudaSuccess) e = cudaMemset(st.m, 0, m_bytes);                      // "initialized to 0"
+  if (e == cudaSuccess) e = cudaMemset(st.seen, 0, (size_t)n_samples);
+  if (e == cudaSuccess) e = cudaMemset(st.status, 0, 2 * sizeof(uint32_t));
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) {
+    cuda_fail(nullptr, e, "aq_create");
+    cudaGetLastError();
+    aq_destroy(h);
+    return nullptr;
+  }
+  st.ticket = st.status + 1;
+  return h;
+}
+
+void aq_destroy(aq_handle* h) {
+  if (!h) return;
+  DeviceGuard g(h->device);
+  cudaStreamSynchronize(h->stream);
+  free_staging(h);
+  cudaFree(h->st.m);
+  cudaFree(h->st.seen);
+  cudaFree(h->st.status);
+  cudaFree(h->sum_dev);
+  delete h;
+}
+
+int aq_configure(aq_handle* h, int key, int64_t value) {
+  if (!h) return fail(nullptr, AQ_EINVAL, "null handle");
+  switch (key) {
+    case AQ_DTYPE:
+      if (value != AQ_FP16 && value != AQ_BF16) return fail(h, AQ_EINVAL, "AQ_DTYPE must be AQ_FP16 or AQ_BF16");
+      h->dtype = (int)value;
+      return AQ_OK;
+    case AQ_BATCH:
+      if (value < 0 || value > 65535) return fail(h, AQ_EINVAL, "AQ_BATCH must be in 0..65535");
+      h->n_batch = (int)value;
+      return AQ_OK;
+    case AQ_STREAM:
+      h->stream = reinterpret_cast<cudaStream_t>(static_cast<intptr_t>(value));
+      return AQ_OK;
+    case AQ_RAW:
+      if (value & 15) return fail(h, AQ_EINVAL, "AQ_RAW pointer must be 16-byte aligned");
+      h->raw = reinterpret_cast<const void*>(static_cast<intptr_t>(value));
+      return AQ_OK;
+    case AQ_FIRST_FLAGS:
+      h->first_flags = reinterpret_cast<uint8_t*>(static_cast<intptr_t>(value));
+      return AQ_OK;
+    default:
+      return fail(h, AQ_EINVAL, "unknown configure key %d", key);
+  }
+}
+
+int aq_encode(aq_handle* h, const void* act, const int32_t* sample_ids, void* packed, float* scales) {
+  if (!h) return fail(nullptr, AQ_EINVAL, "null handle");
+  if (h->n_batch == 0) return AQ_OK;
+  if (!act || !sample_ids || !packed || !scales) return fail(h, AQ_EINVAL, "aq_encode: null pointer");
+  if (!aligned16(act) || !aligned16(packed) || !aligned16(scales))
+    return fail(h, AQ_EINVAL, "aq_encode: act, packed and scales must be 16-byte aligned");
+  DeviceGuard g(h->device);
+  aq::EncodeArgs a{act, sample_ids, static_cast<uint8_t*>(packed), scales, h->first_flags, h->n_batch};
+  AQ_CUDA(h, aq::launch_encode(h->dtype, h->bits, h->st, a, h->stream));
+  return AQ_OK;
+}
+
+int aq_decode(aq_handle* h, const void* packed, const float* scales, const int32_t* sample_ids, void* out) {
+  if (!h) return fail(nullptr, AQ_EINVAL, "null handle");
+  if (h->n_batch == 0) return AQ_OK;
+  if (!packed || !scales || !sample_ids || !out) return fail(h, AQ_EINVAL, "aq_decode: null pointer");
+  if (!aligned16(packed) || !aligned16(scales) || !aligned16(out))
+    return fail(h, AQ_EINVAL, "aq_decode: packed, scales and out must be 16-byte aligned");
+  DeviceGuard g(h->device);
+  aq::DecodeArgs a{static_cast<const uint8_t*>(packed), scales, h->raw, sample_ids, out, h->first_flags, h->n_batch};
+  AQ_CUDA(h, aq::launch_decode(h->dtype, h->bits, h->st, a, h->stream));
+  return AQ_OK;
+}
+
+static int check_grad_args(aq_handle* h, const void* a, const void* b, const void* c, int64_t n_elems, int bits) {
+  if (!h) return fail(nullptr, AQ_EINVAL, "null handle");
+  if (bits < 1 || bits > 8) return fail(h, AQ_EINVAL, "bits must be in 1..8 (got %d)", bits);
+  if (n_elems < 0 || n_elems % h->group) return fail(h, AQ_EINVAL, "n_elems must be a non-negative multiple of group %d", h->group);
+  if (n_elems == 0) return AQ_OK;
+  if (!a || !b || !c) return fail(h, AQ_EINVAL, "null pointer");
+  if (!aligned16(a) || !aligned16(b) || !aligned16(c)) return fail(h, AQ_EINVAL, "pointers must be 16-byte aligned");
+  return AQ_OK;
+}
+
+int aq_quant_grad(aq_handle* h, const void* grad, int64_t n_elems, int bits, void* packed, float* scales) {
+  const int rc = check_grad_args(h, grad, packed, scales, n_elems, bits);
+  if (rc != AQ_OK || n_elems == 0) return rc;
+  DeviceGuard g(h->device);
+  AQ_CUDA(h, aq::launch_quant_grad(h->dtype, bits, h->st.lanes_per_group, grad, n_elems,
+                                   static_cast<uint8_t*>(packed), scales, h->stream));
+  return AQ_OK;
+}
+
+int aq_dequant_grad(aq_handle* h, const void* packed, const float* scales, int64_t n_elems, int bits, void* out) {
+  const int rc = check_grad_args(h, packed, scales, out, n_elems, bits);
+  if (rc != AQ_OK || n_elems == 0) return rc;
+  DeviceGuard g(h->device);
+  AQ_CUDA(h, aq::launch_dequant_grad(h->dtype, bits, h->st.lanes_per_group, static_cast<const uint8_t*>(packed),
+                                     scales, n_elems, out, h->stream));
+  return AQ_OK;
+}
+
+int aq_state_checksum(aq_handle* h, uint64_t* out_host) {
+  if (!h) return fail(nullptr, AQ_EINVAL, "null handle");
+  if (!out_host) return fail(h, AQ_EINVAL, "aq_state_checksum: null pointer");
+  DeviceGuard g(h->device);
+  AQ_CUDA(h, cudaMemsetAsync(h->sum_dev, 0, sizeof(unsigned long long), h->stream));
+  AQ_CUDA(h, aq::launch_checksum(h->st, h->sum_dev, h->stream));
+  unsigned long long v = 0;
+  AQ_CUDA(h, cudaMemcpyAsync(&v, h->sum_dev, sizeof(v), cudaMemcpyDeviceToHost, h->stream));
+  AQ_CUDA(h, cudaStreamSynchronize(h->stream));
+  *out_host = v;
+  return AQ_OK;
+}
+
+int aq_status(aq_handle* h, uint32_t* bits_host) {
+  if (!h) return fail(nullptr, AQ_EINVAL, "null handle");
+  if (!bits_host) return fail(h, AQ_EINVAL, "aq_status: null pointer");
+  DeviceGuard g(h->device);
+  uint32_t v = 0;
+  AQ_CUDA(h, cudaMemcpyAsync(&v, h->st.status, sizeof(v), cudaMemcpyDeviceToHost, h->stream));
+  AQ_CUDA(h, cudaMemsetAsync(h->st.status, 0, sizeof(uint32_t), h->stream));
+  AQ_CUDA(h, cudaStreamSynchronize(h->stream));
+  *bits_host = v;
+  return AQ_OK;
+}
+
+const char* aq_last_error(aq_handle* h) { return h ? h->err : g_create_err; }
+
+int64_t aq_packed_bytes_per_sample(aq_handle* h) { return h ? h->st.packed_bytes : 0; }
+int64_t aq_scales_per_sample(aq_handle* h) { return h ? h->st.groups : 0; }
+
+int aq_encode_host(aq_handle* h, const void* act_host, const int32_t* sample_ids_host, void* packed_host,
+                   float* scales_host) {
+  if (!h) return fail(nullptr, AQ_EINVAL, "null handle");
+  if (h->n_batch == 0) return AQ_OK;
+  if (!act_host || !sample_ids_host || !packed_host || !scales_host) return fail(h, AQ_EINVAL, "aq_encode_host: null pointer");
+  DeviceGuard g(h->device);
+  int rc = ensure_staging(h);
+  if (rc != AQ_OK) return rc;
+  const size_t nb = (size_t)h->n_batch;
+  AQ_CUDA(h, cudaMemcpyAsync(h->d_act, act_host, nb * (size_t)h->st.elems * 2, cudaMemcpyHostToDevice, h->stream));
+  AQ_CUDA(h, cudaMemcpyAsync(h->d_ids, sample_ids_host, nb * sizeof(int32_t), cudaMemcpyHostToDevice, h->stream));
+  rc = aq_encode(h, h->d_act, h->d_ids, h->d_packed, h->d_scales);
+  if (rc != AQ_OK) return rc;
+  AQ_CUDA(h, cudaMemcpyAsync(packed_host, h->d_packed, nb * (size_t)h->st.packed_bytes, cudaMemcpyDeviceToHost, h->stream));
+  AQ_CUDA(h, cudaMemcpyAsync(scales_host, h->d_scales, nb * (size_t)h->st.groups * sizeof(float), cudaMemcpyDeviceToHost, h->stream));
+  AQ_CUDA(h, cudaStreamSynchronize(h->stream));
+  return AQ_OK;
+}
+
+int aq_decode_host(aq_handle* h, const void* packed_host, const float* scales_host, const void* raw_host,
+                   const int32_t* sample_ids_host, void* out_host) {
+  if (!h) return fail(nullptr, AQ_EINVAL, "null handle");
+  if (h->n_batch == 0) return AQ_OK;
+  if (!packed_host || !scales_host || !sample_ids_host || !out_host) return fail(h, AQ_EINVAL, "aq_decode_host: null pointer");
+  DeviceGuard g(h->device);
+  int rc = ensure_staging(h);
+  if (rc != AQ_OK) return rc;
+  const size_t nb = (size_t)h->n_batch;
+  const size_t act_bytes = nb * (size_t)h->st.elems * 2;
+  AQ_CUDA(h, cudaMemcpyAsync(h->d_packed, packed_host, nb * (size_t)h->st.packed_bytes, cudaMemcpyHostToDevice, h->stream));
+  AQ_CUDA(h, cudaMemcpyAsync(h->d_scales, scales_host, nb * (size_t)h->st.groups * sizeof(float), cudaMemcpyHostToDevice, h->stream));
+  AQ_CUDA(h, cudaMemcpyAsync(h->d_ids, sample_ids_host, nb * sizeof(int32_t), cudaMemcpyHostToDevice, h->stream));
+  // the staging block holds the raw message on the way in and the activation on the way out
+  // (every element is read before the same thread overwrites it)
+  if (raw_host) AQ_CUDA(h, cudaMemcpyAsync(h->d_act, raw_host, act_bytes, cudaMemcpyHostToDevice, h->stream));
+  const void* saved_raw = h->raw;
+  h->raw = raw_host ? h->d_act : nullptr;
+  rc = aq_decode(h, h->d_packed, h->d_scales, h->d_ids, h->d_act);
+  h->raw = saved_raw;
+  if (rc != AQ_OK) return rc;
+  AQ_CUDA(h, cudaMemcpyAsync(out_host, h->d_act, act_bytes, cudaMemcpyDeviceToHost, h->stream));
+  AQ_CUDA(h, cudaStreamSynchronize(h->stream));
+  return AQ_OK;
+}
+
+int aq_export_sample(aq_handle* h, int64_t sample_id, void* m_host, uint8_t* seen_host) {
+  if (!h) return fail(nullptr, AQ_EINVAL, "null handle");
+  if (sample_id < 0 || sample_id >= h->st.n_samples) return fail(h, AQ_EINVAL, "sample id out of range");
+  if (!m_host && !seen_host) return fail(h, AQ_EINVAL, "aq_export_sample: null pointers");
+  DeviceGuard g(h->device);
+  const size_t bytes = (size_t)h->st.elems * 2;
+  if (m_host)
+    AQ_CUDA(h, cudaMemcpyAsync(m_host, static_cast<const char*>(h->st.m) + (size_t)sample_id * bytes, bytes,
+                               cudaMemcpyDeviceToHost, h->stream));
+  if (seen_host)
+    AQ_CUDA(h, cudaMemcpyAsync(seen_host, h->st.seen + sample_id, 1, cudaMemcpyDeviceToHost, h->stream));
+  AQ_CUDA(h, cudaStreamSynchronize(h->stream));
+  return AQ_OK;
+}
+
+int aq_import_sample(aq_handle* h, int64_t sample_id, const void* m_host, uint8_t seen) {
+  if (!h) return fail(nullptr, AQ_EINVAL, "null handle");
+  if (sample_id < 0 || sample_id >= h->st.n_samples) return fail(h, AQ_EINVAL, "sample id out of range");
+  if (!m_host) return fail(h, AQ_EINVAL, "aq_import_sample: null pointer");
+  DeviceGuard g(h->device);
+  const size_t bytes = (size_t)h->st.elems * 2;
+  const uint8_t flag = seen ? 1 : 0;
+  AQ_CUDA(h, cudaMemcpyAsync(static_cast<char*>(h->st.m) + (size_t)sample_id * bytes, m_host, bytes,
+                             cudaMemcpyHostToDevice, h->stream));
+  AQ_CUDA(h, cudaMemcpyAsync(h->st.seen + sample_id, &flag, 1, cudaMemcpyHostToDevice, h->stream));
+  AQ_CUDA(h, cudaStreamSynchronize(h->stream));
+  return AQ_OK;
+}
+
+}  // extern "C"

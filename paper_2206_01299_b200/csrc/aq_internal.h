@@ -1,0 +1,56 @@
+// Launch-layer interface between the C ABI (aq_api.cu) and the kernels (aq_kernels.cu).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace aq {
+
+constexpr int kChunk = 8;            // elements per 128-bit access of a 2-byte type
+constexpr int kThreads = 256;        // threads per CTA
+constexpr int kChunksPerThread = 2;  // independent 128-bit chunks in flight per thread
+
+// State of one side of a boundary, as the kernels see it.
+struct State {
+  void* m;                 // T[n_samples][elems]
+  uint8_t* seen;           // [n_samples]
+  uint32_t* status;        // sticky AQ_ST_* bits
+  uint32_t* ticket;        // CTA arrival counter of the running call (returns to 0 by itself)
+  long long n_samples;
+  long long elems;         // seq * hidden
+  long long chunks;        // elems / 8
+  long long packed_bytes;  // per sample
+  long long groups;        // per sample
+  int lanes_per_group;     // group / 8, a power of two <= 32
+  int lg_shift;            // log2(lanes_per_group)
+};
+
+struct EncodeArgs {
+  const void* act;
+  const int32_t* ids;
+  uint8_t* packed;
+  float* scales;
+  uint8_t* first_flags;    // may be null
+  int n_batch;
+};
+
+struct DecodeArgs {
+  const uint8_t* packed;
+  const float* scales;
+  const void* raw;         // may be null
+  const int32_t* ids;
+  void* out;
+  uint8_t* first_flags;    // may be null
+  int n_batch;
+};
+
+cudaError_t launch_encode(int dtype, int bits, const State& st, const EncodeArgs& a, cudaStream_t s);
+cudaError_t launch_decode(int dtype, int bits, const State& st, const DecodeArgs& a, cudaStream_t s);
+cudaError_t launch_quant_grad(int dtype, int bits, int lanes_per_group, const void* grad,
+                              long long n_elems, uint8_t* packed, float* scales, cudaStream_t s);
+cudaError_t launch_dequant_grad(int dtype, int bits, int lanes_per_group, const uint8_t* packed,
+                                const float* scales, long long n_elems, void* out, cudaStream_t s);
+// *sum_dev += digest of (m, seen); the caller zeroes *sum_dev first.
+cudaError_t launch_checksum(const State& st, unsigned long long* sum_dev, cudaStream_t s);
+
+}  // namespace aq

@@ -1,0 +1,276 @@
+"""CUDA library against the CPU oracle, element by element, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2206_01299_b200 as aq
+from paper_2206_01299_b200 import synth
+from codec_harness import DT, GpuSide, bits16, run_boundary
+
+pytestmark = pytest.mark.gpu
+
+
+# ----------------------------------------------------------------- backward direction (stateless)
+
+def _grad_input(n, group, dtype, seed):
+    g = torch.Generator(device="cpu").manual_seed(seed)
+    x = torch.randn(n, generator=g) * 1e-3
+    spikes = torch.rand(n, generator=g) < 0.01
+    x = torch.where(spikes, x * 100, x)
+    xg = x.view(-1, group)
+    if xg.shape[0] >= 8:
+        xg[1] = 0.0                                   # an all-zero group
+        xg[2] = 1e-41                                  # a vanishing group: step below FLT_MIN
+        xg[3, 0] = -0.0
+        xg[4] = 2.0 ** -120                            # tiny but live
+        xg[5] = torch.arange(group) - group / 2        # exact interval edges
+    return x.to(dtype)
+
+
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+@pytest.mark.parametrize("bits", range(1, 9))
+@pytest.mark.parametrize("group,n_groups", [(8, 1), (8, 333), (64, 4097), (128, 777), (256, 130)])
+def test_quant_and_dequant_grad_match_oracle(dtype, bits, group, n_groups):
+    td = torch.float16 if dtype == "fp16" else torch.bfloat16
+    n = group * n_groups                               # ragged: not a multiple of the CTA tile
+    h = aq.aq_create(1, 1, group, 4, group)
+    try:
+        aq.aq_configure(h, aq.AQ_DTYPE, DT[dtype][0])
+        grad = _grad_input(n, group, td, bits * 1000 + group).cuda()
+        packed = torch.full((n * bits // 8 + 16,), 0xCD, dtype=torch.uint8, device="cuda")
+        scales = torch.full((n // group + 4,), -3.0, dtype=torch.float32, device="cuda")
+        out = torch.full((n + 8,), 5.0, dtype=td, device="cuda")
+        aq.aq_quant_grad(h, grad, n, bits, packed, scales)
+        aq.aq_dequant_grad(h, packed, scales, n, bits, out)
+        torch.cuda.synchronize()
+        p_o, s_o = oracle.quant_grad(bits16(grad), bits, group, DT[dtype][1])
+        o_o = oracle.dequant_grad(p_o, s_o, n, bits, group, DT[dtype][1])
+        assert np.array_equal(packed.cpu().numpy()[: n * bits // 8], p_o)
+        assert np.array_equal(scales.cpu().numpy()[: n // group].view(np.uint32), s_o.view(np.uint32))
+        assert np.array_equal(bits16(out)[:n], o_o)
+        # nothing written past the ends
+        assert (packed.cpu().numpy()[n * bits // 8:] == 0xCD).all()
+        assert (scales.cpu().numpy()[n // group:] == -3.0).all()
+        assert (out.float().cpu().numpy()[n:] == 5.0).all()
+    finally:
+        aq.aq_destroy(h)
+
+
+def test_backward_workload_full_size():
+    """Config 'Backward path': 4 x 1024 x 1600 fp16 gradients, 8-bit and 4-bit, group 64."""
+    cfg = synth.BACKWARD
+    h = aq.aq_create(1, 1, cfg.group, 4, cfg.group)
+    try:
+        grad = synth.gradient(cfg, 0, device="cuda")
+        n = cfg.elems
+        g_np = bits16(grad)
+        for bits in cfg.bits:
+            packed = torch.empty(n * bits // 8, dtype=torch.uint8, device="cuda")
+            scales = torch.empty(n // cfg.group, dtype=torch.float32, device="cuda")
+            out = torch.empty(n, dtype=torch.float16, device="cuda")
+            aq.aq_quant_grad(h, grad, n, bits, packed, scales)
+            aq.aq_dequant_grad(h, packed, scales, n, bits, out)
+            torch.cuda.synchronize()
+            p_o, s_o = oracle.quant_grad(g_np, bits, cfg.group, oracle.FP16)
+            o_o = oracle.dequant_grad(p_o, s_o, n, bits, cfg.group, oracle.FP16)
+            assert np.array_equal(packed.cpu().numpy(), p_o)
+            assert np.array_equal(scales.cpu().numpy().view(np.uint32), s_o.view(np.uint32))
+            assert np.array_equal(bits16(out), o_o)
+    finally:
+        aq.aq_destroy(h)
+
+
+def test_gradient_inputs_are_identical_on_cpu_and_gpu():
+    cfg = synth.GradWorkload("g", 1, 16, 1600, "fp16", (4,), 64, seed=9)
+    assert np.array_equal(bits16(synth.gradient(cfg, 3, "cuda")), bits16(synth.gradient(cfg, 3, "cpu")))
+    b = synth.shrink(synth.DEBERTA_XXL, 8, seq=8)
+    assert np.array_equal(bits16(synth.activation(b, [5, 2], 2, "cuda")), bits16(synth.activation(b, [5, 2], 2, "cpu")))
+
+
+# ----------------------------------------------------------------- forward boundary (stateful)
+
+def test_tiny_boundary_all_epochs():
+    """Config 'Tiny boundary', complete: 64 ids, 4 x 128 x 768 fp16, 2 bit, group 128, 3 epochs."""
+    run_boundary(synth.TINY)
+
+
+def test_gpt2_shaped_boundary_reduced_id_space():
+    """Config 'GPT2-1.5B-shaped boundary' with 8 ids instead of 4096 (same per-call shape)."""
+    run_boundary(synth.shrink(synth.GPT2_XL, 8, epochs=3))
+
+
+def test_gpt2_shaped_boundary_batched_launch():
+    run_boundary(synth.shrink(synth.GPT2_XL, 8, seq=192, epochs=3), n_batch=4)
+
+
+def test_deberta_shaped_boundary_reduced_id_space():
+    """Config 'DeBERTa-1.5B-shaped boundary' with 16 ids: bf16, 2 bit, group 128, micro-batch 8."""
+    run_boundary(synth.shrink(synth.DEBERTA_XXL, 16))
+
+
+def test_sweep_forward_three_bit_reduced_id_space():
+    """Forward half of the 'Pipeline sweep' config: 3-bit delta, group 64 (fields straddle bytes)."""
+    run_boundary(synth.shrink(synth.SWEEP_FWD, 4, seq=256))
+
+
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+@pytest.mark.parametrize("bits", range(1, 9))
+def test_every_bit_width_on_ragged_shapes(dtype, bits):
+    # 37 x 136 elements: 629 chunks per sample -- not a multiple of a warp or of a CTA tile
+    cfg = synth.Boundary("ragged", 6, 3, 37, 136, dtype, bits, 8, 3, "outlier", 0.3, seed=20 + bits)
+    run_boundary(cfg)
+    # one chunk per sample; the stream of a sample is `bits` bytes long
+    cfg = synth.Boundary("one-chunk", 4, 2, 1, 8, dtype, bits, 8, 3, "normal", 0.5, seed=40 + bits)
+    run_boundary(cfg)
+
+
+@pytest.mark.parametrize("group", [16, 32, 256])
+def test_other_group_sizes(group):
+    cfg = synth.Boundary("groups", 4, 2, 5, 1024, "fp16", 4, group, 3, "outlier", 0.1, seed=group)
+    run_boundary(cfg)
+    cfg = synth.Boundary("groups3", 4, 2, 5, 1024, "bf16", 3, group, 3, "student_t3", 0.1, seed=group)
+    run_boundary(cfg)
+
+
+def test_revisits_of_an_unchanged_activation_send_zeros():
+    cfg = synth.Boundary("still", 4, 2, 4, 256, "fp16", 4, 64, 3, "normal", 0.0, seed=77)
+
+    def act_fn(ids, epoch):
+        return synth.activation(cfg, ids, 0, device="cuda")
+
+    run_boundary(cfg, act_fn=act_fn)
+    side = GpuSide(cfg, 2)
+    try:
+        ids = torch.tensor([1, 3], dtype=torch.int32, device="cuda")
+        act = act_fn(ids.cpu(), 0)
+        packed = torch.full((2, cfg.packed_bytes), 9, dtype=torch.uint8, device="cuda")
+        scales = torch.full((2, cfg.groups), 9.0, device="cuda")
+        aq.aq_encode(side.h, act, ids, packed, scales)
+        aq.aq_encode(side.h, act, ids, packed, scales)
+        torch.cuda.synchronize()
+        assert not packed.any() and not scales.any()
+        assert np.array_equal(side.m_row(3)[0], bits16(act[1]))
+    finally:
+        side.close()
+
+
+# ----------------------------------------------------------------- error paths and empty inputs
+
+def test_bad_duplicate_and_rawless_ids_are_skipped_like_the_oracle():
+    cfg = synth.Boundary("err", 5, 4, 2, 64, "fp16", 2, 64, 1, "normal", 0.1, seed=5)
+    gs, gr = GpuSide(cfg, 4), GpuSide(cfg, 4)
+    os_, or_ = (oracle.Side(5, 2, 64, 2, 64, oracle.FP16) for _ in range(2))
+    try:
+        packed = torch.empty((4, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
+        scales = torch.empty((4, cfg.groups), dtype=torch.float32, device="cuda")
+        out = torch.empty((4, 2, 64), dtype=torch.float16, device="cuda")
+        for step, id_list in enumerate([[1, 7, 1, 3], [3, -1, 1, 3], [0, 1, 2, 3]]):
+            ids = torch.tensor(id_list, dtype=torch.int32)
+            act = synth.activation(cfg, torch.tensor([10, 11, 12, 13]), step, device="cuda")
+            packed.fill_(1)
+            scales.fill_(1)
+            out.fill_(1)
+            aq.aq_encode(gs.h, act, ids.cuda(), packed, scales)
+            raw = act if step != 2 else None                      # last step: first visits without a raw message
+            aq.aq_configure(gr.h, aq.AQ_RAW, raw)
+            aq.aq_decode(gr.h, packed, scales, ids.cuda(), out)
+            torch.cuda.synchronize()
+            p_o, s_o, f_o = os_.encode(bits16(act), ids.numpy())
+            out_o, fr_o = or_.decode(p_o, s_o, ids.numpy(), raw=bits16(act) if raw is not None else None)
+            assert np.array_equal(packed.cpu().numpy(), p_o)
+            assert np.array_equal(scales.cpu().numpy(), s_o)
+            assert np.array_equal(bits16(out), out_o)
+            assert np.array_equal(gs.first.cpu().numpy(), f_o) and np.array_equal(gr.first.cpu().numpy(), fr_o)
+            st_s, st_r = aq.aq_status(gs.h), aq.aq_status(gr.h)
+            assert st_s == os_.status() and st_r == or_.status()
+            assert aq.aq_status(gs.h) == 0                          # reading clears
+            assert np.array_equal(gs.m_all(), os_.m()) and np.array_equal(gr.m_all(), or_.m())
+            assert aq.aq_state_checksum(gs.h) == os_.checksum()
+            assert aq.aq_state_checksum(gr.h) == or_.checksum()
+        assert st_r & aq.AQ_ST_NO_RAW
+    finally:
+        gs.close()
+        gr.close()
+
+
+def test_host_side_argument_errors():
+    with pytest.raises(aq.AqError):
+        aq.aq_create(4, 2, 100, 4, 64)          # group does not divide hidden
+    with pytest.raises(aq.AqError):
+        aq.aq_create(4, 2, 96, 4, 24)           # unsupported group
+    with pytest.raises(aq.AqError):
+        aq.aq_create(0, 2, 64, 4, 64)
+    h = aq.aq_create(4, 2, 64, 4, 64)
+    try:
+        t = torch.zeros(256, dtype=torch.float16, device="cuda")
+        ids = torch.zeros(1, dtype=torch.int32, device="cuda")
+        with pytest.raises(aq.AqError) as e:
+            aq.aq_encode(h, None, ids, t, t)
+        assert e.value.code == aq.AQ_EINVAL
+        with pytest.raises(aq.AqError):
+            aq.aq_encode(h, t.data_ptr() + 2, ids, t, t)          # misaligned
+        with pytest.raises(aq.AqError):
+            aq.aq_quant_grad(h, t, 100, 4, t, t)                  # not a multiple of the group
+        with pytest.raises(aq.AqError):
+            aq.aq_quant_grad(h, t, 128, 0, t, t)
+        with pytest.raises(aq.AqError):
+            aq.aq_configure(h, aq.AQ_BATCH, 70000)
+        with pytest.raises(aq.AqError):
+            aq.aq_configure(h, 99, 0)
+        # empty inputs are no-ops
+        aq.aq_quant_grad(h, None, 0, 4, None, None)
+        aq.aq_dequant_grad(h, None, None, 0, 4, None)
+        aq.aq_configure(h, aq.AQ_BATCH, 0)
+        aq.aq_encode(h, None, None, None, None)
+        aq.aq_decode(h, None, None, None, None)
+        assert aq.aq_status(h) == 0
+        assert aq.aq_packed_bytes_per_sample(h) == 64 and aq.aq_scales_per_sample(h) == 2
+    finally:
+        aq.aq_destroy(h)
+
+
+def test_non_default_stream_and_host_buffer_forms():
+    cfg = synth.Boundary("host", 6, 3, 9, 192, "bf16", 3, 64, 3, "normal", 0.05, seed=31)
+    stream = torch.cuda.Stream()
+    gs, gr = GpuSide(cfg, 3, stream), GpuSide(cfg, 3, stream)
+    os_, or_ = (oracle.Side(6, 9, 192, 3, 64, oracle.BF16) for _ in range(2))
+    try:
+        for epoch in range(3):
+            order = synth.epoch_order(cfg, epoch)
+            for c in range(2):
+                ids = order[c * 3:(c + 1) * 3].contiguous()
+                act = synth.activation(cfg, ids, epoch).pin_memory()
+                packed = torch.empty((3, cfg.packed_bytes), dtype=torch.uint8).pin_memory()
+                scales = torch.empty((3, cfg.groups), dtype=torch.float32).pin_memory()
+                out = torch.empty_like(act).pin_memory()
+                aq.aq_encode_host(gs.h, act, ids, packed, scales)
+                aq.aq_decode_host(gr.h, packed, scales, act if epoch == 0 else None, ids, out)
+                p_o, s_o, _ = os_.encode(bits16(act), ids.numpy())
+                out_o, _ = or_.decode(p_o, s_o, ids.numpy(), raw=bits16(act))
+                assert np.array_equal(packed.numpy(), p_o) and np.array_equal(scales.numpy(), s_o)
+                assert np.array_equal(bits16(out), out_o)
+        assert aq.aq_state_checksum(gs.h) == aq.aq_state_checksum(gr.h) == os_.checksum()
+        assert np.array_equal(gr.m_all(), or_.m())
+    finally:
+        gs.close()
+        gr.close()
+
+
+def test_import_export_round_trip():
+    cfg = synth.Boundary("ckpt", 3, 1, 4, 64, "fp16", 4, 64, 1, "normal", 0.1, seed=8)
+    a, b = GpuSide(cfg, 1), GpuSide(cfg, 1)
+    try:
+        ids = torch.tensor([2], dtype=torch.int32, device="cuda")
+        act = synth.activation(cfg, [2], 0, device="cuda")
+        p = torch.empty((1, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
+        s = torch.empty((1, cfg.groups), dtype=torch.float32, device="cuda")
+        aq.aq_encode(a.h, act, ids, p, s)
+        for i in range(3):
+            row, seen = a.m_row(i)
+            aq.aq_import_sample(b.h, i, row, seen)
+        assert aq.aq_state_checksum(a.h) == aq.aq_state_checksum(b.h)
+        assert b.m_row(2)[1] == 1 and b.m_row(0)[1] == 0
+    finally:
+        a.close()
+        b.close()
