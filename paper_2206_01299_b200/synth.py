@@ -151,12 +151,8 @@ def outlier_channels(cfg: Boundary, count: int = 4) -> torch.Tensor:
     return torch.argsort(_fmix(ch * _s64(_PHI) + _s64(k)), stable=True)[:count]
 
 
-def activation(cfg: Boundary, ids, epoch: int, device="cpu") -> torch.Tensor:
-    """a(xi) at the given epoch for each id: tensor [len(ids), seq, hidden] of cfg's dtype.
-
-    A_0 follows cfg.kind; A_e = A_{e-1} + drift * z_e accumulated in fp32; the
-    result is A_epoch rounded to the 16-bit type.
-    """
+def base_f32(cfg: Boundary, ids, device="cpu") -> torch.Tensor:
+    """A_0 in fp32 for each id: tensor [len(ids), seq*hidden]."""
     ids = torch.as_tensor(ids, dtype=torch.int64, device=device).reshape(-1)
     ctr = torch.arange(cfg.elems, dtype=torch.int64, device=device).reshape(1, -1)
     key0 = _sample_keys(cfg.seed, cfg.stream, 0, ids)
@@ -168,16 +164,32 @@ def activation(cfg: Boundary, ids, epoch: int, device="cpu") -> torch.Tensor:
             sq = z * z
             acc = sq if acc is None else acc + sq
         a = z0 / torch.sqrt(acc / 3.0)
-        a = torch.clamp(a, -1.0e4, 1.0e4)
-    else:
-        a = _normal(key0, ctr, 0)
-        if cfg.kind == "outlier":
-            gain = torch.ones(cfg.hidden, dtype=torch.float32, device=device)
-            gain[outlier_channels(cfg).to(device)] = 20.0
-            a = (a.reshape(-1, cfg.seq, cfg.hidden) * gain).reshape(-1, cfg.elems)
+        return torch.clamp(a, -1.0e4, 1.0e4)
+    a = _normal(key0, ctr, 0)
+    if cfg.kind == "outlier":
+        gain = torch.ones(cfg.hidden, dtype=torch.float32, device=device)
+        gain[outlier_channels(cfg).to(device)] = 20.0
+        a = (a.reshape(-1, cfg.seq, cfg.hidden) * gain).reshape(-1, cfg.elems)
+    return a
+
+
+def advance_f32(cfg: Boundary, a: torch.Tensor, ids, epoch: int) -> torch.Tensor:
+    """A_epoch = A_{epoch-1} + drift * z_epoch, one fp32 multiply and one fp32 add per element."""
+    ids = torch.as_tensor(ids, dtype=torch.int64, device=a.device).reshape(-1)
+    ctr = torch.arange(cfg.elems, dtype=torch.int64, device=a.device).reshape(1, -1)
+    z = _normal(_sample_keys(cfg.seed, cfg.stream, epoch, ids), ctr, 0)
+    return a + z * cfg.drift
+
+
+def activation(cfg: Boundary, ids, epoch: int, device="cpu") -> torch.Tensor:
+    """a(xi) at the given epoch for each id: tensor [len(ids), seq, hidden] of cfg's dtype.
+
+    A_0 follows cfg.kind; A_e = A_{e-1} + drift * z_e accumulated in fp32; the
+    result is A_epoch rounded to the 16-bit type.
+    """
+    a = base_f32(cfg, ids, device)
     for e in range(1, epoch + 1):
-        z = _normal(_sample_keys(cfg.seed, cfg.stream, e, ids), ctr, 0)
-        a = a + z * cfg.drift
+        a = advance_f32(cfg, a, ids, e)
     return a.to(cfg.torch_dtype).reshape(-1, cfg.seq, cfg.hidden)
 
 
