@@ -45,6 +45,7 @@ def parse_args():
     ap.add_argument("--n-samples", type=int, default=None, help="shrink the id space (profiling runs)")
     ap.add_argument("--per-launch", type=int, default=MACRO, help="micro-batches handed to one aq_encode call")
     ap.add_argument("--graph", action="store_true", help="replay each step as a captured CUDA graph")
+    ap.add_argument("--rows-per-cta", type=int, default=0, help="AQ_ROWS_PER_CTA of both handles (0 = library default)")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-aux", action="store_true")
@@ -256,6 +257,8 @@ def main():
         h = aq.aq_create(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group)
         aq.aq_configure(h, aq.AQ_BATCH, nb)
         aq.aq_configure(h, aq.AQ_STREAM, stream.cuda_stream)
+        if args.rows_per_cta:
+            aq.aq_configure(h, aq.AQ_ROWS_PER_CTA, args.rows_per_cta)
         handles.append(h)
     snd, rcv = handles
 

@@ -72,12 +72,14 @@ enum {
 /* keys of aq_configure */
 enum {
   AQ_DTYPE = 1,          /* AQ_FP16 (default) or AQ_BF16: type T of activations, gradients and m */
-  AQ_BATCH = 2,          /* n_batch: sequences per aq_encode / aq_decode call, 0..65535 (default 1) */
+  AQ_BATCH = 2,          /* n_batch: sequences per aq_encode / aq_decode call, 0..4096 (default 1) */
   AQ_STREAM = 3,         /* cudaStream_t as an integer (default 0, the legacy default stream) */
   AQ_RAW = 4,            /* device pointer T[n_batch][seq][hidden]: the uncompressed message that
                             aq_decode stores for first-visit samples; 0 = none (default) */
-  AQ_FIRST_FLAGS = 5     /* device pointer uint8[n_batch] or 0: aq_encode / aq_decode write 1 for
+  AQ_FIRST_FLAGS = 5,    /* device pointer uint8[n_batch] or 0: aq_encode / aq_decode write 1 for
                             each sample that took the first-visit path, else 0 */
+  AQ_ROWS_PER_CTA = 6    /* tuning: rows (256 chunks = 2048 elements each) that one CTA of aq_encode /
+                            aq_decode walks; 0 (default) = sized so that the grid is one wave of CTAs */
 };
 enum { AQ_FP16 = 0, AQ_BF16 = 1 };
 

@@ -98,6 +98,8 @@ aq_handle* aq_create(int64_t n_samples, int seq, int hidden, int bits, int group
   g_create_err[0] = 0;
   const int lanes = lanes_for_group(group);
   if (n_samples <= 0 || seq <= 0 || hidden <= 0) { fail(nullptr, AQ_EINVAL, "n_samples, seq and hidden must be positive"); return nullptr; }
+  if (n_samples > 0x7fffffffll) { fail(nullptr, AQ_EINVAL, "n_samples must fit the int32 sample ids"); return nullptr; }
+  if ((long long)seq * hidden > (1ll << 30)) { fail(nullptr, AQ_EINVAL, "seq*hidden must not exceed 2^30 elements per sample"); return nullptr; }
   if (bits < 1 || bits > 8) { fail(nullptr, AQ_EINVAL, "bits must be in 1..8 (got %d)", bits); return nullptr; }
   if (!lanes) { fail(nullptr, AQ_EINVAL, "group must be one of 8,16,32,64,128,256 (got %d)", group); return nullptr; }
   if (hidden % group) { fail(nullptr, AQ_EINVAL, "group %d does not divide hidden %d", group, hidden); return nullptr; }
@@ -107,20 +109,26 @@ aq_handle* aq_create(int64_t n_samples, int seq, int hidden, int bits, int group
   aq::State& st = h->st;
   st.n_samples = n_samples;
   st.elems = (long long)seq * hidden;
-  st.chunks = st.elems / aq::kChunk;
+  st.chunks = (int)(st.elems / aq::kChunk);
+  st.rows = (st.chunks + aq::kThreads - 1) / aq::kThreads;
   st.packed_bytes = st.elems * bits / 8;
   st.groups = st.elems / group;
   st.lanes_per_group = lanes;
   st.lg_shift = __builtin_ctz((unsigned)lanes);
   cudaError_t e = cudaGetDevice(&h->device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&st.sms, cudaDevAttrMultiProcessorCount, h->device);
   const size_t m_bytes = (size_t)n_samples * (size_t)st.elems * 2;
+  const size_t seen_bytes = (size_t)n_samples * sizeof(unsigned long long);
+  const unsigned long long first_call = aq::kFirstCall;
   if (e == cudaSuccess) e = cudaMalloc(&st.m, m_bytes);
-  if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&st.seen), (size_t)n_samples);
+  if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&st.seen), seen_bytes);
+  if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&st.call_no), sizeof(unsigned long long));
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&st.status), 2 * sizeof(uint32_t));
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&h->sum_dev), sizeof(unsigned long long));
   if (e == cudaSuccess) e = cudaMemset(st.m, 0, m_bytes);                      // "initialized to 0"
-  if (e == cudaSuccess) e = cudaMemset(st.seen, 0, (size_t)n_samples);
+  if (e == cudaSuccess) e = cudaMemset(st.seen, 0, seen_bytes);
   if (e == cudaSuccess) e = cudaMemset(st.status, 0, 2 * sizeof(uint32_t));
+  if (e == cudaSuccess) e = cudaMemcpy(st.call_no, &first_call, sizeof(first_call), cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
     cuda_fail(nullptr, e, "aq_create");
@@ -139,6 +147,7 @@ void aq_destroy(aq_handle* h) {
   free_staging(h);
   cudaFree(h->st.m);
   cudaFree(h->st.seen);
+  cudaFree(h->st.call_no);
   cudaFree(h->st.status);
   cudaFree(h->sum_dev);
   delete h;
@@ -152,7 +161,7 @@ int aq_configure(aq_handle* h, int key, int64_t value) {
       h->dtype = (int)value;
       return AQ_OK;
     case AQ_BATCH:
-      if (value < 0 || value > 65535) return fail(h, AQ_EINVAL, "AQ_BATCH must be in 0..65535");
+      if (value < 0 || value > aq::kMaxBatch) return fail(h, AQ_EINVAL, "AQ_BATCH must be in 0..%d", aq::kMaxBatch);
       h->n_batch = (int)value;
       return AQ_OK;
     case AQ_STREAM:
@@ -164,6 +173,10 @@ int aq_configure(aq_handle* h, int key, int64_t value) {
       return AQ_OK;
     case AQ_FIRST_FLAGS:
       h->first_flags = reinterpret_cast<uint8_t*>(static_cast<intptr_t>(value));
+      return AQ_OK;
+    case AQ_ROWS_PER_CTA:
+      if (value < 0 || value > (1 << 20)) return fail(h, AQ_EINVAL, "AQ_ROWS_PER_CTA must be in 0..2^20");
+      h->st.rows_per_cta = (int)value;
       return AQ_OK;
     default:
       return fail(h, AQ_EINVAL, "unknown configure key %d", key);
@@ -306,9 +319,11 @@ int aq_export_sample(aq_handle* h, int64_t sample_id, void* m_host, uint8_t* see
   if (m_host)
     AQ_CUDA(h, cudaMemcpyAsync(m_host, static_cast<const char*>(h->st.m) + (size_t)sample_id * bytes, bytes,
                                cudaMemcpyDeviceToHost, h->stream));
+  unsigned long long stamp = 0;
   if (seen_host)
-    AQ_CUDA(h, cudaMemcpyAsync(seen_host, h->st.seen + sample_id, 1, cudaMemcpyDeviceToHost, h->stream));
+    AQ_CUDA(h, cudaMemcpyAsync(&stamp, h->st.seen + sample_id, sizeof(stamp), cudaMemcpyDeviceToHost, h->stream));
   AQ_CUDA(h, cudaStreamSynchronize(h->stream));
+  if (seen_host) *seen_host = stamp != 0 ? 1 : 0;
   return AQ_OK;
 }
 
@@ -318,10 +333,10 @@ int aq_import_sample(aq_handle* h, int64_t sample_id, const void* m_host, uint8_
   if (!m_host) return fail(h, AQ_EINVAL, "aq_import_sample: null pointer");
   DeviceGuard g(h->device);
   const size_t bytes = (size_t)h->st.elems * 2;
-  const uint8_t flag = seen ? 1 : 0;
+  const unsigned long long stamp = seen ? aq::kImportedStamp : 0ull;
   AQ_CUDA(h, cudaMemcpyAsync(static_cast<char*>(h->st.m) + (size_t)sample_id * bytes, m_host, bytes,
                              cudaMemcpyHostToDevice, h->stream));
-  AQ_CUDA(h, cudaMemcpyAsync(h->st.seen + sample_id, &flag, 1, cudaMemcpyHostToDevice, h->stream));
+  AQ_CUDA(h, cudaMemcpyAsync(h->st.seen + sample_id, &stamp, sizeof(stamp), cudaMemcpyHostToDevice, h->stream));
   AQ_CUDA(h, cudaStreamSynchronize(h->stream));
   return AQ_OK;
 }

@@ -7,22 +7,34 @@
 namespace aq {
 
 constexpr int kChunk = 8;            // elements per 128-bit access of a 2-byte type
-constexpr int kThreads = 256;        // threads per CTA
-constexpr int kChunksPerThread = 2;  // independent 128-bit chunks in flight per thread
+constexpr int kThreads = 256;        // threads per CTA; one "row" = kThreads consecutive chunks
+constexpr int kRowsPerIter = 2;      // rows a CTA has in flight per loop iteration
+constexpr int kMaxBatch = 4096;      // samples per encode / decode call
+
+// "Seen before" is kept as a stamp per sample: 0 = never seen, otherwise the number of the
+// call that saw it first (kImportedStamp for a sample loaded through aq_import_sample).  A
+// sample whose stamp equals the number of the running call is still a first visit for every
+// CTA of that call, so the stamp may be written while other CTAs are reading it.
+constexpr unsigned long long kImportedStamp = 1ull;
+constexpr unsigned long long kFirstCall = 2ull;
 
 // State of one side of a boundary, as the kernels see it.
 struct State {
-  void* m;                 // T[n_samples][elems]
-  uint8_t* seen;           // [n_samples]
-  uint32_t* status;        // sticky AQ_ST_* bits
-  uint32_t* ticket;        // CTA arrival counter of the running call (returns to 0 by itself)
+  void* m;                        // T[n_samples][elems]
+  unsigned long long* seen;       // [n_samples] stamps
+  unsigned long long* call_no;    // number of the next encode / decode call (starts at kFirstCall)
+  uint32_t* status;               // sticky AQ_ST_* bits
+  uint32_t* ticket;               // CTA arrival counter of the running call (returns to 0 by itself)
   long long n_samples;
-  long long elems;         // seq * hidden
-  long long chunks;        // elems / 8
-  long long packed_bytes;  // per sample
-  long long groups;        // per sample
-  int lanes_per_group;     // group / 8, a power of two <= 32
-  int lg_shift;            // log2(lanes_per_group)
+  long long elems;                // seq * hidden
+  long long packed_bytes;         // per sample
+  long long groups;               // per sample
+  int chunks;                     // elems / 8
+  int rows;                       // ceil(chunks / kThreads): rows per sample
+  int lanes_per_group;            // group / 8, a power of two <= 32
+  int lg_shift;                   // log2(lanes_per_group)
+  int sms;                        // multiprocessors of the handle's device
+  int rows_per_cta;               // 0 = one wave of CTAs (default); > 0 = fixed rows per CTA
 };
 
 struct EncodeArgs {

@@ -1,16 +1,22 @@
 // sm_100a kernels of the AQ-SGD boundary codec: fused encode, fused decode,
 // gradient quantize / dequantize, state digest.
 //
-// The path is bound by HBM traffic (about 6.5 bytes per element against roughly
-// 20 arithmetic instructions), so the design is about memory: every thread moves
-// 128-bit pieces ("chunks" of 8 elements of a 2-byte type) with several
-// independent loads in flight, the group maximum is a shuffle reduction over the
-// 8 or 16 lanes that hold one group, codes leave as whole 32-bit words, and m is
-// read and rewritten in place by the same thread in one pass.
+// The path is bound by HBM traffic (about 6.5 bytes per element), with the issue slots
+// of the SMs as the second limit (about 36 thread-instructions per element are available
+// at the memory roofline), so the design is about both: every thread moves 128-bit pieces
+// ("chunks" of 8 elements of a 2-byte type) with several independent loads in flight, the
+// group maximum is a shuffle reduction over the 8 or 16 lanes that hold one group, codes
+// leave as whole 32-bit words, m is read and rewritten in place by the same thread in one
+// pass, and the quantizer core is written for few instructions (see quantize8).
 //
-// Arithmetic: one IEEE binary32 rounding per operation (explicit _rn / _rd
-// intrinsics, never contracted into a fused multiply-add), so the result is
-// defined bit for bit.
+// encode / decode run as one wave of CTAs; each CTA walks a contiguous range of "rows"
+// (256 consecutive chunks of one sample), so the per-sample work (id lookup, first-visit
+// test) is done once per CTA and sample, by every warp for itself: the kernels have one
+// block barrier, at their start, and no wait on another CTA.
+//
+// Arithmetic: one IEEE binary32 rounding per operation (explicit _rn / _rd intrinsics;
+// the one explicit fused multiply-add is exact-equivalent, see quantize8), so the result
+// is defined bit for bit.
 
 #include "aq_internal.h"
 
@@ -22,6 +28,7 @@ namespace aq {
 namespace {
 
 constexpr unsigned kFullMask = 0xffffffffu;
+constexpr int kChunksPerThread = 2;                      // grad kernels: chunks per thread
 constexpr int kChunksPerCta = kThreads * kChunksPerThread;
 
 enum { kModeDelta = 0, kModeFirst = 1, kModeSkip = 2 };
@@ -32,6 +39,9 @@ enum { kStBadId = 1, kStDupId = 2, kStNoRaw = 4 };
 template <typename T> struct Conv;
 
 template <> struct Conv<__half> {
+  // |a - m| < 2^17 and every non-zero difference is >= 2^-24: the step Delta and its
+  // reciprocal are normal numbers, far from the ends of the binary32 range.
+  static constexpr bool kWide = false;
   static __device__ __forceinline__ void unpack(const uint4& v, float (&f)[8]) {
     const __half2* h = reinterpret_cast<const __half2*>(&v);
 #pragma unroll
@@ -51,6 +61,7 @@ template <> struct Conv<__half> {
 };
 
 template <> struct Conv<__nv_bfloat16> {
+  static constexpr bool kWide = true;      // full binary32 exponent range
   static __device__ __forceinline__ void unpack(const uint4& v, float (&f)[8]) {
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
@@ -70,9 +81,16 @@ template <> struct Conv<__nv_bfloat16> {
 
 // ------------------------------------------------------------------ quantizer core
 
-// Largest magnitude over the lanes_per_group consecutive lanes that hold one group.
+// Largest magnitude over the LPG consecutive lanes that hold one group (LPG = 0: the
+// lane count is only known at run time).
+template <int LPG>
 __device__ __forceinline__ float group_max(float s, int lanes_per_group) {
-  for (int o = lanes_per_group >> 1; o > 0; o >>= 1) s = fmaxf(s, __shfl_xor_sync(kFullMask, s, o));
+  if constexpr (LPG == 0) {
+    for (int o = lanes_per_group >> 1; o > 0; o >>= 1) s = fmaxf(s, __shfl_xor_sync(kFullMask, s, o));
+  } else {
+#pragma unroll
+    for (int o = LPG >> 1; o > 0; o >>= 1) s = fmaxf(s, __shfl_xor_sync(kFullMask, s, o));
+  }
   return s;
 }
 
@@ -83,34 +101,78 @@ __device__ __forceinline__ float abs_max8(const float (&d)[8]) {
   return s;
 }
 
+// sum over i < n of x << (i * bits)
+__host__ __device__ constexpr uint32_t spread(uint32_t x, int n, int bits) {
+  uint32_t r = 0;
+  for (int i = 0; i < n; ++i) r += x << (i * bits);
+  return r;
+}
+
+// n biased words t_i = 0x4B400000 + k_i  ->  the n two's-complement fields k_i mod 2^b laid
+// end to end (field i at bit i*b), n*b <= 32.  Horner's rule in wrapping 32-bit arithmetic
+// gives sum t_i 2^(ib); adding (h - 0x4B400000) * sum 2^(ib), h = 2^(b-1), turns every
+// term into the offset code k_i + h in [0, 2^b), which cannot borrow from its neighbour;
+// flipping the top bit of each field turns offset codes into two's complement.
+template <int BITS, int N>
+__device__ __forceinline__ uint32_t pack_fields(const uint32_t* tb) {
+  static_assert(BITS * N <= 32, "fields must fit one word");
+  constexpr uint32_t kFlip = spread(1u << (BITS - 1), N, BITS);
+  constexpr uint32_t kFix = kFlip - spread(0x4B400000u, N, BITS);
+  uint32_t acc = tb[N - 1];
+#pragma unroll
+  for (int i = N - 2; i >= 0; --i) acc = (acc << BITS) + tb[i];
+  return (acc + kFix) ^ kFlip;
+}
+
 // Codes and reconstruction of 8 elements whose group has maximum magnitude s.
 //   delta = s * 2^(1-b)  (0 when below FLT_MIN),  k = clamp(floor(d * (1/delta))),
 //   q = (k + 1/2) * delta.
-// floor and the b-bit field come from one addition rounded toward -inf: for
-// |u| <= 128, u + 1.5*2^23 rounded down is 1.5*2^23 + floor(u), whose low mantissa
-// bits are the two's-complement code.  Clamping u to [-2^(b-1), 2^(b-1) - 1/2]
-// before the floor equals clamping the integer afterwards.
-template <int BITS>
+// * floor and the b-bit field come from one addition rounded toward -inf: for |u| <= 128,
+//   u + 1.5*2^23 rounded down is 1.5*2^23 + floor(u), whose low mantissa bits are the
+//   two's-complement code.  Clamping u to [-2^(b-1), 2^(b-1) - 1/2] before the floor equals
+//   clamping the integer afterwards.
+// * The lower clamp is only compiled for the wide type: with |d| <= s and a normal
+//   reciprocal, |d * RN(1/delta)| < 2^(b-1) * (1 + 2^-24), which rounds to at most 2^(b-1).
+// * (k + 1/2) * delta, rounded once, is fma(k, delta, delta/2) whenever delta/2 is exact,
+//   i.e. delta >= 2^-125; the wide type falls back to add-then-multiply below that.
+template <typename T, int BITS>
 __device__ __forceinline__ void quantize8(const float (&d)[8], float s, float& delta,
                                           unsigned long long& codes, float (&q)[8]) {
   constexpr float kTwoPow = 1.0f / (float)(1 << (BITS - 1));
   constexpr float kLo = -(float)(1 << (BITS - 1));
   constexpr float kHi = (float)(1 << (BITS - 1)) - 0.5f;
-  constexpr float kMagic = 12582912.0f;
+  constexpr float kMagic = 12582912.0f;                      // 1.5 * 2^23 = 0x4B400000
   const float dl = __fmul_rn(s, kTwoPow);
   const bool live = dl >= FLT_MIN;
   delta = live ? dl : 0.0f;
-  const float inv = live ? __fdiv_rn(1.0f, dl) : 0.0f;
-  codes = 0ull;
+  const float inv = live ? __frcp_rn(dl) : 0.0f;             // IEEE 1/delta, one rounding
+  const float half_delta = __fmul_rn(delta, 0.5f);
+  uint32_t tb[8];
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
     float u = __fmul_rn(d[j], inv);
-    u = fminf(fmaxf(u, kLo), kHi);
+    if constexpr (Conv<T>::kWide) u = fmaxf(u, kLo);
+    u = fminf(u, kHi);
     const float t = __fadd_rd(u, kMagic);
-    const unsigned c = __float_as_uint(t) & ((1u << BITS) - 1u);
-    codes |= (unsigned long long)c << (j * BITS);
-    const float kf = __fsub_rn(t, kMagic);                 // exact: (float)k
-    q[j] = __fmul_rn(__fadd_rn(kf, 0.5f), delta);
+    tb[j] = __float_as_uint(t);
+    const float kf = __fsub_rn(t, kMagic);                   // exact: (float)k
+    q[j] = __fmaf_rn(kf, delta, half_delta);
+  }
+  if constexpr (Conv<T>::kWide) {
+    if (live && delta < 2.3509887e-38f) {                    // 2^-125: delta/2 may have lost a bit
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const float kf = __fsub_rn(__uint_as_float(tb[j]), kMagic);
+        q[j] = __fmul_rn(__fadd_rn(kf, 0.5f), delta);
+      }
+    }
+  }
+  if constexpr (BITS <= 4) {
+    codes = pack_fields<BITS, 8>(tb);
+  } else {
+    const uint32_t lo = pack_fields<BITS, 4>(tb);
+    const uint32_t hi = pack_fields<BITS, 4>(tb + 4);
+    codes = (unsigned long long)lo | ((unsigned long long)hi << (4 * BITS));
   }
 }
 
@@ -119,13 +181,18 @@ __device__ __forceinline__ void quantize8(const float (&d)[8], float s, float& d
 // bit set; subtracting 1.5*2^22 + 2^(b-1) leaves k + 1/2 exactly.
 template <int BITS>
 __device__ __forceinline__ void dequantize8(unsigned long long codes, float delta, float (&q)[8]) {
-  constexpr unsigned kH = 1u << (BITS - 1);
-  constexpr unsigned kMask = (1u << BITS) - 1u;
+  constexpr uint32_t kH = 1u << (BITS - 1);
+  constexpr uint32_t kField = ((1u << BITS) - 1u) << 1;
+  constexpr uint32_t kBits = 0x4AC00001u | (kH << 1);
   constexpr float kBias = 6291456.0f + (float)kH;
+  constexpr int kPerWord = (BITS <= 4) ? 8 : 4;
+  const uint32_t w[2] = {(uint32_t)codes, (BITS <= 4) ? 0u : (uint32_t)(codes >> (4 * BITS))};
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
-    const unsigned c = (unsigned)(codes >> (j * BITS)) & kMask;
-    const float t = __uint_as_float(0x4AC00000u | ((c ^ kH) << 1) | 1u);
+    const uint32_t x = w[j / kPerWord];
+    const int sh = (j % kPerWord) * BITS - 1;
+    const uint32_t f = (sh >= 0) ? (x >> sh) : (x << 1);
+    const float t = __uint_as_float((f & kField) ^ kBits);
     q[j] = __fmul_rn(__fsub_rn(t, kBias), delta);
   }
 }
@@ -230,201 +297,249 @@ __device__ __forceinline__ unsigned long long load_codes(const uint8_t* stream, 
 __device__ __forceinline__ uint4 ld_stream(const void* p) { return __ldcs(reinterpret_cast<const uint4*>(p)); }
 __device__ __forceinline__ void st_stream(void* p, const uint4& v) { __stcs(reinterpret_cast<uint4*>(p), v); }
 
-// ------------------------------------------------------------------ sample resolution (Algorithm 1, "if xi not seen before")
 
-// Mode of sample y of the call, computed by the whole CTA (uniform result).
-__device__ __forceinline__ int cta_resolve(const State& st, const int32_t* ids, int y, bool need_raw,
-                                           bool have_raw, long long& id) {
-  id = ids[y];
-  const bool bad = id < 0 || id >= st.n_samples;
-  int dup = 0;
-  for (int p = threadIdx.x; p < y; p += kThreads) dup |= (ids[p] == ids[y]);
-  dup = __syncthreads_or(dup);
-  if (bad || dup) return kModeSkip;
-  if (st.seen[id]) return kModeDelta;
-  return (need_raw && !have_raw) ? kModeSkip : kModeFirst;
+// ------------------------------------------------------------------ calls and samples (Algorithm 1, "if xi not seen before")
+
+// Number of the running call, the same in every thread of the grid.  The counter in global
+// memory may only move on after every CTA has read it: each CTA takes a ticket after its
+// read and the CTA that draws the last one (the counter wraps back to 0; nobody waits)
+// stores the next call number.
+__device__ __forceinline__ unsigned long long begin_call(const State& st) {
+  __shared__ unsigned long long s_call;
+  if (threadIdx.x == 0) {
+    const unsigned long long c = __ldcg(st.call_no);
+    s_call = c;
+    __threadfence();
+    if (atomicInc(st.ticket, gridDim.x - 1u) == gridDim.x - 1u) *st.call_no = c + 1ull;
+  }
+  __syncthreads();
+  return s_call;
 }
 
-// End of a call.  The seen flags may only change after every CTA has read them, so the CTA
-// that arrives last (a counter that wraps back to 0; nobody waits) re-derives each sample's
-// mode, marks first visits as seen, writes the optional flags and reports skipped samples.
-__device__ __forceinline__ void cta_commit(const State& st, const int32_t* ids, int n_batch, bool need_raw,
-                                           bool have_raw, uint8_t* first_flags) {
-  __shared__ int s_last;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    __threadfence();
-    const unsigned total = gridDim.x * gridDim.y;
-    s_last = (atomicInc(st.ticket, total - 1u) == total - 1u);
+// Mode of sample y of the call, computed by one warp for itself (all 32 lanes call this
+// together).  `why` gets the status bit of a skipped sample.
+__device__ __forceinline__ int resolve_sample(const State& st, const int32_t* __restrict__ ids, int y, int lane,
+                                              bool need_raw, bool have_raw, unsigned long long call,
+                                              long long& id, unsigned& why) {
+  const int32_t my = ids[y];
+  id = my;
+  why = 0u;
+  if (my < 0 || (long long)my >= st.n_samples) {
+    why = kStBadId;
+    return kModeSkip;
   }
-  __syncthreads();
-  if (!s_last) return;
-  unsigned why = 0;
-  for (int y = threadIdx.x; y < n_batch; y += kThreads) {
-    const long long id = ids[y];
-    int mode;
-    if (id < 0 || id >= st.n_samples) {
-      mode = kModeSkip;
-      why |= kStBadId;
-    } else {
-      bool dup = false;
-      for (int p = 0; p < y; ++p) dup |= (ids[p] == ids[y]);
-      if (dup) {
-        mode = kModeSkip;
-        why |= kStDupId;
-      } else if (st.seen[id]) {
-        mode = kModeDelta;
-      } else if (need_raw && !have_raw) {
-        mode = kModeSkip;
-        why |= kStNoRaw;
-      } else {
-        mode = kModeFirst;
-      }
-    }
-    if (first_flags) first_flags[y] = (uint8_t)(mode == kModeFirst);
-    if (mode == kModeFirst) st.seen[id] = 1;     // distinct ids: no two threads write one flag
+  int dup = 0;
+  for (int p = lane; p < y; p += 32) dup |= (ids[p] == my);
+  if (__any_sync(kFullMask, dup)) {
+    why = kStDupId;
+    return kModeSkip;
   }
+  const unsigned long long stamp = __ldcg(st.seen + my);
+  if (stamp != 0ull && stamp != call) return kModeDelta;
+  if (need_raw && !have_raw) {
+    why = kStNoRaw;
+    return kModeSkip;
+  }
+  return kModeFirst;
+}
+
+// Done once per sample and call, by the thread that owns the sample's first chunk.
+__device__ __forceinline__ void publish_sample(const State& st, int y, int mode, long long id, unsigned why,
+                                               unsigned long long call, uint8_t* first_flags) {
   if (why) atomicOr(st.status, why);
+  if (first_flags) first_flags[y] = (uint8_t)(mode == kModeFirst);
+  if (mode == kModeFirst) st.seen[id] = call;
 }
 
 // ------------------------------------------------------------------ encode (sender)
 
-template <typename T, int BITS>
-__global__ void __launch_bounds__(kThreads) encode_kernel(const State st, const EncodeArgs a) {
-  const int y = blockIdx.y;
-  const int lane = threadIdx.x & 31;
-  long long id;
-  const int mode = cta_resolve(st, a.ids, y, false, false, id);
-
-  const T* act = reinterpret_cast<const T*>(a.act) + (long long)y * st.elems;
-  uint8_t* stream = a.packed + (long long)y * st.packed_bytes;
-  float* scales = a.scales + (long long)y * st.groups;
+template <typename T, int BITS, int LPG>
+__global__ void __launch_bounds__(kThreads) encode_kernel(const State st, const EncodeArgs a, const int rows_per_cta) {
+  const int tid = threadIdx.x;
+  const int lane = tid & 31;
+  const unsigned long long call = begin_call(st);
+  const int total_rows = a.n_batch * st.rows;
+  int r = blockIdx.x * rows_per_cta;
+  const int r_end = min(total_rows, r + rows_per_cta);
   const bool words_ok = (st.packed_bytes & 3) == 0;
-  const long long c0 = (long long)blockIdx.x * kChunksPerCta + threadIdx.x;
+  const int group_lead_mask = st.lanes_per_group - 1;
 
-  if (mode == kModeDelta) {
-    T* m = reinterpret_cast<T*>(st.m) + id * st.elems;
-    uint4 av[kChunksPerThread], mv[kChunksPerThread];
+  int cur_y = -1, mode = kModeSkip;
+  const T* act = nullptr;
+  T* m = nullptr;
+  uint8_t* stream = nullptr;
+  float* scales = nullptr;
+
+  while (r < r_end) {
+    const int y = r / st.rows;
+    const int rin = r - y * st.rows;
+    if (y != cur_y) {
+      cur_y = y;
+      long long id;
+      unsigned why;
+      mode = resolve_sample(st, a.ids, y, lane, false, false, call, id, why);
+      if (rin == 0 && tid == 0) publish_sample(st, y, mode, id, why, call, a.first_flags);
+      act = reinterpret_cast<const T*>(a.act) + (long long)y * st.elems;
+      stream = a.packed + (long long)y * st.packed_bytes;
+      scales = a.scales + (long long)y * st.groups;
+      m = (mode == kModeSkip) ? nullptr : reinterpret_cast<T*>(st.m) + id * st.elems;
+    }
+    const int n = min(kRowsPerIter, min(r_end - r, st.rows - rin));
+    const int c0 = rin * kThreads + tid;
+
+    if (mode == kModeDelta) {
+      uint4 av[kRowsPerIter], mv[kRowsPerIter];
 #pragma unroll
-    for (int i = 0; i < kChunksPerThread; ++i) {
-      const long long c = c0 + i * kThreads;
-      av[i] = make_uint4(0, 0, 0, 0);
-      mv[i] = make_uint4(0, 0, 0, 0);
-      if (c < st.chunks) {
-        av[i] = ld_stream(act + c * kChunk);
-        mv[i] = ld_stream(m + c * kChunk);
+      for (int i = 0; i < kRowsPerIter; ++i) {
+        const int c = c0 + i * kThreads;
+        av[i] = make_uint4(0, 0, 0, 0);
+        mv[i] = make_uint4(0, 0, 0, 0);
+        if (i < n && c < st.chunks) {
+          av[i] = ld_stream(act + (long long)c * kChunk);
+          mv[i] = ld_stream(m + (long long)c * kChunk);
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < kRowsPerIter; ++i) {
+        if (i < n) {                                   // uniform over the CTA
+          const int c = c0 + i * kThreads;
+          const bool active = c < st.chunks;
+          float mf[8], d[8], q[8];
+          {
+            float af[8];
+            Conv<T>::unpack(av[i], af);
+            Conv<T>::unpack(mv[i], mf);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) d[j] = __fsub_rn(af[j], mf[j]);
+          }
+          const float s = group_max<LPG>(abs_max8(d), st.lanes_per_group);
+          float delta;
+          unsigned long long codes;
+          quantize8<T, BITS>(d, s, delta, codes, q);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) mf[j] = __fadd_rn(mf[j], q[j]);
+          if (active) {
+            st_stream(m + (long long)c * kChunk, Conv<T>::pack(mf));
+            if ((lane & group_lead_mask) == 0) scales[c >> st.lg_shift] = delta;
+          }
+          const bool warp_words = words_ok && (c - lane + 32 <= st.chunks);
+          store_codes<BITS>(stream, c, lane, active, warp_words, codes);
+        }
+      }
+    } else {
+      // first visit: the activation itself becomes m(xi); skipped sample: nothing is stored.
+      // Either way the sample's codes and scales are zero.
+#pragma unroll
+      for (int i = 0; i < kRowsPerIter; ++i) {
+        if (i < n) {
+          const int c = c0 + i * kThreads;
+          const bool active = c < st.chunks;
+          if (active) {
+            if (m) st_stream(m + (long long)c * kChunk, ld_stream(act + (long long)c * kChunk));
+            if ((lane & group_lead_mask) == 0) scales[c >> st.lg_shift] = 0.0f;
+          }
+          const bool warp_words = words_ok && (c - lane + 32 <= st.chunks);
+          store_codes<BITS>(stream, c, lane, active, warp_words, 0ull);
+        }
       }
     }
-#pragma unroll
-    for (int i = 0; i < kChunksPerThread; ++i) {
-      const long long c = c0 + i * kThreads;
-      const bool active = c < st.chunks;
-      float af[8], mf[8], d[8], q[8];
-      Conv<T>::unpack(av[i], af);
-      Conv<T>::unpack(mv[i], mf);
-#pragma unroll
-      for (int j = 0; j < 8; ++j) d[j] = __fsub_rn(af[j], mf[j]);
-      const float s = group_max(abs_max8(d), st.lanes_per_group);
-      float delta;
-      unsigned long long codes;
-      quantize8<BITS>(d, s, delta, codes, q);
-#pragma unroll
-      for (int j = 0; j < 8; ++j) mf[j] = __fadd_rn(mf[j], q[j]);
-      if (active) {
-        st_stream(m + c * kChunk, Conv<T>::pack(mf));
-        if ((lane & (st.lanes_per_group - 1)) == 0) scales[c >> st.lg_shift] = delta;
-      }
-      const bool warp_words = words_ok && (c - lane + 32 <= st.chunks);
-      store_codes<BITS>(stream, c, lane, active, warp_words, codes);
-    }
-  } else {
-    // first visit: the activation itself becomes m(xi); skipped sample: nothing is stored.
-    // Either way the sample's codes and scales are zero.
-    T* m = (mode == kModeFirst) ? reinterpret_cast<T*>(st.m) + id * st.elems : nullptr;
-#pragma unroll
-    for (int i = 0; i < kChunksPerThread; ++i) {
-      const long long c = c0 + i * kThreads;
-      const bool active = c < st.chunks;
-      if (active) {
-        if (m) st_stream(m + c * kChunk, ld_stream(act + c * kChunk));
-        if ((lane & (st.lanes_per_group - 1)) == 0) scales[c >> st.lg_shift] = 0.0f;
-      }
-      const bool warp_words = words_ok && (c - lane + 32 <= st.chunks);
-      store_codes<BITS>(stream, c, lane, active, warp_words, 0ull);
-    }
+    r += n;
   }
-  cta_commit(st, a.ids, a.n_batch, false, false, a.first_flags);
 }
 
 // ------------------------------------------------------------------ decode (receiver)
 
 template <typename T, int BITS>
-__global__ void __launch_bounds__(kThreads) decode_kernel(const State st, const DecodeArgs a) {
-  const int y = blockIdx.y;
-  const int lane = threadIdx.x & 31;
-  long long id;
-  const int mode = cta_resolve(st, a.ids, y, true, a.raw != nullptr, id);
+__global__ void __launch_bounds__(kThreads) decode_kernel(const State st, const DecodeArgs a, const int rows_per_cta) {
+  const int tid = threadIdx.x;
+  const int lane = tid & 31;
+  const unsigned long long call = begin_call(st);
+  const int total_rows = a.n_batch * st.rows;
+  int r = blockIdx.x * rows_per_cta;
+  const int r_end = min(total_rows, r + rows_per_cta);
+  const bool words_ok = (st.packed_bytes & 3) == 0;
 
-  T* out = reinterpret_cast<T*>(a.out) + (long long)y * st.elems;
-  const long long c0 = (long long)blockIdx.x * kChunksPerCta + threadIdx.x;
+  int cur_y = -1, mode = kModeSkip;
+  T* out = nullptr;
+  T* m = nullptr;
+  const T* raw = nullptr;
+  const uint8_t* stream = nullptr;
+  const float* scales = nullptr;
 
-  if (mode == kModeDelta) {
-    T* m = reinterpret_cast<T*>(st.m) + id * st.elems;
-    const uint8_t* stream = a.packed + (long long)y * st.packed_bytes;
-    const float* scales = a.scales + (long long)y * st.groups;
-    const bool words_ok = (st.packed_bytes & 3) == 0;
-    uint4 mv[kChunksPerThread];
-    unsigned long long codes[kChunksPerThread];
-    float delta[kChunksPerThread];
-#pragma unroll
-    for (int i = 0; i < kChunksPerThread; ++i) {
-      const long long c = c0 + i * kThreads;
-      const bool active = c < st.chunks;
-      mv[i] = make_uint4(0, 0, 0, 0);
-      delta[i] = 0.0f;
-      if (active) {
-        mv[i] = ld_stream(m + c * kChunk);
-        delta[i] = __ldg(scales + (c >> st.lg_shift));
-      }
-      const bool warp_words = words_ok && (c - lane + 32 <= st.chunks);
-      codes[i] = load_codes<BITS>(stream, c, lane, active, warp_words);
+  while (r < r_end) {
+    const int y = r / st.rows;
+    const int rin = r - y * st.rows;
+    if (y != cur_y) {
+      cur_y = y;
+      long long id;
+      unsigned why;
+      mode = resolve_sample(st, a.ids, y, lane, true, a.raw != nullptr, call, id, why);
+      if (rin == 0 && tid == 0) publish_sample(st, y, mode, id, why, call, a.first_flags);
+      out = reinterpret_cast<T*>(a.out) + (long long)y * st.elems;
+      stream = a.packed + (long long)y * st.packed_bytes;
+      scales = a.scales + (long long)y * st.groups;
+      m = (mode == kModeSkip) ? nullptr : reinterpret_cast<T*>(st.m) + id * st.elems;
+      raw = (mode == kModeFirst) ? reinterpret_cast<const T*>(a.raw) + (long long)y * st.elems : nullptr;
     }
+    const int n = min(kRowsPerIter, min(r_end - r, st.rows - rin));
+    const int c0 = rin * kThreads + tid;
+
+    if (mode == kModeDelta) {
+      uint4 mv[kRowsPerIter];
+      unsigned long long codes[kRowsPerIter];
+      float delta[kRowsPerIter];
 #pragma unroll
-    for (int i = 0; i < kChunksPerThread; ++i) {
-      const long long c = c0 + i * kThreads;
-      if (c < st.chunks) {
-        float mf[8], q[8];
-        Conv<T>::unpack(mv[i], mf);
-        dequantize8<BITS>(codes[i], delta[i], q);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) mf[j] = __fadd_rn(mf[j], q[j]);
-        const uint4 nv = Conv<T>::pack(mf);
-        st_stream(m + c * kChunk, nv);
-        st_stream(out + c * kChunk, nv);
-      }
-    }
-  } else {
-    T* m = (mode == kModeFirst) ? reinterpret_cast<T*>(st.m) + id * st.elems : nullptr;
-    const T* raw = (mode == kModeFirst) ? reinterpret_cast<const T*>(a.raw) + (long long)y * st.elems : nullptr;
-#pragma unroll
-    for (int i = 0; i < kChunksPerThread; ++i) {
-      const long long c = c0 + i * kThreads;
-      if (c < st.chunks) {
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (m) {
-          v = ld_stream(raw + c * kChunk);
-          st_stream(m + c * kChunk, v);
+      for (int i = 0; i < kRowsPerIter; ++i) {
+        const int c = c0 + i * kThreads;
+        const bool active = i < n && c < st.chunks;
+        mv[i] = make_uint4(0, 0, 0, 0);
+        delta[i] = 0.0f;
+        codes[i] = 0ull;
+        if (active) {
+          mv[i] = ld_stream(m + (long long)c * kChunk);
+          delta[i] = __ldg(scales + (c >> st.lg_shift));
         }
-        st_stream(out + c * kChunk, v);
+        if (i < n) {
+          const bool warp_words = words_ok && (c - lane + 32 <= st.chunks);
+          codes[i] = load_codes<BITS>(stream, c, lane, active, warp_words);
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < kRowsPerIter; ++i) {
+        const int c = c0 + i * kThreads;
+        if (i < n && c < st.chunks) {
+          float mf[8], q[8];
+          Conv<T>::unpack(mv[i], mf);
+          dequantize8<BITS>(codes[i], delta[i], q);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) mf[j] = __fadd_rn(mf[j], q[j]);
+          const uint4 nv = Conv<T>::pack(mf);
+          st_stream(m + (long long)c * kChunk, nv);
+          st_stream(out + (long long)c * kChunk, nv);
+        }
+      }
+    } else {
+      // first visit: the raw message becomes m(xi) and the activation; skipped sample: zeros out.
+#pragma unroll
+      for (int i = 0; i < kRowsPerIter; ++i) {
+        const int c = c0 + i * kThreads;
+        if (i < n && c < st.chunks) {
+          uint4 v = make_uint4(0, 0, 0, 0);
+          if (raw) {
+            v = ld_stream(raw + (long long)c * kChunk);
+            st_stream(m + (long long)c * kChunk, v);
+          }
+          st_stream(out + (long long)c * kChunk, v);
+        }
       }
     }
+    r += n;
   }
-  cta_commit(st, a.ids, a.n_batch, true, a.raw != nullptr, a.first_flags);
 }
 
 // ------------------------------------------------------------------ backward direction: direct quantization
 
-template <typename T, int BITS>
+template <typename T, int BITS, int LPG>
 __global__ void __launch_bounds__(kThreads) quant_grad_kernel(const T* __restrict__ grad, long long n_chunks,
                                                               int lanes_per_group, uint8_t* __restrict__ packed,
                                                               float* __restrict__ scales) {
@@ -443,10 +558,10 @@ __global__ void __launch_bounds__(kThreads) quant_grad_kernel(const T* __restric
     const bool active = c < n_chunks;
     float d[8], q[8];
     Conv<T>::unpack(gv[i], d);
-    const float s = group_max(abs_max8(d), lanes_per_group);
+    const float s = group_max<LPG>(abs_max8(d), lanes_per_group);
     float delta;
     unsigned long long codes;
-    quantize8<BITS>(d, s, delta, codes, q);
+    quantize8<T, BITS>(d, s, delta, codes, q);
     if (active && (lane & (lanes_per_group - 1)) == 0) scales[c >> lg_shift] = delta;
     store_codes<BITS>(packed, c, lane, active, c - lane + 32 <= n_chunks, codes);
   }
@@ -489,7 +604,7 @@ __device__ __forceinline__ unsigned long long mix64(unsigned long long index, un
 }
 
 __global__ void __launch_bounds__(kThreads) checksum_kernel(const State st, unsigned long long* sum_out) {
-  const long long n_vec = st.n_samples * st.chunks;      // 16-byte pieces = 4 words each
+  const long long n_vec = st.n_samples * (long long)st.chunks;      // 16-byte pieces = 4 words each
   const uint4* mv = reinterpret_cast<const uint4*>(st.m);
   const long long stride = (long long)gridDim.x * kThreads;
   unsigned long long acc = 0ull;
@@ -499,7 +614,7 @@ __global__ void __launch_bounds__(kThreads) checksum_kernel(const State st, unsi
     acc += mix64(i, w.x) + mix64(i + 1, w.y) + mix64(i + 2, w.z) + mix64(i + 3, w.w);
   }
   for (long long x = (long long)blockIdx.x * kThreads + threadIdx.x; x < st.n_samples; x += stride)
-    acc += mix64((1ull << 40) + (unsigned long long)x, st.seen[x]);
+    acc += mix64((1ull << 40) + (unsigned long long)x, st.seen[x] != 0ull ? 1ull : 0ull);
   for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(kFullMask, acc, o);
   __shared__ unsigned long long part[kThreads / 32];
   if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = acc;
@@ -535,26 +650,62 @@ __global__ void __launch_bounds__(kThreads) checksum_kernel(const State st, unsi
     return cudaErrorInvalidValue;                           \
   }
 
+// group sizes 64 and 128 (8 and 16 lanes) get their own instantiation; the rest share one
+#define AQ_WITH_LPG(lanes, CALL_LPG)                        \
+  switch (lanes) {                                          \
+    case 8: CALL_LPG(8); break;                             \
+    case 16: CALL_LPG(16); break;                           \
+    default: CALL_LPG(0); break;                            \
+  }
+
 inline unsigned grid_x(long long chunks) { return (unsigned)((chunks + kChunksPerCta - 1) / kChunksPerCta); }
+
+// CTAs of `kernel` that fit one multiprocessor (asked once per kernel).
+template <typename K>
+int resident_ctas(K kernel) {
+  static const int n = [kernel] {
+    int v = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, kernel, kThreads, 0) != cudaSuccess || v < 1) v = 1;
+    return v;
+  }();
+  return n;
+}
+
+// One wave: at most sms * resident CTAs, every CTA the same number of rows (the last one the rest).
+template <typename K, typename Args>
+cudaError_t launch_rows(K kernel, const State& st, const Args& a, cudaStream_t s) {
+  const long long total = (long long)a.n_batch * st.rows;
+  if (total <= 0) return cudaSuccess;
+  if (total > 0x7fffffffll) return cudaErrorInvalidValue;
+  const long long wave = (long long)st.sms * resident_ctas(kernel);
+  int per = (int)((total + wave - 1) / wave);
+  if (st.rows_per_cta > 0) per = (int)(st.rows_per_cta < total ? st.rows_per_cta : total);
+  const unsigned grid = (unsigned)((total + per - 1) / per);
+  kernel<<<grid, kThreads, 0, s>>>(st, a, per);
+  return cudaGetLastError();
+}
 
 }  // namespace
 
 cudaError_t launch_encode(int dtype, int bits, const State& st, const EncodeArgs& a, cudaStream_t s) {
-  if (a.n_batch <= 0) return cudaSuccess;
-  const dim3 grid(grid_x(st.chunks), (unsigned)a.n_batch);
-#define AQ_CALL(T, B) encode_kernel<T, B><<<grid, kThreads, 0, s>>>(st, a)
+#define AQ_CALL_LPG(L) return launch_rows(encode_kernel<T_, B_, L>, st, a, s)
+#define AQ_CALL(T, B)                                      \
+  {                                                        \
+    using T_ = T;                                          \
+    constexpr int B_ = B;                                  \
+    AQ_WITH_LPG(st.lanes_per_group, AQ_CALL_LPG)           \
+  }
   AQ_DISPATCH(dtype, bits, AQ_CALL)
 #undef AQ_CALL
-  return cudaGetLastError();
+#undef AQ_CALL_LPG
+  return cudaErrorInvalidValue;
 }
 
 cudaError_t launch_decode(int dtype, int bits, const State& st, const DecodeArgs& a, cudaStream_t s) {
-  if (a.n_batch <= 0) return cudaSuccess;
-  const dim3 grid(grid_x(st.chunks), (unsigned)a.n_batch);
-#define AQ_CALL(T, B) decode_kernel<T, B><<<grid, kThreads, 0, s>>>(st, a)
+#define AQ_CALL(T, B) return launch_rows(decode_kernel<T, B>, st, a, s)
   AQ_DISPATCH(dtype, bits, AQ_CALL)
 #undef AQ_CALL
-  return cudaGetLastError();
+  return cudaErrorInvalidValue;
 }
 
 cudaError_t launch_quant_grad(int dtype, int bits, int lanes_per_group, const void* grad, long long n_elems,
@@ -562,10 +713,17 @@ cudaError_t launch_quant_grad(int dtype, int bits, int lanes_per_group, const vo
   if (n_elems <= 0) return cudaSuccess;
   const long long chunks = n_elems / kChunk;
   const unsigned grid = grid_x(chunks);
-#define AQ_CALL(T, B) \
-  quant_grad_kernel<T, B><<<grid, kThreads, 0, s>>>(reinterpret_cast<const T*>(grad), chunks, lanes_per_group, packed, scales)
+#define AQ_CALL_LPG(L) \
+  quant_grad_kernel<T_, B_, L><<<grid, kThreads, 0, s>>>(reinterpret_cast<const T_*>(grad), chunks, lanes_per_group, packed, scales)
+#define AQ_CALL(T, B)                                      \
+  {                                                        \
+    using T_ = T;                                          \
+    constexpr int B_ = B;                                  \
+    AQ_WITH_LPG(lanes_per_group, AQ_CALL_LPG)              \
+  }
   AQ_DISPATCH(dtype, bits, AQ_CALL)
 #undef AQ_CALL
+#undef AQ_CALL_LPG
   return cudaGetLastError();
 }
 
@@ -582,12 +740,9 @@ cudaError_t launch_dequant_grad(int dtype, int bits, int lanes_per_group, const 
 }
 
 cudaError_t launch_checksum(const State& st, unsigned long long* sum_dev, cudaStream_t s) {
-  int dev = 0, sms = 148;
-  cudaGetDevice(&dev);
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const long long n_vec = st.n_samples * st.chunks;
+  const long long n_vec = st.n_samples * (long long)st.chunks;
   long long want = (n_vec + kThreads - 1) / kThreads;
-  const long long cap = (long long)sms * 8;
+  const long long cap = (long long)st.sms * 8;
   const unsigned grid = (unsigned)(want < 1 ? 1 : (want > cap ? cap : want));
   checksum_kernel<<<grid, kThreads, 0, s>>>(st, sum_dev);
   return cudaGetLastError();
