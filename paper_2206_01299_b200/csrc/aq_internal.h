@@ -34,7 +34,7 @@ struct State {
   int lanes_per_group;            // group / 8, a power of two <= 32
   int lg_shift;                   // log2(lanes_per_group)
   int sms;                        // multiprocessors of the handle's device
-  int rows_per_cta;               // 0 = one wave of CTAs (default); > 0 = fixed rows per CTA
+  int rows_per_cta;               // 0 = chosen by the launch layer (default); > 0 = fixed rows per CTA
 };
 
 struct EncodeArgs {

@@ -351,18 +351,91 @@ __device__ __forceinline__ void publish_sample(const State& st, int y, int mode,
   if (mode == kModeFirst) st.seen[id] = call;
 }
 
+// ------------------------------------------------------------------ row walk shared by encode and decode
+
+// Position of a CTA inside its contiguous range of rows.  A row is kThreads consecutive
+// chunks of one sample; the last row of a sample may be ragged.
+struct RowCursor {
+  int r, r_end;      // global row index and end of the CTA's range
+  int y, rin;        // sample of the call and row inside the sample
+  __device__ __forceinline__ RowCursor(int rows_per_cta, int total_rows, int rows_per_sample) {
+    r = blockIdx.x * rows_per_cta;
+    r_end = min(total_rows, r + rows_per_cta);
+    y = r / rows_per_sample;
+    rin = r - y * rows_per_sample;
+  }
+  __device__ __forceinline__ bool done() const { return r >= r_end; }
+  // rows handled by the next iteration: they belong to one sample
+  __device__ __forceinline__ int take(int rows_per_sample) const {
+    return min(kRowsPerIter, min(r_end - r, rows_per_sample - rin));
+  }
+  __device__ __forceinline__ void advance(int n, int rows_per_sample) {
+    r += n;
+    rin += n;
+    if (rin >= rows_per_sample) {
+      rin = 0;
+      ++y;
+    }
+  }
+};
+
 // ------------------------------------------------------------------ encode (sender)
 
+// Delta visit of n rows starting at chunk c0 of one sample.  FULL: n == kRowsPerIter and every
+// chunk is inside the sample, so no bounds are checked.
+template <typename T, int BITS, int LPG, bool FULL>
+__device__ __forceinline__ void encode_rows(const State& st, const T* __restrict__ act, T* __restrict__ m,
+                                            uint8_t* __restrict__ stream, float* __restrict__ scales, int c0,
+                                            int n, int lane, bool words_ok) {
+  uint4 av[kRowsPerIter], mv[kRowsPerIter];
+#pragma unroll
+  for (int i = 0; i < kRowsPerIter; ++i) {
+    const int c = c0 + i * kThreads;
+    if (FULL || (i < n && c < st.chunks)) {
+      av[i] = ld_stream(act + (size_t)c * kChunk);
+      mv[i] = ld_stream(m + (size_t)c * kChunk);
+    } else {
+      av[i] = make_uint4(0, 0, 0, 0);
+      mv[i] = make_uint4(0, 0, 0, 0);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < kRowsPerIter; ++i) {
+    if (FULL || i < n) {                              // uniform over the CTA
+      const int c = c0 + i * kThreads;
+      const bool active = FULL || c < st.chunks;
+      float mf[8], d[8], q[8];
+      {
+        float af[8];
+        Conv<T>::unpack(av[i], af);
+        Conv<T>::unpack(mv[i], mf);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) d[j] = __fsub_rn(af[j], mf[j]);
+      }
+      const float s = group_max<LPG>(abs_max8(d), st.lanes_per_group);
+      float delta;
+      unsigned long long codes;
+      quantize8<T, BITS>(d, s, delta, codes, q);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) mf[j] = __fadd_rn(mf[j], q[j]);
+      if (active) {
+        st_stream(m + (size_t)c * kChunk, Conv<T>::pack(mf));
+        if ((lane & (st.lanes_per_group - 1)) == 0) scales[c >> st.lg_shift] = delta;
+      }
+      const bool warp_words = words_ok && (FULL || c - lane + 32 <= st.chunks);
+      store_codes<BITS>(stream, c, lane, active, warp_words, codes);
+    }
+  }
+}
+
 template <typename T, int BITS, int LPG>
-__global__ void __launch_bounds__(kThreads) encode_kernel(const State st, const EncodeArgs a, const int rows_per_cta) {
+__global__ void __launch_bounds__(kThreads, (BITS == 3 || BITS >= 5) ? 4 : 6)
+    encode_kernel(const State st, const EncodeArgs a, const int rows_per_cta) {
   const int tid = threadIdx.x;
   const int lane = tid & 31;
   const unsigned long long call = begin_call(st);
-  const int total_rows = a.n_batch * st.rows;
-  int r = blockIdx.x * rows_per_cta;
-  const int r_end = min(total_rows, r + rows_per_cta);
+  RowCursor cur(rows_per_cta, a.n_batch * st.rows, st.rows);
   const bool words_ok = (st.packed_bytes & 3) == 0;
-  const int group_lead_mask = st.lanes_per_group - 1;
 
   int cur_y = -1, mode = kModeSkip;
   const T* act = nullptr;
@@ -370,62 +443,26 @@ __global__ void __launch_bounds__(kThreads) encode_kernel(const State st, const 
   uint8_t* stream = nullptr;
   float* scales = nullptr;
 
-  while (r < r_end) {
-    const int y = r / st.rows;
-    const int rin = r - y * st.rows;
-    if (y != cur_y) {
-      cur_y = y;
+  while (!cur.done()) {
+    if (cur.y != cur_y) {
+      cur_y = cur.y;
       long long id;
       unsigned why;
-      mode = resolve_sample(st, a.ids, y, lane, false, false, call, id, why);
-      if (rin == 0 && tid == 0) publish_sample(st, y, mode, id, why, call, a.first_flags);
-      act = reinterpret_cast<const T*>(a.act) + (long long)y * st.elems;
-      stream = a.packed + (long long)y * st.packed_bytes;
-      scales = a.scales + (long long)y * st.groups;
+      mode = resolve_sample(st, a.ids, cur_y, lane, false, false, call, id, why);
+      if (cur.rin == 0 && tid == 0) publish_sample(st, cur_y, mode, id, why, call, a.first_flags);
+      act = reinterpret_cast<const T*>(a.act) + (long long)cur_y * st.elems;
+      stream = a.packed + (long long)cur_y * st.packed_bytes;
+      scales = a.scales + (long long)cur_y * st.groups;
       m = (mode == kModeSkip) ? nullptr : reinterpret_cast<T*>(st.m) + id * st.elems;
     }
-    const int n = min(kRowsPerIter, min(r_end - r, st.rows - rin));
-    const int c0 = rin * kThreads + tid;
+    const int n = cur.take(st.rows);
+    const int c0 = cur.rin * kThreads + tid;
 
     if (mode == kModeDelta) {
-      uint4 av[kRowsPerIter], mv[kRowsPerIter];
-#pragma unroll
-      for (int i = 0; i < kRowsPerIter; ++i) {
-        const int c = c0 + i * kThreads;
-        av[i] = make_uint4(0, 0, 0, 0);
-        mv[i] = make_uint4(0, 0, 0, 0);
-        if (i < n && c < st.chunks) {
-          av[i] = ld_stream(act + (long long)c * kChunk);
-          mv[i] = ld_stream(m + (long long)c * kChunk);
-        }
-      }
-#pragma unroll
-      for (int i = 0; i < kRowsPerIter; ++i) {
-        if (i < n) {                                   // uniform over the CTA
-          const int c = c0 + i * kThreads;
-          const bool active = c < st.chunks;
-          float mf[8], d[8], q[8];
-          {
-            float af[8];
-            Conv<T>::unpack(av[i], af);
-            Conv<T>::unpack(mv[i], mf);
-#pragma unroll
-            for (int j = 0; j < 8; ++j) d[j] = __fsub_rn(af[j], mf[j]);
-          }
-          const float s = group_max<LPG>(abs_max8(d), st.lanes_per_group);
-          float delta;
-          unsigned long long codes;
-          quantize8<T, BITS>(d, s, delta, codes, q);
-#pragma unroll
-          for (int j = 0; j < 8; ++j) mf[j] = __fadd_rn(mf[j], q[j]);
-          if (active) {
-            st_stream(m + (long long)c * kChunk, Conv<T>::pack(mf));
-            if ((lane & group_lead_mask) == 0) scales[c >> st.lg_shift] = delta;
-          }
-          const bool warp_words = words_ok && (c - lane + 32 <= st.chunks);
-          store_codes<BITS>(stream, c, lane, active, warp_words, codes);
-        }
-      }
+      if ((cur.rin + kRowsPerIter) * kThreads <= st.chunks && n == kRowsPerIter)
+        encode_rows<T, BITS, LPG, true>(st, act, m, stream, scales, c0, n, lane, words_ok);
+      else
+        encode_rows<T, BITS, LPG, false>(st, act, m, stream, scales, c0, n, lane, words_ok);
     } else {
       // first visit: the activation itself becomes m(xi); skipped sample: nothing is stored.
       // Either way the sample's codes and scales are zero.
@@ -435,28 +472,66 @@ __global__ void __launch_bounds__(kThreads) encode_kernel(const State st, const 
           const int c = c0 + i * kThreads;
           const bool active = c < st.chunks;
           if (active) {
-            if (m) st_stream(m + (long long)c * kChunk, ld_stream(act + (long long)c * kChunk));
-            if ((lane & group_lead_mask) == 0) scales[c >> st.lg_shift] = 0.0f;
+            if (m) st_stream(m + (size_t)c * kChunk, ld_stream(act + (size_t)c * kChunk));
+            if ((lane & (st.lanes_per_group - 1)) == 0) scales[c >> st.lg_shift] = 0.0f;
           }
           const bool warp_words = words_ok && (c - lane + 32 <= st.chunks);
           store_codes<BITS>(stream, c, lane, active, warp_words, 0ull);
         }
       }
     }
-    r += n;
+    cur.advance(n, st.rows);
   }
 }
 
 // ------------------------------------------------------------------ decode (receiver)
 
+template <typename T, int BITS, bool FULL>
+__device__ __forceinline__ void decode_rows(const State& st, const uint8_t* __restrict__ stream,
+                                            const float* __restrict__ scales, T* __restrict__ m,
+                                            T* __restrict__ out, int c0, int n, int lane, bool words_ok) {
+  uint4 mv[kRowsPerIter];
+  unsigned long long codes[kRowsPerIter];
+  float delta[kRowsPerIter];
+#pragma unroll
+  for (int i = 0; i < kRowsPerIter; ++i) {
+    const int c = c0 + i * kThreads;
+    const bool active = FULL || (i < n && c < st.chunks);
+    if (active) {
+      mv[i] = ld_stream(m + (size_t)c * kChunk);
+      delta[i] = __ldg(scales + (c >> st.lg_shift));
+    } else {
+      mv[i] = make_uint4(0, 0, 0, 0);
+      delta[i] = 0.0f;
+    }
+    codes[i] = 0ull;
+    if (FULL || i < n) {                              // uniform over the CTA
+      const bool warp_words = words_ok && (FULL || c - lane + 32 <= st.chunks);
+      codes[i] = load_codes<BITS>(stream, c, lane, active, warp_words);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < kRowsPerIter; ++i) {
+    const int c = c0 + i * kThreads;
+    if (FULL || (i < n && c < st.chunks)) {
+      float mf[8], q[8];
+      Conv<T>::unpack(mv[i], mf);
+      dequantize8<BITS>(codes[i], delta[i], q);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) mf[j] = __fadd_rn(mf[j], q[j]);
+      const uint4 nv = Conv<T>::pack(mf);
+      st_stream(m + (size_t)c * kChunk, nv);
+      st_stream(out + (size_t)c * kChunk, nv);
+    }
+  }
+}
+
 template <typename T, int BITS>
-__global__ void __launch_bounds__(kThreads) decode_kernel(const State st, const DecodeArgs a, const int rows_per_cta) {
+__global__ void __launch_bounds__(kThreads, 6) decode_kernel(const State st, const DecodeArgs a, const int rows_per_cta) {
   const int tid = threadIdx.x;
   const int lane = tid & 31;
   const unsigned long long call = begin_call(st);
-  const int total_rows = a.n_batch * st.rows;
-  int r = blockIdx.x * rows_per_cta;
-  const int r_end = min(total_rows, r + rows_per_cta);
+  RowCursor cur(rows_per_cta, a.n_batch * st.rows, st.rows);
   const bool words_ok = (st.packed_bytes & 3) == 0;
 
   int cur_y = -1, mode = kModeSkip;
@@ -466,58 +541,27 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(const State st, const 
   const uint8_t* stream = nullptr;
   const float* scales = nullptr;
 
-  while (r < r_end) {
-    const int y = r / st.rows;
-    const int rin = r - y * st.rows;
-    if (y != cur_y) {
-      cur_y = y;
+  while (!cur.done()) {
+    if (cur.y != cur_y) {
+      cur_y = cur.y;
       long long id;
       unsigned why;
-      mode = resolve_sample(st, a.ids, y, lane, true, a.raw != nullptr, call, id, why);
-      if (rin == 0 && tid == 0) publish_sample(st, y, mode, id, why, call, a.first_flags);
-      out = reinterpret_cast<T*>(a.out) + (long long)y * st.elems;
-      stream = a.packed + (long long)y * st.packed_bytes;
-      scales = a.scales + (long long)y * st.groups;
+      mode = resolve_sample(st, a.ids, cur_y, lane, true, a.raw != nullptr, call, id, why);
+      if (cur.rin == 0 && tid == 0) publish_sample(st, cur_y, mode, id, why, call, a.first_flags);
+      out = reinterpret_cast<T*>(a.out) + (long long)cur_y * st.elems;
+      stream = a.packed + (long long)cur_y * st.packed_bytes;
+      scales = a.scales + (long long)cur_y * st.groups;
       m = (mode == kModeSkip) ? nullptr : reinterpret_cast<T*>(st.m) + id * st.elems;
-      raw = (mode == kModeFirst) ? reinterpret_cast<const T*>(a.raw) + (long long)y * st.elems : nullptr;
+      raw = (mode == kModeFirst) ? reinterpret_cast<const T*>(a.raw) + (long long)cur_y * st.elems : nullptr;
     }
-    const int n = min(kRowsPerIter, min(r_end - r, st.rows - rin));
-    const int c0 = rin * kThreads + tid;
+    const int n = cur.take(st.rows);
+    const int c0 = cur.rin * kThreads + tid;
 
     if (mode == kModeDelta) {
-      uint4 mv[kRowsPerIter];
-      unsigned long long codes[kRowsPerIter];
-      float delta[kRowsPerIter];
-#pragma unroll
-      for (int i = 0; i < kRowsPerIter; ++i) {
-        const int c = c0 + i * kThreads;
-        const bool active = i < n && c < st.chunks;
-        mv[i] = make_uint4(0, 0, 0, 0);
-        delta[i] = 0.0f;
-        codes[i] = 0ull;
-        if (active) {
-          mv[i] = ld_stream(m + (long long)c * kChunk);
-          delta[i] = __ldg(scales + (c >> st.lg_shift));
-        }
-        if (i < n) {
-          const bool warp_words = words_ok && (c - lane + 32 <= st.chunks);
-          codes[i] = load_codes<BITS>(stream, c, lane, active, warp_words);
-        }
-      }
-#pragma unroll
-      for (int i = 0; i < kRowsPerIter; ++i) {
-        const int c = c0 + i * kThreads;
-        if (i < n && c < st.chunks) {
-          float mf[8], q[8];
-          Conv<T>::unpack(mv[i], mf);
-          dequantize8<BITS>(codes[i], delta[i], q);
-#pragma unroll
-          for (int j = 0; j < 8; ++j) mf[j] = __fadd_rn(mf[j], q[j]);
-          const uint4 nv = Conv<T>::pack(mf);
-          st_stream(m + (long long)c * kChunk, nv);
-          st_stream(out + (long long)c * kChunk, nv);
-        }
-      }
+      if ((cur.rin + kRowsPerIter) * kThreads <= st.chunks && n == kRowsPerIter)
+        decode_rows<T, BITS, true>(st, stream, scales, m, out, c0, n, lane, words_ok);
+      else
+        decode_rows<T, BITS, false>(st, stream, scales, m, out, c0, n, lane, words_ok);
     } else {
       // first visit: the raw message becomes m(xi) and the activation; skipped sample: zeros out.
 #pragma unroll
@@ -526,14 +570,14 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(const State st, const 
         if (i < n && c < st.chunks) {
           uint4 v = make_uint4(0, 0, 0, 0);
           if (raw) {
-            v = ld_stream(raw + (long long)c * kChunk);
-            st_stream(m + (long long)c * kChunk, v);
+            v = ld_stream(raw + (size_t)c * kChunk);
+            st_stream(m + (size_t)c * kChunk, v);
           }
-          st_stream(out + (long long)c * kChunk, v);
+          st_stream(out + (size_t)c * kChunk, v);
         }
       }
     }
-    r += n;
+    cur.advance(n, st.rows);
   }
 }
 
@@ -660,28 +704,25 @@ __global__ void __launch_bounds__(kThreads) checksum_kernel(const State st, unsi
 
 inline unsigned grid_x(long long chunks) { return (unsigned)((chunks + kChunksPerCta - 1) / kChunksPerCta); }
 
-// CTAs of `kernel` that fit one multiprocessor (asked once per kernel).
-template <typename K>
-int resident_ctas(K kernel) {
-  static const int n = [kernel] {
-    int v = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, kernel, kThreads, 0) != cudaSuccess || v < 1) v = 1;
-    return v;
-  }();
-  return n;
-}
+// Several waves of short CTAs: the hardware hands out CTAs in order, so the CTAs in flight cover
+// one moving window of memory, and a finished CTA is replaced at once.  A CTA walks
+// kRowsPerCta rows when the call is large (its per-sample work is then paid once per 16384
+// elements), fewer when that would leave multiprocessors idle.
+constexpr int kRowsPerCta = 8;
 
-// One wave: at most sms * resident CTAs, every CTA the same number of rows (the last one the rest).
 template <typename K, typename Args>
 cudaError_t launch_rows(K kernel, const State& st, const Args& a, cudaStream_t s) {
   const long long total = (long long)a.n_batch * st.rows;
   if (total <= 0) return cudaSuccess;
   if (total > 0x7fffffffll) return cudaErrorInvalidValue;
-  const long long wave = (long long)st.sms * resident_ctas(kernel);
-  int per = (int)((total + wave - 1) / wave);
-  if (st.rows_per_cta > 0) per = (int)(st.rows_per_cta < total ? st.rows_per_cta : total);
+  long long per = st.rows_per_cta;
+  if (per <= 0) {
+    per = total / ((long long)st.sms * 12);
+    per = per < kRowsPerIter ? kRowsPerIter : (per > kRowsPerCta ? kRowsPerCta : per);
+  }
+  if (per > total) per = total;
   const unsigned grid = (unsigned)((total + per - 1) / per);
-  kernel<<<grid, kThreads, 0, s>>>(st, a, per);
+  kernel<<<grid, kThreads, 0, s>>>(st, a, (int)per);
   return cudaGetLastError();
 }
 
