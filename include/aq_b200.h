@@ -144,6 +144,26 @@ int aq_dequant_grad(aq_handle* h, const void* packed, const float* scales, int64
  */
 int aq_state_checksum(aq_handle* h, uint64_t* out_host);
 
+/*
+ * The same digest as aq_state_checksum, for callers that must not allocate device memory
+ * when they call: code inside a CUDA-graph capture, a step loop that cannot afford the
+ * device-wide synchronisation an allocation may bring, a process whose memory was all handed
+ * out at start-up.  (The paper has no counterpart; this entry point exists for such callers
+ * only.)  Its working memory is a fixed array inside the library image -- 512 KiB of device
+ * memory that every GPU which loads the library holds until the process exits -- so the call
+ * itself runs no cudaMalloc, cudaFree or other allocating routine.
+ *   - Limit: m of at most 64 GiB (65536 slabs of 1 MiB, one partial sum each); a larger
+ *     state is refused with AQ_EUNSUPPORTED and a message, nothing is launched.
+ *   - The first call on each device looks up the array's device address (once per device,
+ *     with that device current).  Make that first call outside any stream capture.
+ *   - Every call, on any handle, uses the same array and leaves its partial sums there; each
+ *     call rewrites every slot it reads, so nothing has to be cleared.  Calls that overlap
+ *     on one GPU (different streams, different threads) race on the array and return
+ *     garbage: keep them ordered.
+ * Synchronises the handle's stream; *out_host is host memory.
+ */
+int aq_state_checksum_noalloc(aq_handle* h, uint64_t* out_host);
+
 /* Synchronises the stream, returns the sticky AQ_ST_* bits in *bits_host (host) and clears them. */
 int aq_status(aq_handle* h, uint32_t* bits_host);
 

@@ -26,6 +26,7 @@ SIGNATURES = {
     "aq_quant_grad": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_void_p, C.c_void_p]),
     "aq_dequant_grad": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_void_p]),
     "aq_state_checksum": (C.c_int, [C.c_void_p, C.POINTER(C.c_uint64)]),
+    "aq_state_checksum_noalloc": (C.c_int, [C.c_void_p, C.POINTER(C.c_uint64)]),
     "aq_status": (C.c_int, [C.c_void_p, C.POINTER(C.c_uint32)]),
     "aq_last_error": (C.c_char_p, [C.c_void_p]),
     "aq_packed_bytes_per_sample": (C.c_int64, [C.c_void_p]),
@@ -116,6 +117,13 @@ def aq_dequant_grad(h, packed, scales, n_elems, bits, out):
 def aq_state_checksum(h):
     v = C.c_uint64(0)
     _check(h, lib().aq_state_checksum(h, C.byref(v)))
+    return v.value
+
+
+def aq_state_checksum_noalloc(h):
+    """aq_state_checksum through the library's fixed scratch array: no device allocation."""
+    v = C.c_uint64(0)
+    _check(h, lib().aq_state_checksum_noalloc(h, C.byref(v)))
     return v.value
 
 

@@ -5,7 +5,7 @@ import sys
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
-SOURCES = [os.path.join(CSRC, f) for f in ("aq_api.cu", "aq_kernels.cu")]
+SOURCES = [os.path.join(CSRC, f) for f in ("aq_api.cu", "aq_kernels.cu", "aq_noalloc.cu")]
 HEADERS = [os.path.join(CSRC, "aq_internal.h"),
            os.path.join(os.path.dirname(HERE), "include", "aq_b200.h")]
 LIB = os.path.join(HERE, "libaq_b200.so")

@@ -342,3 +342,16 @@ int aq_import_sample(aq_handle* h, int64_t sample_id, const void* m_host, uint8_
 }
 
 }  // extern "C"
+
+// ---- access for entry points that live in other files of the library
+
+namespace aq {
+
+const State* handle_state(aq_handle* h) { return &h->st; }
+cudaStream_t handle_stream(aq_handle* h) { return h->stream; }
+int handle_device(aq_handle* h) { return h->device; }
+
+int handle_fail(aq_handle* h, int code, const char* msg) { return fail(h, code, "%s", msg); }
+
+}  // namespace aq
+

@@ -66,3 +66,12 @@ cudaError_t launch_dequant_grad(int dtype, int bits, int lanes_per_group, const 
 cudaError_t launch_checksum(const State& st, unsigned long long* sum_dev, cudaStream_t s);
 
 }  // namespace aq
+
+// The handle is defined in aq_api.cu; entry points in other files reach it through these.
+struct aq_handle;
+namespace aq {
+const State* handle_state(aq_handle* h);
+cudaStream_t handle_stream(aq_handle* h);
+int handle_device(aq_handle* h);
+int handle_fail(aq_handle* h, int code, const char* msg);   // records msg for aq_last_error, returns code
+}  // namespace aq
