@@ -217,8 +217,7 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
 
-    from dataclasses import replace
-    from paper_2206_01299_b200 import synth
+    from paper_2206_01299_b200 import replicas, synth
     cfg = synth.GPT2_XL
     if args.n_samples:
         cfg = synth.shrink(cfg, args.n_samples)
@@ -240,7 +239,7 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     # data-parallel replicas: every rank owns its own 4096-id shard of a world-times larger id
     # space (weak scaling); sample rows never cross ranks, so the data path has no collective
-    cfg = replace(cfg, stream=rank)
+    cfg = replicas.shard_for_rank(cfg, rank, world)
 
     nb = args.per_launch
     assert cfg.n_samples % MACRO == 0 and MACRO % nb == 0
@@ -373,10 +372,7 @@ def main():
     digests_equal = aq.aq_state_checksum(snd) == aq.aq_state_checksum(rcv)
     assert status == 0 and digests_equal, "sender and receiver state diverged"
 
-    if dist:
-        tmax = torch.tensor([elapsed_ms], device="cuda")
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(tmax.item())
+    elapsed_ms = replicas.max_over_ranks(elapsed_ms, dist, "cuda")
 
     result_extra = {}
     if rank == 0 and not args.skip_aux:
@@ -405,7 +401,7 @@ def main():
     enc_gbs = launch_bytes / (enc_ms * 1e-3) / 1e9
     dec_gbs = launch_bytes / (dec_ms * 1e-3) / 1e9
     traffic = NCU_TRAFFIC_BYTES_PER_ELEMENT["encode"]
-    value = world * args.steps * step_bytes / (elapsed_ms * 1e-3) / 1e9
+    value = replicas.whole_job_rate(args.steps * step_bytes, world, elapsed_ms) / 1e9
     line = {
         "metric": "activation encode+decode GB/s", "value": value, "unit": "GB/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -417,7 +413,7 @@ def main():
                    "m_bytes_per_side": cfg.n_samples * cfg.elems * 2, "steady_epochs_resident": n_arenas,
                    "l2": "inputs larger than L2 (each step touches 315 MB of fresh HBM; no flush needed)",
                    "parallelism": f"dp{world} replicas, no collective"},
-        "samples_per_s": world * args.steps * MACRO / (elapsed_ms * 1e-3),
+        "samples_per_s": replicas.whole_job_rate(args.steps * MACRO, world, elapsed_ms),
         "frac_of_measured_hbm": value / world / peak, "frac_of_8000_spec": value / world / 8000.0,
         "roofline": {"bound": "hbm", "kernel": "encode_kernel", "achieved": enc_gbs, "peak": peak, "unit": "GB/s",
                      "frac": enc_gbs / peak, "peak_kind": peak_kind,
@@ -500,10 +496,8 @@ def run_e2e(aq, torch, cfg, snd, rcv, arena, ids_dev, steps, dist):
         step(t)
     torch.cuda.synchronize()
     dt = time.perf_counter() - t0
-    if dist:
-        tm = torch.tensor([dt], device="cuda")
-        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-        dt = float(tm.item())
+    from paper_2206_01299_b200 import replicas
+    dt = replicas.max_over_ranks(dt, dist, "cuda")
     assert aq.aq_status(snd) == 0 and aq.aq_status(rcv) == 0
     assert aq.aq_state_checksum(snd) == aq.aq_state_checksum(rcv)
     world = dist.get_world_size() if dist else 1

@@ -1,0 +1,154 @@
+"""The 'Pipeline sweep' workload on one GPU (reduced sequence length and id space, same
+structure): 8 stage boundaries, 16 micro-batches per macro-batch, forward 3-bit deltas and
+backward 6-bit direct quantization at every boundary, the wire between sender and receiver
+being a device-to-device byte copy.  Boundaries are independent (one (m, Q) pair per boundary),
+so they run one after the other with one sender/receiver pair alive at a time.
+
+Also here: the two large boundaries at their full id-space size, in the launch shape the
+benchmark times, checked against the oracle on sampled sequences."""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2206_01299_b200 as aq
+from paper_2206_01299_b200 import synth
+from codec_harness import DT, GpuSide, bits16
+
+pytestmark = pytest.mark.gpu
+
+
+def test_pipeline_sweep_boundary_major():
+    seq, n_ids, epochs = 24, 32, 3
+    fwd0 = synth.shrink(synth.SWEEP_FWD, n_ids, seq=seq, epochs=epochs)
+    bwd = replace(synth.SWEEP_BWD, seq=seq)
+    n = fwd0.elems
+    bbits = bwd.bits[0]
+    assert (fwd0.bits, bbits, fwd0.group) == (3, 6, 64)
+    # wire buffers: the sender's and the receiver's ends of the channel
+    tx_p = torch.empty((1, fwd0.packed_bytes), dtype=torch.uint8, device="cuda")
+    tx_s = torch.empty((1, fwd0.groups), dtype=torch.float32, device="cuda")
+    rx_p, rx_s = torch.empty_like(tx_p), torch.empty_like(tx_s)
+    rx_raw = torch.empty((1, seq, fwd0.hidden), dtype=torch.float16, device="cuda")
+    out = torch.empty_like(rx_raw)
+    gtx_p = torch.empty(n * bbits // 8, dtype=torch.uint8, device="cuda")
+    gtx_s = torch.empty(n // bwd.group, dtype=torch.float32, device="cuda")
+    grx_p, grx_s = torch.empty_like(gtx_p), torch.empty_like(gtx_s)
+    gout = torch.empty(n, dtype=torch.float16, device="cuda")
+    digests = []
+    for boundary in range(synth.SWEEP_BOUNDARIES):
+        cfg = replace(fwd0, stream=boundary)
+        gs, gr = GpuSide(cfg, 1), GpuSide(cfg, 1)
+        os_, or_ = (oracle.Side(n_ids, seq, cfg.hidden, cfg.bits, cfg.group, oracle.FP16) for _ in range(2))
+        try:
+            aq.aq_configure(gr.h, aq.AQ_RAW, rx_raw)
+            call = 0
+            for epoch in range(epochs):
+                order = synth.epoch_order(cfg, epoch)
+                for macro in range(n_ids // synth.SWEEP_MICRO_BATCHES):
+                    for mb in range(synth.SWEEP_MICRO_BATCHES):
+                        ids = order[macro * synth.SWEEP_MICRO_BATCHES + mb:][:1].contiguous()
+                        ids_d = ids.cuda()
+                        act = synth.activation(cfg, ids, epoch, device="cuda")
+                        # forward: sender -> channel -> receiver
+                        aq.aq_encode(gs.h, act, ids_d, tx_p, tx_s)
+                        rx_p.copy_(tx_p)
+                        rx_s.copy_(tx_s)
+                        if epoch == 0:
+                            rx_raw.copy_(act)                       # first visit: the message is the activation
+                        aq.aq_decode(gr.h, rx_p, rx_s, ids_d, out)
+                        # backward: receiver -> channel -> sender
+                        grad = synth.gradient(bwd, call, device="cuda", stream=boundary)
+                        aq.aq_quant_grad(gr.h, grad, n, bbits, gtx_p, gtx_s)
+                        grx_p.copy_(gtx_p)
+                        grx_s.copy_(gtx_s)
+                        aq.aq_dequant_grad(gs.h, grx_p, grx_s, n, bbits, gout)
+                        torch.cuda.synchronize()
+                        a_np = bits16(act)
+                        p_o, s_o, _ = os_.encode(a_np, ids.numpy())
+                        out_o, _ = or_.decode(p_o, s_o, ids.numpy(), raw=a_np if epoch == 0 else None)
+                        assert np.array_equal(rx_p.cpu().numpy(), p_o), (boundary, epoch, macro, mb)
+                        assert np.array_equal(rx_s.cpu().numpy().view(np.uint32), s_o.view(np.uint32))
+                        assert np.array_equal(bits16(out), out_o)
+                        gp_o, gs_o = oracle.quant_grad(bits16(grad), bbits, bwd.group, oracle.FP16)
+                        assert np.array_equal(grx_p.cpu().numpy(), gp_o)
+                        assert np.array_equal(grx_s.cpu().numpy().view(np.uint32), gs_o.view(np.uint32))
+                        assert np.array_equal(bits16(gout), oracle.dequant_grad(gp_o, gs_o, n, bbits, bwd.group, oracle.FP16))
+                        assert tx_p.numel() + tx_s.numel() * 4 == n * 3 // 8 + n // 64 * 4     # forward wire bytes
+                        call += 1
+                d = aq.aq_state_checksum(gs.h)
+                assert d == aq.aq_state_checksum(gr.h) == os_.checksum() == or_.checksum()
+            assert aq.aq_status(gs.h) == 0 and aq.aq_status(gr.h) == 0
+            digests.append(d)
+        finally:
+            gs.close()
+            gr.close()
+            os_.close()
+            or_.close()
+    assert len(set(digests)) == synth.SWEEP_BOUNDARIES              # every boundary saw its own data
+
+
+def _full_size_sampled(cfg, per_launch, steps, samples_per_launch):
+    """Full id space, the benchmark's launch shape; the oracle follows only the sampled ids."""
+    od = DT[cfg.dtype][1]
+    gs, gr = GpuSide(cfg, per_launch), GpuSide(cfg, per_launch)
+    packed = torch.empty((per_launch, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
+    scales = torch.empty((per_launch, cfg.groups), dtype=torch.float32, device="cuda")
+    out = torch.empty((per_launch, cfg.seq, cfg.hidden), dtype=cfg.torch_dtype, device="cuda")
+    tracked = {}                                                     # sample id -> (oracle sender, oracle receiver)
+    try:
+        order = synth.epoch_order(cfg, 0)
+        for epoch in range(3):                                        # the same launches each epoch: first visit, then deltas
+            for step in steps:
+                ids = order[step * per_launch:(step + 1) * per_launch].contiguous()
+                act = synth.activation(cfg, ids, epoch, device="cuda")
+                aq.aq_encode(gs.h, act, ids.cuda(), packed, scales)
+                aq.aq_configure(gr.h, aq.AQ_RAW, act if epoch == 0 else None)
+                aq.aq_decode(gr.h, packed, scales, ids.cuda(), out)
+                torch.cuda.synchronize()
+                assert gs.first.cpu().numpy().all() == (epoch == 0)
+                for y in np.linspace(0, per_launch - 1, samples_per_launch).astype(int):
+                    sid = int(ids[y])
+                    if sid not in tracked:
+                        tracked[sid] = tuple(oracle.Side(1, cfg.seq, cfg.hidden, cfg.bits, cfg.group, od) for _ in range(2))
+                    o_s, o_r = tracked[sid]
+                    zero = np.zeros(1, np.int32)
+                    a_np = bits16(act[y:y + 1])
+                    p_o, s_o, f_o = o_s.encode(a_np, zero)
+                    out_o, _ = o_r.decode(p_o, s_o, zero, raw=a_np if epoch == 0 else None)
+                    assert f_o[0] == (epoch == 0)
+                    assert np.array_equal(packed[y].cpu().numpy(), p_o[0]), (epoch, step, y, "packed")
+                    assert np.array_equal(scales[y].cpu().numpy().view(np.uint32), s_o[0].view(np.uint32)), (epoch, step, y)
+                    assert np.array_equal(bits16(out[y]), out_o[0]), (epoch, step, y, "out")
+                    assert np.array_equal(gs.m_row(sid)[0], o_s.m()[0]) and np.array_equal(gr.m_row(sid)[0], o_r.m()[0])
+        assert aq.aq_status(gs.h) == 0 and aq.aq_status(gr.h) == 0
+        assert aq.aq_state_checksum(gs.h) == aq.aq_state_checksum(gr.h)
+        assert aq.aq_state_checksum_noalloc(gs.h) == aq.aq_state_checksum(gs.h)
+    finally:
+        gs.close()
+        gr.close()
+        for pair in tracked.values():
+            for side in pair:
+                side.close()
+
+
+def _needs_gb(gb):
+    free, _ = torch.cuda.mem_get_info()
+    if free < gb * 2 ** 30:
+        pytest.skip(f"needs {gb} GiB of free device memory")
+
+
+def test_gpt2_boundary_full_id_space_in_the_benchmark_launch_shape():
+    """4096 ids (13.4 GB of m per side), 32 micro-batches of 1 x 1024 x 1600 fp16 per launch."""
+    _needs_gb(34)
+    cfg = synth.GPT2_XL
+    _full_size_sampled(cfg, 32, steps=[0, 1, cfg.n_samples // 32 - 1], samples_per_launch=2)
+
+
+def test_deberta_boundary_full_id_space():
+    """32768 ids (25.8 GB of m per side), micro-batch 8 x 256 x 1536 bf16, 2 bit, group 128."""
+    _needs_gb(60)
+    cfg = synth.DEBERTA_XXL
+    _full_size_sampled(cfg, cfg.n_batch, steps=[0, 7, cfg.n_samples // cfg.n_batch - 1], samples_per_launch=3)
