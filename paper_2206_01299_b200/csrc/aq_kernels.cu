@@ -316,26 +316,41 @@ __device__ __forceinline__ unsigned long long begin_call(const State& st) {
   return s_call;
 }
 
-// Mode of sample y of the call, computed by one warp for itself (all 32 lanes call this
-// together).  `why` gets the status bit of a skipped sample.
-__device__ __forceinline__ int resolve_sample(const State& st, const int32_t* __restrict__ ids, int y, int lane,
-                                              bool need_raw, bool have_raw, unsigned long long call,
-                                              long long& id, unsigned& why) {
-  const int32_t my = ids[y];
-  id = my;
+// What a warp reads from memory about sample y of the call.  The loads are issued here and
+// first used in settle_sample, so they can be in flight across the start-of-call barrier.
+struct SampleProbe {
+  int32_t id;
+  int dup;                       // this lane saw the id earlier in the call
+  bool in_range;
+  unsigned long long stamp;
+};
+
+__device__ __forceinline__ SampleProbe probe_sample(const State& st, const int32_t* __restrict__ ids, int y,
+                                                    int lane) {
+  SampleProbe p;
+  p.id = ids[y];
+  p.in_range = p.id >= 0 && (long long)p.id < st.n_samples;
+  p.dup = 0;
+  for (int q = lane; q < y; q += 32) p.dup |= (ids[q] == p.id);
+  p.stamp = p.in_range ? __ldcg(st.seen + p.id) : 0ull;
+  return p;
+}
+
+// Mode of the probed sample, computed by one warp for itself (all 32 lanes call this together).
+// `why` gets the status bit of a skipped sample.
+__device__ __forceinline__ int settle_sample(const SampleProbe& p, bool need_raw, bool have_raw,
+                                             unsigned long long call, long long& id, unsigned& why) {
+  id = p.id;
   why = 0u;
-  if (my < 0 || (long long)my >= st.n_samples) {
+  if (!p.in_range) {
     why = kStBadId;
     return kModeSkip;
   }
-  int dup = 0;
-  for (int p = lane; p < y; p += 32) dup |= (ids[p] == my);
-  if (__any_sync(kFullMask, dup)) {
+  if (__any_sync(kFullMask, p.dup)) {
     why = kStDupId;
     return kModeSkip;
   }
-  const unsigned long long stamp = __ldcg(st.seen + my);
-  if (stamp != 0ull && stamp != call) return kModeDelta;
+  if (p.stamp != 0ull && p.stamp != call) return kModeDelta;
   if (need_raw && !have_raw) {
     why = kStNoRaw;
     return kModeSkip;
@@ -428,14 +443,28 @@ __device__ __forceinline__ void encode_rows(const State& st, const T* __restrict
   }
 }
 
+// CTAs per multiprocessor that the register budget is cut for: the most that compile without
+// spilling (the wide type carries two more guards; fields that straddle words need shuffles).
+template <typename T, int BITS>
+constexpr int encode_ctas_per_sm() {
+  const bool whole_words = BITS == 1 || BITS == 2 || BITS == 4;
+  return !whole_words ? (Conv<T>::kWide ? 3 : 4) : (Conv<T>::kWide ? 5 : 6);
+}
+template <int BITS>
+constexpr int decode_ctas_per_sm() {
+  return (BITS == 1 || BITS == 2 || BITS == 4 || BITS == 8) ? 6 : (BITS == 3 ? 5 : 4);
+}
+
 template <typename T, int BITS, int LPG>
-__global__ void __launch_bounds__(kThreads, (BITS == 3 || BITS >= 5) ? 4 : 6)
+__global__ void __launch_bounds__(kThreads, encode_ctas_per_sm<T, BITS>())
     encode_kernel(const State st, const EncodeArgs a, const int rows_per_cta) {
   const int tid = threadIdx.x;
   const int lane = tid & 31;
-  const unsigned long long call = begin_call(st);
   RowCursor cur(rows_per_cta, a.n_batch * st.rows, st.rows);
+  SampleProbe probe = probe_sample(st, a.ids, cur.y, lane);       // every CTA has at least one row
+  const unsigned long long call = begin_call(st);
   const bool words_ok = (st.packed_bytes & 3) == 0;
+  const int whole_rows = st.chunks / kThreads;                    // rows of a sample without a ragged end
 
   int cur_y = -1, mode = kModeSkip;
   const T* act = nullptr;
@@ -445,27 +474,35 @@ __global__ void __launch_bounds__(kThreads, (BITS == 3 || BITS >= 5) ? 4 : 6)
 
   while (!cur.done()) {
     if (cur.y != cur_y) {
+      if (cur_y >= 0) probe = probe_sample(st, a.ids, cur.y, lane);
       cur_y = cur.y;
       long long id;
       unsigned why;
-      mode = resolve_sample(st, a.ids, cur_y, lane, false, false, call, id, why);
+      mode = settle_sample(probe, false, false, call, id, why);
       if (cur.rin == 0 && tid == 0) publish_sample(st, cur_y, mode, id, why, call, a.first_flags);
       act = reinterpret_cast<const T*>(a.act) + (long long)cur_y * st.elems;
       stream = a.packed + (long long)cur_y * st.packed_bytes;
       scales = a.scales + (long long)cur_y * st.groups;
       m = (mode == kModeSkip) ? nullptr : reinterpret_cast<T*>(st.m) + id * st.elems;
     }
-    const int n = cur.take(st.rows);
-    const int c0 = cur.rin * kThreads + tid;
+    int c0 = cur.rin * kThreads + tid;
 
     if (mode == kModeDelta) {
-      if ((cur.rin + kRowsPerIter) * kThreads <= st.chunks && n == kRowsPerIter)
-        encode_rows<T, BITS, LPG, true>(st, act, m, stream, scales, c0, n, lane, words_ok);
-      else
+      // whole iterations that stay inside this sample and this CTA's range: no bounds to check
+      const int iters = min(cur.r_end - cur.r, whole_rows - cur.rin) / kRowsPerIter;
+      if (iters > 0) {
+        for (int k = 0; k < iters; ++k, c0 += kRowsPerIter * kThreads)
+          encode_rows<T, BITS, LPG, true>(st, act, m, stream, scales, c0, kRowsPerIter, lane, words_ok);
+        cur.advance(iters * kRowsPerIter, st.rows);
+      } else {
+        const int n = cur.take(st.rows);
         encode_rows<T, BITS, LPG, false>(st, act, m, stream, scales, c0, n, lane, words_ok);
+        cur.advance(n, st.rows);
+      }
     } else {
       // first visit: the activation itself becomes m(xi); skipped sample: nothing is stored.
       // Either way the sample's codes and scales are zero.
+      const int n = cur.take(st.rows);
 #pragma unroll
       for (int i = 0; i < kRowsPerIter; ++i) {
         if (i < n) {
@@ -479,8 +516,8 @@ __global__ void __launch_bounds__(kThreads, (BITS == 3 || BITS >= 5) ? 4 : 6)
           store_codes<BITS>(stream, c, lane, active, warp_words, 0ull);
         }
       }
+      cur.advance(n, st.rows);
     }
-    cur.advance(n, st.rows);
   }
 }
 
@@ -527,12 +564,14 @@ __device__ __forceinline__ void decode_rows(const State& st, const uint8_t* __re
 }
 
 template <typename T, int BITS>
-__global__ void __launch_bounds__(kThreads, 6) decode_kernel(const State st, const DecodeArgs a, const int rows_per_cta) {
+__global__ void __launch_bounds__(kThreads, decode_ctas_per_sm<BITS>()) decode_kernel(const State st, const DecodeArgs a, const int rows_per_cta) {
   const int tid = threadIdx.x;
   const int lane = tid & 31;
-  const unsigned long long call = begin_call(st);
   RowCursor cur(rows_per_cta, a.n_batch * st.rows, st.rows);
+  SampleProbe probe = probe_sample(st, a.ids, cur.y, lane);       // every CTA has at least one row
+  const unsigned long long call = begin_call(st);
   const bool words_ok = (st.packed_bytes & 3) == 0;
+  const int whole_rows = st.chunks / kThreads;
 
   int cur_y = -1, mode = kModeSkip;
   T* out = nullptr;
@@ -543,10 +582,11 @@ __global__ void __launch_bounds__(kThreads, 6) decode_kernel(const State st, con
 
   while (!cur.done()) {
     if (cur.y != cur_y) {
+      if (cur_y >= 0) probe = probe_sample(st, a.ids, cur.y, lane);
       cur_y = cur.y;
       long long id;
       unsigned why;
-      mode = resolve_sample(st, a.ids, cur_y, lane, true, a.raw != nullptr, call, id, why);
+      mode = settle_sample(probe, true, a.raw != nullptr, call, id, why);
       if (cur.rin == 0 && tid == 0) publish_sample(st, cur_y, mode, id, why, call, a.first_flags);
       out = reinterpret_cast<T*>(a.out) + (long long)cur_y * st.elems;
       stream = a.packed + (long long)cur_y * st.packed_bytes;
@@ -554,16 +594,22 @@ __global__ void __launch_bounds__(kThreads, 6) decode_kernel(const State st, con
       m = (mode == kModeSkip) ? nullptr : reinterpret_cast<T*>(st.m) + id * st.elems;
       raw = (mode == kModeFirst) ? reinterpret_cast<const T*>(a.raw) + (long long)cur_y * st.elems : nullptr;
     }
-    const int n = cur.take(st.rows);
-    const int c0 = cur.rin * kThreads + tid;
+    int c0 = cur.rin * kThreads + tid;
 
     if (mode == kModeDelta) {
-      if ((cur.rin + kRowsPerIter) * kThreads <= st.chunks && n == kRowsPerIter)
-        decode_rows<T, BITS, true>(st, stream, scales, m, out, c0, n, lane, words_ok);
-      else
+      const int iters = min(cur.r_end - cur.r, whole_rows - cur.rin) / kRowsPerIter;
+      if (iters > 0) {
+        for (int k = 0; k < iters; ++k, c0 += kRowsPerIter * kThreads)
+          decode_rows<T, BITS, true>(st, stream, scales, m, out, c0, kRowsPerIter, lane, words_ok);
+        cur.advance(iters * kRowsPerIter, st.rows);
+      } else {
+        const int n = cur.take(st.rows);
         decode_rows<T, BITS, false>(st, stream, scales, m, out, c0, n, lane, words_ok);
+        cur.advance(n, st.rows);
+      }
     } else {
       // first visit: the raw message becomes m(xi) and the activation; skipped sample: zeros out.
+      const int n = cur.take(st.rows);
 #pragma unroll
       for (int i = 0; i < kRowsPerIter; ++i) {
         const int c = c0 + i * kThreads;
@@ -576,8 +622,8 @@ __global__ void __launch_bounds__(kThreads, 6) decode_kernel(const State st, con
           st_stream(out + (size_t)c * kChunk, v);
         }
       }
+      cur.advance(n, st.rows);
     }
-    cur.advance(n, st.rows);
   }
 }
 
