@@ -9,10 +9,10 @@
 // leave as whole 32-bit words, m is read and rewritten in place by the same thread in one
 // pass, and the quantizer core is written for few instructions (see quantize8).
 //
-// encode / decode run as one wave of CTAs; each CTA walks a contiguous range of "rows"
-// (256 consecutive chunks of one sample), so the per-sample work (id lookup, first-visit
-// test) is done once per CTA and sample, by every warp for itself: the kernels have one
-// block barrier, at their start, and no wait on another CTA.
+// encode / decode run as several waves of short CTAs; each CTA walks a contiguous range of
+// "rows" (256 consecutive chunks of one sample), so the per-sample work (id lookup,
+// first-visit test) is done once per CTA and sample, by every warp for itself: the kernels
+// have one block barrier, at their very end, and no wait on another CTA.
 //
 // Arithmetic: one IEEE binary32 rounding per operation (explicit _rn / _rd intrinsics;
 // the one explicit fused multiply-add is exact-equivalent, see quantize8), so the result
@@ -300,20 +300,20 @@ __device__ __forceinline__ void st_stream(void* p, const uint4& v) { __stcs(rein
 
 // ------------------------------------------------------------------ calls and samples (Algorithm 1, "if xi not seen before")
 
-// Number of the running call, the same in every thread of the grid.  The counter in global
-// memory may only move on after every CTA has read it: each CTA takes a ticket after its
-// read and the CTA that draws the last one (the counter wraps back to 0; nobody waits)
+// Number of the running call: every thread reads the counter for itself, so no warp waits
+// for another one at the start of the kernel.
+__device__ __forceinline__ unsigned long long begin_call(const State& st) { return __ldcg(st.call_no); }
+
+// The counter may only move on after every thread of the grid has read it.  A CTA takes a
+// ticket once all its threads have finished (the barrier: a thread that is done has done its
+// read) and the CTA that draws the last one (the ticket counter wraps back to 0; nobody waits)
 // stores the next call number.
-__device__ __forceinline__ unsigned long long begin_call(const State& st) {
-  __shared__ unsigned long long s_call;
-  if (threadIdx.x == 0) {
-    const unsigned long long c = __ldcg(st.call_no);
-    s_call = c;
-    __threadfence();
-    if (atomicInc(st.ticket, gridDim.x - 1u) == gridDim.x - 1u) *st.call_no = c + 1ull;
-  }
+__device__ __forceinline__ void end_call(const State& st, unsigned long long call) {
   __syncthreads();
-  return s_call;
+  if (threadIdx.x == 0) {
+    __threadfence();
+    if (atomicInc(st.ticket, gridDim.x - 1u) == gridDim.x - 1u) *st.call_no = call + 1ull;
+  }
 }
 
 // What a warp reads from memory about sample y of the call.  The loads are issued here and
@@ -519,6 +519,7 @@ __global__ void __launch_bounds__(kThreads, encode_ctas_per_sm<T, BITS>())
       cur.advance(n, st.rows);
     }
   }
+  end_call(st, call);
 }
 
 // ------------------------------------------------------------------ decode (receiver)
@@ -625,6 +626,7 @@ __global__ void __launch_bounds__(kThreads, decode_ctas_per_sm<BITS>()) decode_k
       cur.advance(n, st.rows);
     }
   }
+  end_call(st, call);
 }
 
 // ------------------------------------------------------------------ backward direction: direct quantization
