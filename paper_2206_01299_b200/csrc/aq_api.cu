@@ -119,16 +119,15 @@ aq_handle* aq_create(int64_t n_samples, int seq, int hidden, int bits, int group
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&st.sms, cudaDevAttrMultiProcessorCount, h->device);
   const size_t m_bytes = (size_t)n_samples * (size_t)st.elems * 2;
   const size_t seen_bytes = (size_t)n_samples * sizeof(unsigned long long);
-  const unsigned long long first_call = aq::kFirstCall;
   if (e == cudaSuccess) e = cudaMalloc(&st.m, m_bytes);
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&st.seen), seen_bytes);
-  if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&st.call_no), sizeof(unsigned long long));
-  if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&st.status), 2 * sizeof(uint32_t));
+  if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&st.arrivals), sizeof(unsigned long long));
+  if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&st.status), sizeof(uint32_t));
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&h->sum_dev), sizeof(unsigned long long));
   if (e == cudaSuccess) e = cudaMemset(st.m, 0, m_bytes);                      // "initialized to 0"
   if (e == cudaSuccess) e = cudaMemset(st.seen, 0, seen_bytes);
-  if (e == cudaSuccess) e = cudaMemset(st.status, 0, 2 * sizeof(uint32_t));
-  if (e == cudaSuccess) e = cudaMemcpy(st.call_no, &first_call, sizeof(first_call), cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaMemset(st.status, 0, sizeof(uint32_t));
+  if (e == cudaSuccess) e = cudaMemset(st.arrivals, 0, sizeof(unsigned long long));
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
     cuda_fail(nullptr, e, "aq_create");
@@ -136,7 +135,6 @@ aq_handle* aq_create(int64_t n_samples, int seq, int hidden, int bits, int group
     aq_destroy(h);
     return nullptr;
   }
-  st.ticket = st.status + 1;
   return h;
 }
 
@@ -147,7 +145,7 @@ void aq_destroy(aq_handle* h) {
   free_staging(h);
   cudaFree(h->st.m);
   cudaFree(h->st.seen);
-  cudaFree(h->st.call_no);
+  cudaFree(h->st.arrivals);
   cudaFree(h->st.status);
   cudaFree(h->sum_dev);
   delete h;

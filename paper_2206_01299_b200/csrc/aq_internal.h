@@ -17,14 +17,15 @@ constexpr int kMaxBatch = 4096;      // samples per encode / decode call
 // CTA of that call, so the stamp may be written while other CTAs are reading it.
 constexpr unsigned long long kImportedStamp = 1ull;
 constexpr unsigned long long kFirstCall = 2ull;
+// what one encode / decode launch adds to the handle's arrival counter; also the largest grid
+constexpr unsigned long long kCallQuantum = 1ull << 20;
 
 // State of one side of a boundary, as the kernels see it.
 struct State {
   void* m;                        // T[n_samples][elems]
   unsigned long long* seen;       // [n_samples] stamps
-  unsigned long long* call_no;    // number of the next encode / decode call (starts at kFirstCall)
+  unsigned long long* arrivals;   // grows by kCallQuantum per encode / decode launch (starts at 0)
   uint32_t* status;               // sticky AQ_ST_* bits
-  uint32_t* ticket;               // CTA arrival counter of the running call (returns to 0 by itself)
   long long n_samples;
   long long elems;                // seq * hidden
   long long packed_bytes;         // per sample

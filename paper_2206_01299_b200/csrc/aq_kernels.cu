@@ -12,7 +12,7 @@
 // encode / decode run as several waves of short CTAs; each CTA walks a contiguous range of
 // "rows" (256 consecutive chunks of one sample), so the per-sample work (id lookup,
 // first-visit test) is done once per CTA and sample, by every warp for itself: the kernels
-// have one block barrier, at their very end, and no wait on another CTA.
+// have one block barrier, at their start, and no wait on another CTA.
 //
 // Arithmetic: one IEEE binary32 rounding per operation (explicit _rn / _rd intrinsics;
 // the one explicit fused multiply-add is exact-equivalent, see quantize8), so the result
@@ -300,20 +300,24 @@ __device__ __forceinline__ void st_stream(void* p, const uint4& v) { __stcs(rein
 
 // ------------------------------------------------------------------ calls and samples (Algorithm 1, "if xi not seen before")
 
-// Number of the running call: every thread reads the counter for itself, so no warp waits
-// for another one at the start of the kernel.
-__device__ __forceinline__ unsigned long long begin_call(const State& st) { return __ldcg(st.call_no); }
-
-// The counter may only move on after every thread of the grid has read it.  A CTA takes a
-// ticket once all its threads have finished (the barrier: a thread that is done has done its
-// read) and the CTA that draws the last one (the ticket counter wraps back to 0; nobody waits)
-// stores the next call number.
-__device__ __forceinline__ void end_call(const State& st, unsigned long long call) {
-  __syncthreads();
+// Number of the running call, the same in every thread of the grid, different for every launch
+// on the handle.  The handle keeps one 64-bit arrival counter that only grows.  Each CTA adds
+// its share of kCallQuantum to it, the shares of one grid adding up to exactly kCallQuantum
+// (CTA 0 takes the remainder), so the counter is a multiple of kCallQuantum between launches
+// and every value a CTA gets back from its add lies in [c * kCallQuantum, (c+1) * kCallQuantum)
+// for the same c: the number of launches before this one.  No CTA has to be the last one, nothing
+// is reset, and a replayed CUDA graph counts like any other launch.  One atomic per CTA, issued
+// by thread 0 while the other warps are already fetching their sample's id; one barrier hands
+// the result to the CTA.
+__device__ __forceinline__ unsigned long long begin_call(const State& st) {
+  __shared__ unsigned long long s_call;
   if (threadIdx.x == 0) {
-    __threadfence();
-    if (atomicInc(st.ticket, gridDim.x - 1u) == gridDim.x - 1u) *st.call_no = call + 1ull;
+    const unsigned long long share = kCallQuantum / gridDim.x;
+    const unsigned long long mine = blockIdx.x == 0 ? kCallQuantum - share * (gridDim.x - 1u) : share;
+    s_call = atomicAdd(st.arrivals, mine) / kCallQuantum + kFirstCall;
   }
+  __syncthreads();
+  return s_call;
 }
 
 // What a warp reads from memory about sample y of the call.  The loads are issued here and
@@ -519,7 +523,6 @@ __global__ void __launch_bounds__(kThreads, encode_ctas_per_sm<T, BITS>())
       cur.advance(n, st.rows);
     }
   }
-  end_call(st, call);
 }
 
 // ------------------------------------------------------------------ decode (receiver)
@@ -626,7 +629,6 @@ __global__ void __launch_bounds__(kThreads, decode_ctas_per_sm<BITS>()) decode_k
       cur.advance(n, st.rows);
     }
   }
-  end_call(st, call);
 }
 
 // ------------------------------------------------------------------ backward direction: direct quantization
@@ -769,6 +771,7 @@ cudaError_t launch_rows(K kernel, const State& st, const Args& a, cudaStream_t s
     per = per < kRowsPerIter ? kRowsPerIter : (per > kRowsPerCta ? kRowsPerCta : per);
   }
   if (per > total) per = total;
+  if ((total + per - 1) / per > (long long)kCallQuantum) per = (total + kCallQuantum - 1) / kCallQuantum;
   const unsigned grid = (unsigned)((total + per - 1) / per);
   kernel<<<grid, kThreads, 0, s>>>(st, a, (int)per);
   return cudaGetLastError();

@@ -274,3 +274,44 @@ def test_import_export_round_trip():
     finally:
         a.close()
         b.close()
+
+
+def test_replayed_cuda_graph_counts_every_replay_as_a_call():
+    """One captured encode + decode, replayed: the first replay is a first visit, the later ones
+    are delta visits of the same activation (and a second graph, other ids, interleaves)."""
+    cfg = synth.Boundary("graph", 6, 2, 5, 320, "fp16", 3, 64, 1, "outlier", 0.2, seed=61)
+    stream = torch.cuda.Stream()
+    gs, gr = GpuSide(cfg, 2, stream), GpuSide(cfg, 2, stream)
+    os_, or_ = (oracle.Side(6, 5, 320, 3, 64, oracle.FP16) for _ in range(2))
+    try:
+        graphs = []
+        for ids_list, epoch in (([4, 1], 0), ([2, 4], 1)):
+            ids = torch.tensor(ids_list, dtype=torch.int32)
+            act = synth.activation(cfg, ids, epoch, device="cuda")
+            ids_d = ids.cuda()
+            packed = torch.empty((2, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
+            scales = torch.empty((2, cfg.groups), dtype=torch.float32, device="cuda")
+            out = torch.empty((2, cfg.seq, cfg.hidden), dtype=torch.float16, device="cuda")
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                aq.aq_configure(gr.h, aq.AQ_RAW, act)
+                aq.aq_encode(gs.h, act, ids_d, packed, scales)
+                aq.aq_decode(gr.h, packed, scales, ids_d, out)
+            graphs.append((g, ids, act, packed, scales, out, ids_d))     # the graph reads ids_d: keep it alive
+        for which in (0, 0, 1, 0, 1, 1):
+            g, ids, act, packed, scales, out, _ = graphs[which]
+            aq.aq_configure(gr.h, aq.AQ_RAW, act)            # host-side setting only; the graph holds its own pointer
+            g.replay()
+            torch.cuda.synchronize()
+            p_o, s_o, f_o = os_.encode(bits16(act), ids.numpy())
+            out_o, fr_o = or_.decode(p_o, s_o, ids.numpy(), raw=bits16(act))
+            assert np.array_equal(packed.cpu().numpy(), p_o)
+            assert np.array_equal(scales.cpu().numpy().view(np.uint32), s_o.view(np.uint32))
+            assert np.array_equal(bits16(out), out_o)
+            assert np.array_equal(gs.first.cpu().numpy(), f_o) and np.array_equal(gr.first.cpu().numpy(), fr_o)
+        assert aq.aq_state_checksum(gs.h) == aq.aq_state_checksum(gr.h) == os_.checksum() == or_.checksum()
+        assert np.array_equal(gs.m_all(), os_.m())
+    finally:
+        gs.close()
+        gr.close()
