@@ -79,7 +79,7 @@ enum {
   AQ_FIRST_FLAGS = 5,    /* device pointer uint8[n_batch] or 0: aq_encode / aq_decode write 1 for
                             each sample that took the first-visit path, else 0 */
   AQ_ROWS_PER_CTA = 6    /* tuning: rows (256 chunks = 2048 elements each) that one CTA of aq_encode /
-                            aq_decode walks; 0 (default) = chosen from the size of the call (2..8) */
+                            aq_decode walks; 0 (default) = chosen from the size of the call (2..4) */
 };
 enum { AQ_FP16 = 0, AQ_BF16 = 1 };
 

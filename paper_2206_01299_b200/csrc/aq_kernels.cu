@@ -756,9 +756,9 @@ inline unsigned grid_x(long long chunks) { return (unsigned)((chunks + kChunksPe
 
 // Several waves of short CTAs: the hardware hands out CTAs in order, so the CTAs in flight cover
 // one moving window of memory, and a finished CTA is replaced at once.  A CTA walks
-// kRowsPerCta rows when the call is large (its per-sample work is then paid once per 16384
+// kRowsPerCta rows when the call is large (its per-sample work is then paid once per 8192
 // elements), fewer when that would leave multiprocessors idle.
-constexpr int kRowsPerCta = 8;
+constexpr int kRowsPerCta = 4;
 
 template <typename K, typename Args>
 cudaError_t launch_rows(K kernel, const State& st, const Args& a, cudaStream_t s) {
