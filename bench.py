@@ -28,7 +28,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-MACRO = 32            # micro-batches per macro-batch (GPT2 fine-tuning setting of the paper)
+MACRO = 32            # sequences per step: the macro-batch (32 x micro-batch 1 in the paper's GPT2 runs)
+# name -> (recipe in synth, sequences per macro-batch, label); the paper's DeBERTa/QNLI runs use macro-batch 64
+WORKLOADS = {"gpt2": ("GPT2_XL", 32, "GPT2-1.5B-shaped boundary (configs[1])"),
+             "deberta": ("DEBERTA_XXL", 64, "DeBERTa-1.5B-shaped boundary (configs[2])")}
 FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the named kernel, from the ncu
@@ -43,7 +46,8 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=16)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--n-samples", type=int, default=None, help="shrink the id space (profiling runs)")
-    ap.add_argument("--per-launch", type=int, default=MACRO, help="micro-batches handed to one aq_encode call")
+    ap.add_argument("--workload", default="gpt2", choices=sorted(WORKLOADS))
+    ap.add_argument("--per-launch", type=int, default=0, help="sequences handed to one aq_encode call (0 = the whole macro-batch)")
     ap.add_argument("--graph", action="store_true", help="replay each step as a captured CUDA graph")
     ap.add_argument("--rows-per-cta", type=int, default=0, help="AQ_ROWS_PER_CTA of both handles (0 = library default)")
     ap.add_argument("--skip-cpu", action="store_true")
@@ -199,7 +203,7 @@ def run_reference(args, cfg):
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": elapsed / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": "GPT2-1.5B-shaped boundary (configs[1]), CPU oracle on a bounded sample",
+        "config": {"workload": WORKLOADS[args.workload][2] + ", CPU oracle on a bounded sample",
                    "hidden": cfg.hidden, "seq": cfg.seq, "bits": cfg.bits, "group": cfg.group,
                    "act_dtype": cfg.dtype},
         "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
@@ -218,7 +222,9 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
 
     from paper_2206_01299_b200 import replicas, synth
-    cfg = synth.GPT2_XL
+    global MACRO
+    recipe, MACRO, label = WORKLOADS[args.workload]
+    cfg = getattr(synth, recipe)
     if args.n_samples:
         cfg = synth.shrink(cfg, args.n_samples)
 
@@ -241,12 +247,14 @@ def main():
     # space (weak scaling); sample rows never cross ranks, so the data path has no collective
     cfg = replicas.shard_for_rank(cfg, rank, world)
 
-    nb = args.per_launch
+    nb = args.per_launch or MACRO
     assert cfg.n_samples % MACRO == 0 and MACRO % nb == 0
     steps_per_epoch = cfg.n_samples // MACRO
     launches_per_step = MACRO // nb
     total_steps = args.steps + args.warmup
-    n_arenas = min(4, (total_steps + steps_per_epoch - 1) // steps_per_epoch)
+    # resident steady-state epochs: as many as the timed steps need, at most 4 (2 for the 26 GB boundary)
+    max_arenas = 4 if cfg.n_samples * cfg.elems * 2 < 20e9 else 2
+    n_arenas = min(max_arenas, (total_steps + steps_per_epoch - 1) // steps_per_epoch)
     stream = torch.cuda.Stream()
     bpe = bytes_per_element(cfg.bits, cfg.group)
     step_bytes = 2 * MACRO * cfg.elems * bpe          # encode + decode
@@ -394,6 +402,7 @@ def main():
 
     result_extra = {}
     if rank == 0 and not args.skip_aux:
+        result_extra["isolated_call"] = isolated_calls(aq, torch, stream, snd, rcv, cfg, arenas[0], id_lists[0])
         result_extra["aux"] = aux_kernels(aq, torch, synth, stream, snd, cfg)
 
     # ---- end to end through the host-buffer entry points (pinned host memory both ways)
@@ -425,11 +434,11 @@ def main():
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": "GPT2-1.5B-shaped boundary (configs[1])", "hidden": cfg.hidden, "seq": cfg.seq,
-                   "micro_batch": cfg.n_batch, "micro_batches_per_step": MACRO, "micro_batches_per_launch": nb, "cuda_graph": bool(args.graph),
+        "config": {"workload": label, "hidden": cfg.hidden, "seq": cfg.seq,
+                   "micro_batch": cfg.n_batch, "sequences_per_step": MACRO, "sequences_per_launch": nb, "cuda_graph": bool(args.graph),
                    "act_dtype": cfg.dtype, "bits": cfg.bits, "group": cfg.group, "n_samples_per_side": cfg.n_samples,
                    "m_bytes_per_side": cfg.n_samples * cfg.elems * 2, "steady_epochs_resident": n_arenas,
-                   "l2": "inputs larger than L2 (each step touches 315 MB of fresh HBM; no flush needed)",
+                   "l2": f"inputs larger than L2 (each step touches {int(MACRO * cfg.elems * 6 / 1e6)} MB of fresh HBM; no flush needed)",
                    "parallelism": f"dp{world} replicas, no collective"},
         "samples_per_s": replicas.whole_job_rate(args.steps * MACRO, world, elapsed_ms),
         "frac_of_measured_hbm": value / world / peak, "frac_of_8000_spec": value / world / 8000.0,
@@ -445,6 +454,35 @@ def main():
     }
     line.update(result_extra)
     print(json.dumps(line))
+
+
+def isolated_calls(aq, torch, stream, snd, rcv, cfg, arena, ids_dev, reps=40):
+    """Latency of one micro-batch call on an idle GPU (the workload's own micro-batch size):
+    event, aq_encode, event, aq_decode, event, synchronise; median over `reps` calls."""
+    nb = cfg.n_batch
+    for h in (snd, rcv):
+        aq.aq_configure(h, aq.AQ_BATCH, nb)
+    packed = torch.empty((nb, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
+    scales = torch.empty((nb, cfg.groups), dtype=torch.float32, device="cuda")
+    out = torch.empty((nb, cfg.seq, cfg.hidden), dtype=cfg.torch_dtype, device="cuda")
+    enc, dec = [], []
+    with torch.cuda.stream(stream):
+        for r in range(reps + 5):
+            lo = (r * 37 % (cfg.n_samples // nb)) * nb
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+            e[0].record(stream)
+            aq.aq_encode(snd, arena[lo:lo + nb], ids_dev[lo:lo + nb], packed, scales)
+            e[1].record(stream)
+            aq.aq_decode(rcv, packed, scales, ids_dev[lo:lo + nb], out)
+            e[2].record(stream)
+            torch.cuda.synchronize()
+            if r >= 5:
+                enc.append(e[0].elapsed_time(e[1]) * 1e3)
+                dec.append(e[1].elapsed_time(e[2]) * 1e3)
+    bytes_call = nb * cfg.elems * bytes_per_element(cfg.bits, cfg.group)
+    enc_us, dec_us = statistics.median(enc), statistics.median(dec)
+    return {"sequences_per_call": nb, "encode_us": enc_us, "decode_us": dec_us,
+            "encode_GB/s": bytes_call / enc_us / 1e3, "decode_GB/s": bytes_call / dec_us / 1e3}
 
 
 def aux_kernels(aq, torch, synth, stream, h, cfg):

@@ -9,10 +9,10 @@
 // leave as whole 32-bit words, m is read and rewritten in place by the same thread in one
 // pass, and the quantizer core is written for few instructions (see quantize8).
 //
-// encode / decode run as several waves of short CTAs; each CTA walks a contiguous range of
-// "rows" (256 consecutive chunks of one sample), so the per-sample work (id lookup,
-// first-visit test) is done once per CTA and sample, by every warp for itself: the kernels
-// have one block barrier, at their start, and no wait on another CTA.
+// encode / decode run as several waves of short CTAs on a (rows, samples) grid; each CTA walks
+// a few "rows" (256 consecutive chunks) of one sample, so the per-sample work (id lookup,
+// first-visit test) is done once per CTA, by every warp for itself: the kernels have one
+// block barrier, at their start, and no wait on another CTA.
 //
 // Arithmetic: one IEEE binary32 rounding per operation (explicit _rn / _rd intrinsics;
 // the one explicit fused multiply-add is exact-equivalent, see quantize8), so the result
@@ -32,6 +32,13 @@ constexpr int kChunksPerThread = 2;                      // grad kernels: chunks
 constexpr int kChunksPerCta = kThreads * kChunksPerThread;
 
 enum { kModeDelta = 0, kModeFirst = 1, kModeSkip = 2 };
+
+// What the launch layer decides for one encode / decode launch.
+struct LaunchPlan {
+  int rows_per_cta;        // rows of one sample that a CTA walks; grid = (ceil(rows / rows_per_cta), n_batch)
+  unsigned share;          // what a CTA adds to the arrival counter ...
+  unsigned first_share;    // ... and what CTA (0,0) adds, so that the grid adds kCallQuantum in all
+};
 enum { kStBadId = 1, kStDupId = 2, kStNoRaw = 4 };
 
 // ------------------------------------------------------------------ 16-bit types
@@ -303,18 +310,17 @@ __device__ __forceinline__ void st_stream(void* p, const uint4& v) { __stcs(rein
 // Number of the running call, the same in every thread of the grid, different for every launch
 // on the handle.  The handle keeps one 64-bit arrival counter that only grows.  Each CTA adds
 // its share of kCallQuantum to it, the shares of one grid adding up to exactly kCallQuantum
-// (CTA 0 takes the remainder), so the counter is a multiple of kCallQuantum between launches
-// and every value a CTA gets back from its add lies in [c * kCallQuantum, (c+1) * kCallQuantum)
-// for the same c: the number of launches before this one.  No CTA has to be the last one, nothing
-// is reset, and a replayed CUDA graph counts like any other launch.  One atomic per CTA, issued
-// by thread 0 while the other warps are already fetching their sample's id; one barrier hands
-// the result to the CTA.
-__device__ __forceinline__ unsigned long long begin_call(const State& st) {
+// (the first CTA takes the remainder; the launch layer works the shares out), so the counter is
+// a multiple of kCallQuantum between launches and every value a CTA gets back from its add lies
+// in [c * kCallQuantum, (c+1) * kCallQuantum) for the same c: the number of launches before
+// this one.  No CTA has to be the last one, nothing is reset, and a replayed CUDA graph counts
+// like any other launch.  One atomic per CTA, issued by thread 0 while the other warps are
+// already fetching their sample's id; one barrier hands the result to the CTA.
+__device__ __forceinline__ unsigned long long begin_call(const State& st, const LaunchPlan& plan) {
   __shared__ unsigned long long s_call;
   if (threadIdx.x == 0) {
-    const unsigned long long share = kCallQuantum / gridDim.x;
-    const unsigned long long mine = blockIdx.x == 0 ? kCallQuantum - share * (gridDim.x - 1u) : share;
-    s_call = atomicAdd(st.arrivals, mine) / kCallQuantum + kFirstCall;
+    const unsigned mine = (blockIdx.x | blockIdx.y) == 0 ? plan.first_share : plan.share;
+    s_call = atomicAdd(st.arrivals, (unsigned long long)mine) / kCallQuantum + kFirstCall;
   }
   __syncthreads();
   return s_call;
@@ -369,34 +375,6 @@ __device__ __forceinline__ void publish_sample(const State& st, int y, int mode,
   if (first_flags) first_flags[y] = (uint8_t)(mode == kModeFirst);
   if (mode == kModeFirst) st.seen[id] = call;
 }
-
-// ------------------------------------------------------------------ row walk shared by encode and decode
-
-// Position of a CTA inside its contiguous range of rows.  A row is kThreads consecutive
-// chunks of one sample; the last row of a sample may be ragged.
-struct RowCursor {
-  int r, r_end;      // global row index and end of the CTA's range
-  int y, rin;        // sample of the call and row inside the sample
-  __device__ __forceinline__ RowCursor(int rows_per_cta, int total_rows, int rows_per_sample) {
-    r = blockIdx.x * rows_per_cta;
-    r_end = min(total_rows, r + rows_per_cta);
-    y = r / rows_per_sample;
-    rin = r - y * rows_per_sample;
-  }
-  __device__ __forceinline__ bool done() const { return r >= r_end; }
-  // rows handled by the next iteration: they belong to one sample
-  __device__ __forceinline__ int take(int rows_per_sample) const {
-    return min(kRowsPerIter, min(r_end - r, rows_per_sample - rin));
-  }
-  __device__ __forceinline__ void advance(int n, int rows_per_sample) {
-    r += n;
-    rin += n;
-    if (rin >= rows_per_sample) {
-      rin = 0;
-      ++y;
-    }
-  }
-};
 
 // ------------------------------------------------------------------ encode (sender)
 
@@ -461,66 +439,46 @@ constexpr int decode_ctas_per_sm() {
 
 template <typename T, int BITS, int LPG>
 __global__ void __launch_bounds__(kThreads, encode_ctas_per_sm<T, BITS>())
-    encode_kernel(const State st, const EncodeArgs a, const int rows_per_cta) {
+    encode_kernel(const State st, const EncodeArgs a, const LaunchPlan plan) {
   const int tid = threadIdx.x;
   const int lane = tid & 31;
-  RowCursor cur(rows_per_cta, a.n_batch * st.rows, st.rows);
-  SampleProbe probe = probe_sample(st, a.ids, cur.y, lane);       // every CTA has at least one row
-  const unsigned long long call = begin_call(st);
+  const int y = blockIdx.y;                                       // sample of the call
+  const SampleProbe probe = probe_sample(st, a.ids, y, lane);
+  const unsigned long long call = begin_call(st, plan);
+  long long id;
+  unsigned why;
+  const int mode = settle_sample(probe, false, false, call, id, why);
+  if (blockIdx.x == 0 && tid == 0) publish_sample(st, y, mode, id, why, call, a.first_flags);
+
+  const T* act = reinterpret_cast<const T*>(a.act) + (size_t)y * (size_t)st.elems;
+  uint8_t* stream = a.packed + (size_t)y * (size_t)st.packed_bytes;
+  float* scales = a.scales + (size_t)y * (size_t)st.groups;
   const bool words_ok = (st.packed_bytes & 3) == 0;
-  const int whole_rows = st.chunks / kThreads;                    // rows of a sample without a ragged end
+  int r = blockIdx.x * plan.rows_per_cta;                         // this CTA's rows of the sample: [r, r_end)
+  const int r_end = min(st.rows, r + plan.rows_per_cta);
 
-  int cur_y = -1, mode = kModeSkip;
-  const T* act = nullptr;
-  T* m = nullptr;
-  uint8_t* stream = nullptr;
-  float* scales = nullptr;
-
-  while (!cur.done()) {
-    if (cur.y != cur_y) {
-      if (cur_y >= 0) probe = probe_sample(st, a.ids, cur.y, lane);
-      cur_y = cur.y;
-      long long id;
-      unsigned why;
-      mode = settle_sample(probe, false, false, call, id, why);
-      if (cur.rin == 0 && tid == 0) publish_sample(st, cur_y, mode, id, why, call, a.first_flags);
-      act = reinterpret_cast<const T*>(a.act) + (long long)cur_y * st.elems;
-      stream = a.packed + (long long)cur_y * st.packed_bytes;
-      scales = a.scales + (long long)cur_y * st.groups;
-      m = (mode == kModeSkip) ? nullptr : reinterpret_cast<T*>(st.m) + id * st.elems;
-    }
-    int c0 = cur.rin * kThreads + tid;
-
-    if (mode == kModeDelta) {
-      // whole iterations that stay inside this sample and this CTA's range: no bounds to check
-      const int iters = min(cur.r_end - cur.r, whole_rows - cur.rin) / kRowsPerIter;
-      if (iters > 0) {
-        for (int k = 0; k < iters; ++k, c0 += kRowsPerIter * kThreads)
-          encode_rows<T, BITS, LPG, true>(st, act, m, stream, scales, c0, kRowsPerIter, lane, words_ok);
-        cur.advance(iters * kRowsPerIter, st.rows);
-      } else {
-        const int n = cur.take(st.rows);
-        encode_rows<T, BITS, LPG, false>(st, act, m, stream, scales, c0, n, lane, words_ok);
-        cur.advance(n, st.rows);
+  if (mode == kModeDelta) {
+    T* m = reinterpret_cast<T*>(st.m) + (size_t)id * (size_t)st.elems;
+    // whole iterations first (rows without a ragged end: no bounds to check), then the rest
+    const int whole_end = min(r_end, st.chunks / kThreads);
+    for (; r + kRowsPerIter <= whole_end; r += kRowsPerIter)
+      encode_rows<T, BITS, LPG, true>(st, act, m, stream, scales, r * kThreads + tid, kRowsPerIter, lane, words_ok);
+    for (; r < r_end; r += kRowsPerIter)
+      encode_rows<T, BITS, LPG, false>(st, act, m, stream, scales, r * kThreads + tid, min(kRowsPerIter, r_end - r),
+                                       lane, words_ok);
+  } else {
+    // first visit: the activation itself becomes m(xi); skipped sample: nothing is stored.
+    // Either way the sample's codes and scales are zero.
+    T* m = (mode == kModeFirst) ? reinterpret_cast<T*>(st.m) + (size_t)id * (size_t)st.elems : nullptr;
+    for (; r < r_end; ++r) {
+      const int c = r * kThreads + tid;
+      const bool active = c < st.chunks;
+      if (active) {
+        if (m) st_stream(m + (size_t)c * kChunk, ld_stream(act + (size_t)c * kChunk));
+        if ((lane & (st.lanes_per_group - 1)) == 0) scales[c >> st.lg_shift] = 0.0f;
       }
-    } else {
-      // first visit: the activation itself becomes m(xi); skipped sample: nothing is stored.
-      // Either way the sample's codes and scales are zero.
-      const int n = cur.take(st.rows);
-#pragma unroll
-      for (int i = 0; i < kRowsPerIter; ++i) {
-        if (i < n) {
-          const int c = c0 + i * kThreads;
-          const bool active = c < st.chunks;
-          if (active) {
-            if (m) st_stream(m + (size_t)c * kChunk, ld_stream(act + (size_t)c * kChunk));
-            if ((lane & (st.lanes_per_group - 1)) == 0) scales[c >> st.lg_shift] = 0.0f;
-          }
-          const bool warp_words = words_ok && (c - lane + 32 <= st.chunks);
-          store_codes<BITS>(stream, c, lane, active, warp_words, 0ull);
-        }
-      }
-      cur.advance(n, st.rows);
+      const bool warp_words = words_ok && (c - lane + 32 <= st.chunks);
+      store_codes<BITS>(stream, c, lane, active, warp_words, 0ull);
     }
   }
 }
@@ -568,65 +526,47 @@ __device__ __forceinline__ void decode_rows(const State& st, const uint8_t* __re
 }
 
 template <typename T, int BITS>
-__global__ void __launch_bounds__(kThreads, decode_ctas_per_sm<BITS>()) decode_kernel(const State st, const DecodeArgs a, const int rows_per_cta) {
+__global__ void __launch_bounds__(kThreads, decode_ctas_per_sm<BITS>()) decode_kernel(const State st, const DecodeArgs a, const LaunchPlan plan) {
   const int tid = threadIdx.x;
   const int lane = tid & 31;
-  RowCursor cur(rows_per_cta, a.n_batch * st.rows, st.rows);
-  SampleProbe probe = probe_sample(st, a.ids, cur.y, lane);       // every CTA has at least one row
-  const unsigned long long call = begin_call(st);
-  const bool words_ok = (st.packed_bytes & 3) == 0;
-  const int whole_rows = st.chunks / kThreads;
+  const int y = blockIdx.y;                                       // sample of the call
+  const SampleProbe probe = probe_sample(st, a.ids, y, lane);
+  const unsigned long long call = begin_call(st, plan);
+  long long id;
+  unsigned why;
+  const int mode = settle_sample(probe, true, a.raw != nullptr, call, id, why);
+  if (blockIdx.x == 0 && tid == 0) publish_sample(st, y, mode, id, why, call, a.first_flags);
 
-  int cur_y = -1, mode = kModeSkip;
-  T* out = nullptr;
-  T* m = nullptr;
-  const T* raw = nullptr;
-  const uint8_t* stream = nullptr;
-  const float* scales = nullptr;
+  T* out = reinterpret_cast<T*>(a.out) + (size_t)y * (size_t)st.elems;
+  int r = blockIdx.x * plan.rows_per_cta;                         // this CTA's rows of the sample: [r, r_end)
+  const int r_end = min(st.rows, r + plan.rows_per_cta);
 
-  while (!cur.done()) {
-    if (cur.y != cur_y) {
-      if (cur_y >= 0) probe = probe_sample(st, a.ids, cur.y, lane);
-      cur_y = cur.y;
-      long long id;
-      unsigned why;
-      mode = settle_sample(probe, true, a.raw != nullptr, call, id, why);
-      if (cur.rin == 0 && tid == 0) publish_sample(st, cur_y, mode, id, why, call, a.first_flags);
-      out = reinterpret_cast<T*>(a.out) + (long long)cur_y * st.elems;
-      stream = a.packed + (long long)cur_y * st.packed_bytes;
-      scales = a.scales + (long long)cur_y * st.groups;
-      m = (mode == kModeSkip) ? nullptr : reinterpret_cast<T*>(st.m) + id * st.elems;
-      raw = (mode == kModeFirst) ? reinterpret_cast<const T*>(a.raw) + (long long)cur_y * st.elems : nullptr;
-    }
-    int c0 = cur.rin * kThreads + tid;
-
-    if (mode == kModeDelta) {
-      const int iters = min(cur.r_end - cur.r, whole_rows - cur.rin) / kRowsPerIter;
-      if (iters > 0) {
-        for (int k = 0; k < iters; ++k, c0 += kRowsPerIter * kThreads)
-          decode_rows<T, BITS, true>(st, stream, scales, m, out, c0, kRowsPerIter, lane, words_ok);
-        cur.advance(iters * kRowsPerIter, st.rows);
-      } else {
-        const int n = cur.take(st.rows);
-        decode_rows<T, BITS, false>(st, stream, scales, m, out, c0, n, lane, words_ok);
-        cur.advance(n, st.rows);
-      }
-    } else {
-      // first visit: the raw message becomes m(xi) and the activation; skipped sample: zeros out.
-      const int n = cur.take(st.rows);
-#pragma unroll
-      for (int i = 0; i < kRowsPerIter; ++i) {
-        const int c = c0 + i * kThreads;
-        if (i < n && c < st.chunks) {
-          uint4 v = make_uint4(0, 0, 0, 0);
-          if (raw) {
-            v = ld_stream(raw + (size_t)c * kChunk);
-            st_stream(m + (size_t)c * kChunk, v);
-          }
-          st_stream(out + (size_t)c * kChunk, v);
+  if (mode == kModeDelta) {
+    T* m = reinterpret_cast<T*>(st.m) + (size_t)id * (size_t)st.elems;
+    const uint8_t* stream = a.packed + (size_t)y * (size_t)st.packed_bytes;
+    const float* scales = a.scales + (size_t)y * (size_t)st.groups;
+    const bool words_ok = (st.packed_bytes & 3) == 0;
+    const int whole_end = min(r_end, st.chunks / kThreads);
+    for (; r + kRowsPerIter <= whole_end; r += kRowsPerIter)
+      decode_rows<T, BITS, true>(st, stream, scales, m, out, r * kThreads + tid, kRowsPerIter, lane, words_ok);
+    for (; r < r_end; r += kRowsPerIter)
+      decode_rows<T, BITS, false>(st, stream, scales, m, out, r * kThreads + tid, min(kRowsPerIter, r_end - r), lane,
+                                  words_ok);
+  } else {
+    // first visit: the raw message becomes m(xi) and the activation; skipped sample: zeros out.
+    const bool first = mode == kModeFirst;
+    T* m = first ? reinterpret_cast<T*>(st.m) + (size_t)id * (size_t)st.elems : nullptr;
+    const T* raw = first ? reinterpret_cast<const T*>(a.raw) + (size_t)y * (size_t)st.elems : nullptr;
+    for (; r < r_end; ++r) {
+      const int c = r * kThreads + tid;
+      if (c < st.chunks) {
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (first) {
+          v = ld_stream(raw + (size_t)c * kChunk);
+          st_stream(m + (size_t)c * kChunk, v);
         }
+        st_stream(out + (size_t)c * kChunk, v);
       }
-      cur.advance(n, st.rows);
     }
   }
 }
@@ -754,26 +694,35 @@ __global__ void __launch_bounds__(kThreads) checksum_kernel(const State st, unsi
 
 inline unsigned grid_x(long long chunks) { return (unsigned)((chunks + kChunksPerCta - 1) / kChunksPerCta); }
 
-// Several waves of short CTAs: the hardware hands out CTAs in order, so the CTAs in flight cover
-// one moving window of memory, and a finished CTA is replaced at once.  A CTA walks
-// kRowsPerCta rows when the call is large (its per-sample work is then paid once per 8192
-// elements), fewer when that would leave multiprocessors idle.
+// Several waves of short CTAs: the hardware hands out CTAs in order (x fastest, then the
+// sample y), so the CTAs in flight cover one moving window of memory, and a finished CTA is
+// replaced at once.  A CTA walks kRowsPerCta rows of one sample when the call is large (its
+// per-sample work is then paid once per 8192 elements), fewer when that would leave
+// multiprocessors idle.
 constexpr int kRowsPerCta = 4;
 
 template <typename K, typename Args>
 cudaError_t launch_rows(K kernel, const State& st, const Args& a, cudaStream_t s) {
+  if (a.n_batch <= 0) return cudaSuccess;
   const long long total = (long long)a.n_batch * st.rows;
-  if (total <= 0) return cudaSuccess;
-  if (total > 0x7fffffffll) return cudaErrorInvalidValue;
   long long per = st.rows_per_cta;
   if (per <= 0) {
     per = total / ((long long)st.sms * 12);
     per = per < kRowsPerIter ? kRowsPerIter : (per > kRowsPerCta ? kRowsPerCta : per);
   }
-  if (per > total) per = total;
-  if ((total + per - 1) / per > (long long)kCallQuantum) per = (total + kCallQuantum - 1) / kCallQuantum;
-  const unsigned grid = (unsigned)((total + per - 1) / per);
-  kernel<<<grid, kThreads, 0, s>>>(st, a, (int)per);
+  if (per > st.rows) per = st.rows;
+  long long gx = (st.rows + per - 1) / per;
+  if (gx * a.n_batch > (long long)kCallQuantum) {            // keep every CTA's share of the quantum >= 1
+    gx = (long long)kCallQuantum / a.n_batch;
+    per = (st.rows + gx - 1) / gx;
+    gx = (st.rows + per - 1) / per;
+  }
+  const unsigned long long ctas = (unsigned long long)gx * (unsigned long long)a.n_batch;
+  LaunchPlan plan;
+  plan.rows_per_cta = (int)per;
+  plan.share = (unsigned)(kCallQuantum / ctas);
+  plan.first_share = (unsigned)(kCallQuantum - (unsigned long long)plan.share * (ctas - 1ull));
+  kernel<<<dim3((unsigned)gx, (unsigned)a.n_batch), kThreads, 0, s>>>(st, a, plan);
   return cudaGetLastError();
 }
 
