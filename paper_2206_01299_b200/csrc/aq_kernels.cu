@@ -326,6 +326,15 @@ __device__ __forceinline__ unsigned long long begin_call(const State& st, const 
   return s_call;
 }
 
+// Programmatic dependent launch: let the next kernel of the stream place its CTAs on the
+// multiprocessors while this grid is draining, and do not read anything before the previous
+// kernel of the stream has completed and its writes are visible.  (Both are hardware-managed
+// and no-ops for neighbours launched the ordinary way.)
+__device__ __forceinline__ void overlap_with_neighbours() {
+  asm volatile("griddepcontrol.launch_dependents;");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // What a warp reads from memory about sample y of the call.  The loads are issued here and
 // first used in settle_sample, so they can be in flight across the start-of-call barrier.
 struct SampleProbe {
@@ -443,6 +452,7 @@ __global__ void __launch_bounds__(kThreads, encode_ctas_per_sm<T, BITS>())
   const int tid = threadIdx.x;
   const int lane = tid & 31;
   const int y = blockIdx.y;                                       // sample of the call
+  overlap_with_neighbours();
   const SampleProbe probe = probe_sample(st, a.ids, y, lane);
   const unsigned long long call = begin_call(st, plan);
   long long id;
@@ -530,6 +540,7 @@ __global__ void __launch_bounds__(kThreads, decode_ctas_per_sm<BITS>()) decode_k
   const int tid = threadIdx.x;
   const int lane = tid & 31;
   const int y = blockIdx.y;                                       // sample of the call
+  overlap_with_neighbours();
   const SampleProbe probe = probe_sample(st, a.ids, y, lane);
   const unsigned long long call = begin_call(st, plan);
   long long id;
@@ -722,8 +733,16 @@ cudaError_t launch_rows(K kernel, const State& st, const Args& a, cudaStream_t s
   plan.rows_per_cta = (int)per;
   plan.share = (unsigned)(kCallQuantum / ctas);
   plan.first_share = (unsigned)(kCallQuantum - (unsigned long long)plan.share * (ctas - 1ull));
-  kernel<<<dim3((unsigned)gx, (unsigned)a.n_batch), kThreads, 0, s>>>(st, a, plan);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)gx, (unsigned)a.n_batch);
+  cfg.blockDim = dim3(kThreads);
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // see overlap_with_neighbours
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, st, a, plan);
 }
 
 }  // namespace
