@@ -591,6 +591,7 @@ __global__ void __launch_bounds__(kThreads) quant_grad_kernel(const T* __restric
   const int lane = threadIdx.x & 31;
   const int lg_shift = __ffs(lanes_per_group) - 1;
   const long long c0 = (long long)blockIdx.x * kChunksPerCta + threadIdx.x;
+  overlap_with_neighbours();
   uint4 gv[kChunksPerThread];
 #pragma unroll
   for (int i = 0; i < kChunksPerThread; ++i) {
@@ -619,6 +620,7 @@ __global__ void __launch_bounds__(kThreads) dequant_grad_kernel(const uint8_t* _
   const int lane = threadIdx.x & 31;
   const int lg_shift = __ffs(lanes_per_group) - 1;
   const long long c0 = (long long)blockIdx.x * kChunksPerCta + threadIdx.x;
+  overlap_with_neighbours();
   unsigned long long codes[kChunksPerThread];
   float delta[kChunksPerThread];
 #pragma unroll
@@ -705,6 +707,21 @@ __global__ void __launch_bounds__(kThreads) checksum_kernel(const State st, unsi
 
 inline unsigned grid_x(long long chunks) { return (unsigned)((chunks + kChunksPerCta - 1) / kChunksPerCta); }
 
+// Launch with programmatic stream serialisation (see overlap_with_neighbours).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, cudaStream_t s, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(kThreads);
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // Several waves of short CTAs: the hardware hands out CTAs in order (x fastest, then the
 // sample y), so the CTAs in flight cover one moving window of memory, and a finished CTA is
 // replaced at once.  A CTA walks kRowsPerCta rows of one sample when the call is large (its
@@ -733,16 +750,7 @@ cudaError_t launch_rows(K kernel, const State& st, const Args& a, cudaStream_t s
   plan.rows_per_cta = (int)per;
   plan.share = (unsigned)(kCallQuantum / ctas);
   plan.first_share = (unsigned)(kCallQuantum - (unsigned long long)plan.share * (ctas - 1ull));
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)gx, (unsigned)a.n_batch);
-  cfg.blockDim = dim3(kThreads);
-  cfg.stream = s;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // see overlap_with_neighbours
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kernel, st, a, plan);
+  return launch_overlapped(kernel, dim3((unsigned)gx, (unsigned)a.n_batch), s, st, a, plan);
 }
 
 }  // namespace
@@ -774,7 +782,7 @@ cudaError_t launch_quant_grad(int dtype, int bits, int lanes_per_group, const vo
   const long long chunks = n_elems / kChunk;
   const unsigned grid = grid_x(chunks);
 #define AQ_CALL_LPG(L) \
-  quant_grad_kernel<T_, B_, L><<<grid, kThreads, 0, s>>>(reinterpret_cast<const T_*>(grad), chunks, lanes_per_group, packed, scales)
+  return launch_overlapped(quant_grad_kernel<T_, B_, L>, dim3(grid), s, reinterpret_cast<const T_*>(grad), chunks, lanes_per_group, packed, scales)
 #define AQ_CALL(T, B)                                      \
   {                                                        \
     using T_ = T;                                          \
@@ -793,7 +801,7 @@ cudaError_t launch_dequant_grad(int dtype, int bits, int lanes_per_group, const 
   const long long chunks = n_elems / kChunk;
   const unsigned grid = grid_x(chunks);
 #define AQ_CALL(T, B) \
-  dequant_grad_kernel<T, B><<<grid, kThreads, 0, s>>>(packed, scales, chunks, lanes_per_group, reinterpret_cast<T*>(out))
+  return launch_overlapped(dequant_grad_kernel<T, B>, dim3(grid), s, packed, scales, chunks, lanes_per_group, reinterpret_cast<T*>(out))
   AQ_DISPATCH(dtype, bits, AQ_CALL)
 #undef AQ_CALL
   return cudaGetLastError();
