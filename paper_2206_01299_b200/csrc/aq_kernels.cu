@@ -11,8 +11,8 @@
 //
 // encode / decode run as several waves of short CTAs on a (rows, samples) grid; each CTA walks
 // a few "rows" (256 consecutive chunks) of one sample, so the per-sample work (id lookup,
-// first-visit test) is done once per CTA, by every warp for itself: the kernels have one
-// block barrier, at their start, and no wait on another CTA.
+// first-visit test) is done once per CTA, by its first warp: the kernels have one block
+// barrier, at their start, and no wait on another CTA.
 //
 // Arithmetic: one IEEE binary32 rounding per operation (explicit _rn / _rd intrinsics;
 // the one explicit fused multiply-add is exact-equivalent, see quantize8), so the result
@@ -307,23 +307,17 @@ __device__ __forceinline__ void st_stream(void* p, const uint4& v) { __stcs(rein
 
 // ------------------------------------------------------------------ calls and samples (Algorithm 1, "if xi not seen before")
 
-// Number of the running call, the same in every thread of the grid, different for every launch
-// on the handle.  The handle keeps one 64-bit arrival counter that only grows.  Each CTA adds
-// its share of kCallQuantum to it, the shares of one grid adding up to exactly kCallQuantum
-// (the first CTA takes the remainder; the launch layer works the shares out), so the counter is
-// a multiple of kCallQuantum between launches and every value a CTA gets back from its add lies
+// Number of the running call, the same in every CTA of the grid, different for every launch on
+// the handle.  The handle keeps one 64-bit arrival counter that only grows.  Each CTA adds its
+// share of kCallQuantum to it, the shares of one grid adding up to exactly kCallQuantum (the
+// first CTA takes the remainder; the launch layer works the shares out), so the counter is a
+// multiple of kCallQuantum between launches and every value a CTA gets back from its add lies
 // in [c * kCallQuantum, (c+1) * kCallQuantum) for the same c: the number of launches before
 // this one.  No CTA has to be the last one, nothing is reset, and a replayed CUDA graph counts
-// like any other launch.  One atomic per CTA, issued by thread 0 while the other warps are
-// already fetching their sample's id; one barrier hands the result to the CTA.
-__device__ __forceinline__ unsigned long long begin_call(const State& st, const LaunchPlan& plan) {
-  __shared__ unsigned long long s_call;
-  if (threadIdx.x == 0) {
-    const unsigned mine = (blockIdx.x | blockIdx.y) == 0 ? plan.first_share : plan.share;
-    s_call = atomicAdd(st.arrivals, (unsigned long long)mine) / kCallQuantum + kFirstCall;
-  }
-  __syncthreads();
-  return s_call;
+// like any other launch.
+__device__ __forceinline__ unsigned long long take_call_number(const State& st, const LaunchPlan& plan) {
+  const unsigned mine = (blockIdx.x | blockIdx.y) == 0 ? plan.first_share : plan.share;
+  return atomicAdd(st.arrivals, (unsigned long long)mine) / kCallQuantum + kFirstCall;
 }
 
 // Programmatic dependent launch: let the next kernel of the stream place its CTAs on the
@@ -335,54 +329,59 @@ __device__ __forceinline__ void overlap_with_neighbours() {
   asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
-// What a warp reads from memory about sample y of the call.  The loads are issued here and
-// first used in settle_sample, so they can be in flight across the start-of-call barrier.
-struct SampleProbe {
+// What a CTA knows about its sample after open_sample.
+struct Sample {
+  int mode;
   int32_t id;
-  int dup;                       // this lane saw the id earlier in the call
-  bool in_range;
-  unsigned long long stamp;
 };
 
-__device__ __forceinline__ SampleProbe probe_sample(const State& st, const int32_t* __restrict__ ids, int y,
-                                                    int lane) {
-  SampleProbe p;
-  p.id = ids[y];
-  p.in_range = p.id >= 0 && (long long)p.id < st.n_samples;
-  p.dup = 0;
-  for (int q = lane; q < y; q += 32) p.dup |= (ids[q] == p.id);
-  p.stamp = p.in_range ? __ldcg(st.seen + p.id) : 0ull;
-  return p;
-}
-
-// Mode of the probed sample, computed by one warp for itself (all 32 lanes call this together).
-// `why` gets the status bit of a skipped sample.
-__device__ __forceinline__ int settle_sample(const SampleProbe& p, bool need_raw, bool have_raw,
-                                             unsigned long long call, long long& id, unsigned& why) {
-  id = p.id;
-  why = 0u;
-  if (!p.in_range) {
-    why = kStBadId;
-    return kModeSkip;
+// Sample y of the call, resolved by warp 0 for the whole CTA (one barrier): its id, whether it
+// is in range, whether the id appeared earlier in the call (each lane checks a stride of the
+// earlier ids), its "seen" stamp and the call number -- four independent memory operations in
+// flight together, the stamp one step behind the id.  Lane 0 of the CTA that owns the sample's
+// first row also records the visit: status bit of a skipped sample, first-visit flag, stamp.
+__device__ __forceinline__ Sample open_sample(const State& st, const LaunchPlan& plan,
+                                              const int32_t* __restrict__ ids, int y, bool need_raw,
+                                              bool have_raw, uint8_t* first_flags) {
+  __shared__ Sample s_sample;
+  if (threadIdx.x < 32) {
+    const int lane = threadIdx.x;
+    unsigned long long call = 0ull;
+    if (lane == 0) call = take_call_number(st, plan);
+    const int32_t id = ids[y];
+    const bool in_range = id >= 0 && (long long)id < st.n_samples;
+    int dup = 0;
+    for (int q = lane; q < y; q += 32) dup |= (ids[q] == id);
+    const unsigned long long stamp = (lane == 0 && in_range) ? __ldcg(st.seen + id) : 0ull;
+    dup = __any_sync(kFullMask, dup);
+    if (lane == 0) {
+      int mode;
+      unsigned why = 0u;
+      if (!in_range) {
+        mode = kModeSkip;
+        why = kStBadId;
+      } else if (dup) {
+        mode = kModeSkip;
+        why = kStDupId;
+      } else if (stamp != 0ull && stamp != call) {
+        mode = kModeDelta;
+      } else if (need_raw && !have_raw) {
+        mode = kModeSkip;
+        why = kStNoRaw;
+      } else {
+        mode = kModeFirst;
+      }
+      s_sample.mode = mode;
+      s_sample.id = id;
+      if (blockIdx.x == 0) {                     // once per sample and call
+        if (why) atomicOr(st.status, why);
+        if (first_flags) first_flags[y] = (uint8_t)(mode == kModeFirst);
+        if (mode == kModeFirst) st.seen[id] = call;
+      }
+    }
   }
-  if (__any_sync(kFullMask, p.dup)) {
-    why = kStDupId;
-    return kModeSkip;
-  }
-  if (p.stamp != 0ull && p.stamp != call) return kModeDelta;
-  if (need_raw && !have_raw) {
-    why = kStNoRaw;
-    return kModeSkip;
-  }
-  return kModeFirst;
-}
-
-// Done once per sample and call, by the thread that owns the sample's first chunk.
-__device__ __forceinline__ void publish_sample(const State& st, int y, int mode, long long id, unsigned why,
-                                               unsigned long long call, uint8_t* first_flags) {
-  if (why) atomicOr(st.status, why);
-  if (first_flags) first_flags[y] = (uint8_t)(mode == kModeFirst);
-  if (mode == kModeFirst) st.seen[id] = call;
+  __syncthreads();
+  return s_sample;
 }
 
 // ------------------------------------------------------------------ encode (sender)
@@ -453,22 +452,19 @@ __global__ void __launch_bounds__(kThreads, encode_ctas_per_sm<T, BITS>())
   const int lane = tid & 31;
   const int y = blockIdx.y;                                       // sample of the call
   overlap_with_neighbours();
-  const SampleProbe probe = probe_sample(st, a.ids, y, lane);
-  const unsigned long long call = begin_call(st, plan);
-  long long id;
-  unsigned why;
-  const int mode = settle_sample(probe, false, false, call, id, why);
-  if (blockIdx.x == 0 && tid == 0) publish_sample(st, y, mode, id, why, call, a.first_flags);
-
-  const T* act = reinterpret_cast<const T*>(a.act) + (size_t)y * (size_t)st.elems;
-  uint8_t* stream = a.packed + (size_t)y * (size_t)st.packed_bytes;
-  float* scales = a.scales + (size_t)y * (size_t)st.groups;
+  const Sample sample = open_sample(st, plan, a.ids, y, false, false, a.first_flags);
+  const int mode = sample.mode;
+  // sizes per sample fit 32 bits (checked at create): 32 x 32 -> 64-bit products
+  const unsigned elems = (unsigned)st.elems;
+  const T* act = reinterpret_cast<const T*>(a.act) + (unsigned long long)(unsigned)y * elems;
+  uint8_t* stream = a.packed + (unsigned long long)(unsigned)y * (unsigned)st.packed_bytes;
+  float* scales = a.scales + (unsigned long long)(unsigned)y * (unsigned)st.groups;
   const bool words_ok = (st.packed_bytes & 3) == 0;
   int r = blockIdx.x * plan.rows_per_cta;                         // this CTA's rows of the sample: [r, r_end)
   const int r_end = min(st.rows, r + plan.rows_per_cta);
 
   if (mode == kModeDelta) {
-    T* m = reinterpret_cast<T*>(st.m) + (size_t)id * (size_t)st.elems;
+    T* m = reinterpret_cast<T*>(st.m) + (unsigned long long)(unsigned)sample.id * elems;
     // whole iterations first (rows without a ragged end: no bounds to check), then the rest
     const int whole_end = min(r_end, st.chunks / kThreads);
     for (; r + kRowsPerIter <= whole_end; r += kRowsPerIter)
@@ -479,7 +475,7 @@ __global__ void __launch_bounds__(kThreads, encode_ctas_per_sm<T, BITS>())
   } else {
     // first visit: the activation itself becomes m(xi); skipped sample: nothing is stored.
     // Either way the sample's codes and scales are zero.
-    T* m = (mode == kModeFirst) ? reinterpret_cast<T*>(st.m) + (size_t)id * (size_t)st.elems : nullptr;
+    T* m = (mode == kModeFirst) ? reinterpret_cast<T*>(st.m) + (unsigned long long)(unsigned)sample.id * elems : nullptr;
     for (; r < r_end; ++r) {
       const int c = r * kThreads + tid;
       const bool active = c < st.chunks;
@@ -541,21 +537,17 @@ __global__ void __launch_bounds__(kThreads, decode_ctas_per_sm<BITS>()) decode_k
   const int lane = tid & 31;
   const int y = blockIdx.y;                                       // sample of the call
   overlap_with_neighbours();
-  const SampleProbe probe = probe_sample(st, a.ids, y, lane);
-  const unsigned long long call = begin_call(st, plan);
-  long long id;
-  unsigned why;
-  const int mode = settle_sample(probe, true, a.raw != nullptr, call, id, why);
-  if (blockIdx.x == 0 && tid == 0) publish_sample(st, y, mode, id, why, call, a.first_flags);
-
-  T* out = reinterpret_cast<T*>(a.out) + (size_t)y * (size_t)st.elems;
+  const Sample sample = open_sample(st, plan, a.ids, y, true, a.raw != nullptr, a.first_flags);
+  const int mode = sample.mode;
+  const unsigned elems = (unsigned)st.elems;
+  T* out = reinterpret_cast<T*>(a.out) + (unsigned long long)(unsigned)y * elems;
   int r = blockIdx.x * plan.rows_per_cta;                         // this CTA's rows of the sample: [r, r_end)
   const int r_end = min(st.rows, r + plan.rows_per_cta);
 
   if (mode == kModeDelta) {
-    T* m = reinterpret_cast<T*>(st.m) + (size_t)id * (size_t)st.elems;
-    const uint8_t* stream = a.packed + (size_t)y * (size_t)st.packed_bytes;
-    const float* scales = a.scales + (size_t)y * (size_t)st.groups;
+    T* m = reinterpret_cast<T*>(st.m) + (unsigned long long)(unsigned)sample.id * elems;
+    const uint8_t* stream = a.packed + (unsigned long long)(unsigned)y * (unsigned)st.packed_bytes;
+    const float* scales = a.scales + (unsigned long long)(unsigned)y * (unsigned)st.groups;
     const bool words_ok = (st.packed_bytes & 3) == 0;
     const int whole_end = min(r_end, st.chunks / kThreads);
     for (; r + kRowsPerIter <= whole_end; r += kRowsPerIter)
@@ -566,8 +558,8 @@ __global__ void __launch_bounds__(kThreads, decode_ctas_per_sm<BITS>()) decode_k
   } else {
     // first visit: the raw message becomes m(xi) and the activation; skipped sample: zeros out.
     const bool first = mode == kModeFirst;
-    T* m = first ? reinterpret_cast<T*>(st.m) + (size_t)id * (size_t)st.elems : nullptr;
-    const T* raw = first ? reinterpret_cast<const T*>(a.raw) + (size_t)y * (size_t)st.elems : nullptr;
+    T* m = first ? reinterpret_cast<T*>(st.m) + (unsigned long long)(unsigned)sample.id * elems : nullptr;
+    const T* raw = first ? reinterpret_cast<const T*>(a.raw) + (unsigned long long)(unsigned)y * elems : nullptr;
     for (; r < r_end; ++r) {
       const int c = r * kThreads + tid;
       if (c < st.chunks) {
