@@ -34,9 +34,11 @@ WORKLOADS = {"gpt2": ("GPT2_XL", 32, "GPT2-1.5B-shaped boundary (configs[1])"),
              "deberta": ("DEBERTA_XXL", 64, "DeBERTa-1.5B-shaped boundary (configs[2])")}
 FALLBACK_HBM_GBS = 6650.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the named kernel, from the ncu
-# capture summarised in profiles/ (scaled to this launch's units); None until captured.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = {"encode": None, "decode": None}
+# dram__bytes_read.sum + dram__bytes_write.sum of one delta-visit launch of 32 GPT2-shaped sequences
+# (52,428,800 elements), from the ncu capture summarised in profiles/encode_decode_gpt2_boundary_ncu.md;
+# scaled by the elements of a launch.  Set to None when the kernels change after the capture.
+NCU_TRAFFIC_BYTES_PER_ELEMENT = {"encode": 288901632 / 52428800, "decode": 287772928 / 52428800}
+NCU_TRAFFIC_WORKLOAD = "gpt2"
 
 
 def parse_args():
@@ -427,7 +429,7 @@ def main():
     launch_bytes = nb * cfg.elems * bpe
     enc_gbs = launch_bytes / (enc_ms * 1e-3) / 1e9
     dec_gbs = launch_bytes / (dec_ms * 1e-3) / 1e9
-    traffic = NCU_TRAFFIC_BYTES_PER_ELEMENT["encode"]
+    traffic = NCU_TRAFFIC_BYTES_PER_ELEMENT["encode"] if args.workload == NCU_TRAFFIC_WORKLOAD else None
     value = replicas.whole_job_rate(args.steps * step_bytes, world, elapsed_ms) / 1e9
     line = {
         "metric": "activation encode+decode GB/s", "value": value, "unit": "GB/s",
