@@ -57,6 +57,17 @@ def lib():
         L.aqo_quant_grad.argtypes = [u16p, C.c_int64, C.c_int, C.c_int, C.c_int, u8p, f32p]
         L.aqo_dequant_grad.restype = None
         L.aqo_dequant_grad.argtypes = [u8p, f32p, C.c_int64, C.c_int, C.c_int, C.c_int, u16p]
+        u32p = C.POINTER(C.c_uint32)
+        L.aqo_philox4x32_10.restype = None
+        L.aqo_philox4x32_10.argtypes = [u32p, u32p, u32p]
+        L.aqo_quantize_group_stochastic.restype = None
+        L.aqo_quantize_group_stochastic.argtypes = [f32p, C.c_int, C.c_int, C.c_uint64, C.c_uint64, C.c_uint32,
+                                                    C.c_int64, i32p, f32p]
+        L.aqo_set_rounding.restype = None
+        L.aqo_set_rounding.argtypes = [C.c_void_p, C.c_int, C.c_uint64, C.c_uint64]
+        L.aqo_quant_grad_stochastic.restype = None
+        L.aqo_quant_grad_stochastic.argtypes = [u16p, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_uint64, C.c_uint64,
+                                                u8p, f32p]
         L.aqo_state_checksum.restype = C.c_uint64
         L.aqo_state_checksum.argtypes = [C.c_void_p]
         _lib = L
@@ -100,6 +111,25 @@ def quantize_group(d, bits):
     delta = C.c_float(0)
     lib().aqo_quantize_group(_p(d, C.c_float), d.shape[0], bits, _p(k, C.c_int32),
                              C.byref(delta))
+    return k, np.float32(delta.value)
+
+
+def philox4x32_10(counter, key):
+    """counter: 4 uint32, key: 2 uint32 -> 4 uint32 (Philox4x32, 10 rounds)."""
+    c = np.array(counter, np.uint32)
+    k = np.array(key, np.uint32)
+    out = np.zeros(4, np.uint32)
+    lib().aqo_philox4x32_10(_p(c, C.c_uint32), _p(k, C.c_uint32), _p(out, C.c_uint32))
+    return out
+
+
+def quantize_group_stochastic(d, bits, seed, epoch, stream_id, first_elem=0):
+    """d: float32[G] (G a multiple of 8) -> (k int32[G], Delta float), unbiased stochastic Q."""
+    d = _c(d, np.float32)
+    k = np.zeros(d.shape[0], np.int32)
+    delta = C.c_float(0)
+    lib().aqo_quantize_group_stochastic(_p(d, C.c_float), d.shape[0], bits, seed, epoch, stream_id, first_elem,
+                                        _p(k, C.c_int32), C.byref(delta))
     return k, np.float32(delta.value)
 
 
@@ -154,6 +184,9 @@ class Side:
     def status(self):
         return lib().aqo_status(self.h)
 
+    def set_rounding(self, stochastic, seed=0, epoch=0):
+        lib().aqo_set_rounding(self.h, int(bool(stochastic)), seed, epoch)
+
     def encode(self, act, ids):
         """act uint16[n_batch, seq, hidden], ids int32[n_batch] ->
         (packed uint8[n_batch, pbytes], scales float32[n_batch, ngroups], first uint8[n_batch])"""
@@ -195,6 +228,17 @@ def quant_grad(grad, bits, group, dtype=FP16):
     scales = np.empty(n // group, np.float32)
     lib().aqo_quant_grad(_p(grad, C.c_uint16), n, bits, group, dtype,
                          _p(packed, C.c_uint8), _p(scales, C.c_float))
+    return packed, scales
+
+
+def quant_grad_stochastic(grad, bits, group, seed, epoch, dtype=FP16):
+    grad = _c(grad, np.uint16).reshape(-1)
+    n = grad.shape[0]
+    assert n % group == 0 and (n * bits) % 8 == 0
+    packed = np.empty(n * bits // 8, np.uint8)
+    scales = np.empty(n // group, np.float32)
+    lib().aqo_quant_grad_stochastic(_p(grad, C.c_uint16), n, bits, group, dtype, seed, epoch,
+                                    _p(packed, C.c_uint8), _p(scales, C.c_float))
     return packed, scales
 
 

@@ -18,7 +18,9 @@
 // hand-derived code vectors, exact-rational brute force of the interval index,
 // the error bound Delta/2, sender/receiver buffer identity, first-visit
 // identity, zero-delta fixed point, step-change decay, bitstream length, and
-// published splitmix64 vectors for the checksum mixer.
+// published splitmix64 vectors for the checksum mixer; for the stochastic
+// quantizer: Philox4x32-10 known-answer vectors, exact-rational brute force,
+// E[Q(d)] = d, level structure.
 //
 // Parity with the paper authors' own implementation is UNPINNED: the paper
 // prints no codes, scales or bit layout; mid-rise reconstruction, the fp32
@@ -155,6 +157,97 @@ inline float reconstruct(int32_t k, float delta) {
 }
 
 // ---------------------------------------------------------------------------
+// Unbiased variant of Q (the quantizer that Theorem 3.1 assumes; its footnote
+// sketches it as "rounding to the closest k/2^b, stochastically").  Reading
+// fixed here: the 2^b levels are spread evenly over the whole of [-s, s],
+//
+//   Delta = s / (2^(b-1) - 1/2),   level_k = (k + 1/2) * Delta,  k in [-2^(b-1), 2^(b-1)-1]
+//   (level_min = -s, level_max = +s),
+//
+// and d is rounded to one of its two neighbouring levels with probabilities
+// proportional to the distance from the other one:
+//
+//   k = floor(d / Delta - 1/2 + r),  r uniform in [0,1)    =>  E[level_k] = d  for every |d| <= s.
+//
+// In fp32, with the random number folded into one addition:
+//   delta = s / (2^(b-1) - 0.5f);  inv = 1.0f / delta;
+//   t = d * inv + rc,  rc = (h - 32767.5) * 2^-16  for a 16-bit random integer h  (rc = r - 1/2, exact);
+//   k = clamp(floor(t)).
+// The receiver needs nothing new: it reconstructs (k + 1/2) * Delta from the
+// transmitted Delta exactly as before.
+//
+// Random numbers: Philox4x32-10 (Salmon, Moraes, Dror, Shaw, "Parallel random
+// numbers: as easy as 1, 2, 3", SC 2011), a counter-based generator, so that
+// any element of any call can be regenerated alone.  One 128-bit output serves
+// the 8 elements of a chunk, 16 bits each:
+//   key     = { seed low word, seed high word }
+//   counter = { chunk index inside the stream, stream id, epoch low word, epoch high word }
+//   element j of the chunk uses bits [16*(j%2), 16*(j%2)+16) of output word j/2.
+// The stream id is the sample id for activations and 0xFFFFFFFF for gradients.
+// ---------------------------------------------------------------------------
+
+void philox4x32_10(const uint32_t counter[4], const uint32_t key[2], uint32_t out[4]) {
+  const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;      // round multipliers
+  const uint32_t W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;      // key schedule (Weyl) increments
+  uint32_t c0 = counter[0], c1 = counter[1], c2 = counter[2], c3 = counter[3];
+  uint32_t k0 = key[0], k1 = key[1];
+  for (int round = 0; round < 10; ++round) {
+    const uint64_t p0 = (uint64_t)M0 * c0;
+    const uint64_t p1 = (uint64_t)M1 * c2;
+    const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+    const uint32_t n1 = (uint32_t)p1;
+    const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+    const uint32_t n3 = (uint32_t)p0;
+    c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    k0 += W0; k1 += W1;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// centred random offsets rc = r - 1/2 of the 8 elements of one chunk
+void chunk_offsets(uint64_t seed, uint64_t epoch, uint32_t stream_id, uint32_t chunk, float rc[8]) {
+  const uint32_t counter[4] = {chunk, stream_id, (uint32_t)epoch, (uint32_t)(epoch >> 32)};
+  const uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+  uint32_t w[4];
+  philox4x32_10(counter, key, w);
+  for (int j = 0; j < 8; ++j) {
+    const uint32_t h = (w[j / 2] >> (16 * (j % 2))) & 0xFFFFu;
+    rc[j] = ((float)h - 32767.5f) * 1.52587890625e-05f;   // 2^-16; both steps exact
+  }
+}
+
+// d[0..G) are elements first_elem .. first_elem+G of the stream (first_elem is a multiple of 8)
+void quantize_group_stochastic(const float* d, int G, int bits, uint64_t seed, uint64_t epoch,
+                               uint32_t stream_id, int64_t first_elem, int32_t* k, float* delta_out) {
+  float s = 0.0f;
+  for (int j = 0; j < G; ++j) {
+    const float a = std::fabs(d[j]);
+    if (a > s) s = a;
+  }
+  const float top = (float)(1 << (bits - 1)) - 0.5f;        // level index of +s, plus 1/2
+  const float delta = s / top;
+  if (!(delta >= FLT_MIN)) {
+    *delta_out = 0.0f;
+    for (int j = 0; j < G; ++j) k[j] = 0;
+    return;
+  }
+  const float inv = 1.0f / delta;
+  const float kmin = -(float)(1 << (bits - 1));
+  const float kmax = (float)((1 << (bits - 1)) - 1);
+  float rc[8];
+  for (int j = 0; j < G; ++j) {
+    if (j % 8 == 0) chunk_offsets(seed, epoch, stream_id, (uint32_t)((first_elem + j) / 8), rc);
+    const float u = d[j] * inv;
+    const float t = u + rc[j % 8];
+    float kf = std::floor(t);
+    if (kf < kmin) kf = kmin;
+    if (kf > kmax) kf = kmax;
+    k[j] = (int32_t)kf;
+  }
+  *delta_out = delta;
+}
+
+// ---------------------------------------------------------------------------
 // Bitstream: element j of a stream owns bits [j*b, (j+1)*b); bit t of the
 // stream is bit (t mod 8) of byte (t div 8).  The field is the low b bits of
 // the two's-complement code.
@@ -194,6 +287,8 @@ struct Side {
   std::vector<uint16_t> m;       // [n_samples][seq][hidden], activation dtype
   std::vector<uint8_t> seen;     // [n_samples]
   uint32_t status;               // sticky: 1 id out of range, 2 duplicate id in a call, 4 first visit at decode with no raw message
+  int rounding = 0;              // 0: interval number (deterministic), 1: stochastic, unbiased
+  uint64_t seed = 0, epoch = 0;  // stochastic rounding: generator key and the caller's call counter
 };
 
 enum { ST_BAD_ID = 1, ST_DUP_ID = 2, ST_NO_RAW = 4 };
@@ -230,6 +325,11 @@ uint64_t aqo_mix64(uint64_t index, uint64_t word) { return mix64(index, word); }
 void aqo_quantize_group(const float* d, int G, int bits, int32_t* k, float* delta) {
   quantize_group(d, G, bits, k, delta);
 }
+void aqo_philox4x32_10(const uint32_t* counter, const uint32_t* key, uint32_t* out) { philox4x32_10(counter, key, out); }
+void aqo_quantize_group_stochastic(const float* d, int G, int bits, uint64_t seed, uint64_t epoch, uint32_t stream_id,
+                                   int64_t first_elem, int32_t* k, float* delta) {
+  quantize_group_stochastic(d, G, bits, seed, epoch, stream_id, first_elem, k, delta);
+}
 float aqo_reconstruct(int32_t k, float delta) { return reconstruct(k, delta); }
 void aqo_put_code(uint8_t* stream, int64_t j, int bits, int32_t k) { put_code(stream, j, bits, k); }
 int32_t aqo_get_code(const uint8_t* stream, int64_t j, int bits) { return get_code(stream, j, bits); }
@@ -250,6 +350,12 @@ void* aqo_create(int64_t n_samples, int seq, int hidden, int bits, int group, in
 }
 
 void aqo_destroy(void* h) { delete (Side*)h; }
+
+// rounding: 0 = interval number (default), 1 = stochastic; seed and epoch only matter for 1
+void aqo_set_rounding(void* h, int rounding, uint64_t seed, uint64_t epoch) {
+  Side* S = (Side*)h;
+  S->rounding = rounding; S->seed = seed; S->epoch = epoch;
+}
 
 const uint16_t* aqo_m(void* h) { return ((Side*)h)->m.data(); }
 const uint8_t* aqo_seen(void* h) { return ((Side*)h)->seen.data(); }
@@ -292,7 +398,10 @@ void aqo_encode(void* h, const uint16_t* act, const int32_t* ids, int n_batch,
       for (int j = 0; j < S->group; ++j)
         d[j] = t_to_float(a[base + j], S->dtype) - t_to_float(M[base + j], S->dtype);
       float delta;
-      quantize_group(d.data(), S->group, S->bits, k.data(), &delta);
+      if (S->rounding == 1)
+        quantize_group_stochastic(d.data(), S->group, S->bits, S->seed, S->epoch, (uint32_t)ids[y], base, k.data(), &delta);
+      else
+        quantize_group(d.data(), S->group, S->bits, k.data(), &delta);
       SC[g] = delta;
       for (int j = 0; j < S->group; ++j) {
         put_code(P, base + j, S->bits, k[j]);
@@ -354,6 +463,23 @@ void aqo_quant_grad(const uint16_t* grad, int64_t n_elems, int bits, int group, 
     for (int j = 0; j < group; ++j) d[j] = t_to_float(grad[base + j], dtype);
     float delta;
     quantize_group(d.data(), group, bits, k.data(), &delta);
+    scales[g] = delta;
+    for (int j = 0; j < group; ++j) put_code(packed, base + j, bits, k[j]);
+  }
+}
+
+// The same with the unbiased stochastic Q (stream id 0xFFFFFFFF; the caller gives every call
+// its own epoch value).
+void aqo_quant_grad_stochastic(const uint16_t* grad, int64_t n_elems, int bits, int group, int dtype,
+                               uint64_t seed, uint64_t epoch, uint8_t* packed, float* scales) {
+  std::vector<float> d(group);
+  std::vector<int32_t> k(group);
+  std::memset(packed, 0, (size_t)(n_elems * bits / 8));
+  for (int64_t g = 0; g < n_elems / group; ++g) {
+    const int64_t base = g * group;
+    for (int j = 0; j < group; ++j) d[j] = t_to_float(grad[base + j], dtype);
+    float delta;
+    quantize_group_stochastic(d.data(), group, bits, seed, epoch, 0xFFFFFFFFu, base, k.data(), &delta);
     scales[g] = delta;
     for (int j = 0; j < group; ++j) put_code(packed, base + j, bits, k[j]);
   }
