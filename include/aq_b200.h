@@ -78,10 +78,30 @@ enum {
                             aq_decode stores for first-visit samples; 0 = none (default) */
   AQ_FIRST_FLAGS = 5,    /* device pointer uint8[n_batch] or 0: aq_encode / aq_decode write 1 for
                             each sample that took the first-visit path, else 0 */
+  AQ_ROUNDING = 7,       /* AQ_ROUND_INTERVAL (default) or AQ_ROUND_STOCHASTIC: how aq_encode and
+                            aq_quant_grad pick the code, see below */
+  AQ_SEED = 8,           /* 64-bit key of the random numbers of AQ_ROUND_STOCHASTIC (default 0) */
+  AQ_EPOCH = 9,          /* 64-bit counter that the caller sets before a call: two calls that should draw
+                            independent random numbers need different values (for activations the epoch
+                            or step number; for gradients any number unique to the call); default 0 */
   AQ_ROWS_PER_CTA = 6    /* tuning: rows (256 chunks = 2048 elements each) that one CTA of aq_encode /
                             aq_decode walks; 0 (default) = chosen from the size of the call (2..4) */
 };
 enum { AQ_FP16 = 0, AQ_BF16 = 1 };
+/*
+ * AQ_ROUND_INTERVAL: Q of Section 4.1 as described at the top of this file.
+ * AQ_ROUND_STOCHASTIC: the unbiased Q that Theorem 3.1 assumes (its footnote: rounding to the
+ * uniform grid "stochastically").  The 2^b levels reach from -s to +s,
+ *   Delta = s / (2^(b-1) - 1/2),  k = clamp(floor(d * (1/Delta) + (r - 1/2))),  r uniform in [0,1),
+ * so that E[(k + 1/2) * Delta] = d for every element of the group.  Receivers need no setting:
+ * aq_decode / aq_dequant_grad rebuild (k + 1/2) * Delta from the Delta they are sent.  r comes
+ * from Philox4x32-10 (Salmon et al., SC 2011), 16 bits per element: key = AQ_SEED, counter =
+ * { chunk (element index / 8) inside the sample or gradient, sample id (0xFFFFFFFF for
+ * gradients), AQ_EPOCH low word, AQ_EPOCH high word }; element j of a chunk takes bits
+ * [16*(j%2), 16*(j%2)+16) of output word j/2 and r - 1/2 = (bits - 32767.5) * 2^-16.  The
+ * result is a pure function of (seed, epoch, sample id, element, inputs).
+ */
+enum { AQ_ROUND_INTERVAL = 0, AQ_ROUND_STOCHASTIC = 1 };
 
 /* sticky bits of aq_status */
 enum {

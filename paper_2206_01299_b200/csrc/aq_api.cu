@@ -14,6 +14,8 @@ struct aq_handle {
   int seq = 0, hidden = 0, bits = 0, group = 0;
   int dtype = AQ_FP16;
   int n_batch = 1;
+  int rounding = AQ_ROUND_INTERVAL;
+  unsigned long long seed = 0, epoch = 0;
   int device = 0;
   cudaStream_t stream = nullptr;
   const void* raw = nullptr;
@@ -172,6 +174,17 @@ int aq_configure(aq_handle* h, int key, int64_t value) {
     case AQ_FIRST_FLAGS:
       h->first_flags = reinterpret_cast<uint8_t*>(static_cast<intptr_t>(value));
       return AQ_OK;
+    case AQ_ROUNDING:
+      if (value != AQ_ROUND_INTERVAL && value != AQ_ROUND_STOCHASTIC)
+        return fail(h, AQ_EINVAL, "AQ_ROUNDING must be AQ_ROUND_INTERVAL or AQ_ROUND_STOCHASTIC");
+      h->rounding = (int)value;
+      return AQ_OK;
+    case AQ_SEED:
+      h->seed = (unsigned long long)value;
+      return AQ_OK;
+    case AQ_EPOCH:
+      h->epoch = (unsigned long long)value;
+      return AQ_OK;
     case AQ_ROWS_PER_CTA:
       if (value < 0 || value > (1 << 20)) return fail(h, AQ_EINVAL, "AQ_ROWS_PER_CTA must be in 0..2^20");
       h->st.rows_per_cta = (int)value;
@@ -188,7 +201,8 @@ int aq_encode(aq_handle* h, const void* act, const int32_t* sample_ids, void* pa
   if (!aligned16(act) || !aligned16(packed) || !aligned16(scales))
     return fail(h, AQ_EINVAL, "aq_encode: act, packed and scales must be 16-byte aligned");
   DeviceGuard g(h->device);
-  aq::EncodeArgs a{act, sample_ids, static_cast<uint8_t*>(packed), scales, h->first_flags, h->n_batch};
+  aq::EncodeArgs a{act, sample_ids, static_cast<uint8_t*>(packed), scales, h->first_flags, h->n_batch,
+                   h->rounding == AQ_ROUND_STOCHASTIC, h->seed, h->epoch};
   AQ_CUDA(h, aq::launch_encode(h->dtype, h->bits, h->st, a, h->stream));
   return AQ_OK;
 }
@@ -219,8 +233,11 @@ int aq_quant_grad(aq_handle* h, const void* grad, int64_t n_elems, int bits, voi
   const int rc = check_grad_args(h, grad, packed, scales, n_elems, bits);
   if (rc != AQ_OK || n_elems == 0) return rc;
   DeviceGuard g(h->device);
+  const bool stochastic = h->rounding == AQ_ROUND_STOCHASTIC;
+  if (stochastic && n_elems / aq::kChunk > 0xFFFFFFFFll)
+    return fail(h, AQ_EINVAL, "aq_quant_grad: stochastic rounding numbers chunks with 32 bits (n_elems < 2^35)");
   AQ_CUDA(h, aq::launch_quant_grad(h->dtype, bits, h->st.lanes_per_group, grad, n_elems,
-                                   static_cast<uint8_t*>(packed), scales, h->stream));
+                                   static_cast<uint8_t*>(packed), scales, stochastic, h->seed, h->epoch, h->stream));
   return AQ_OK;
 }
 

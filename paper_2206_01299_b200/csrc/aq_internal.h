@@ -45,6 +45,8 @@ struct EncodeArgs {
   float* scales;
   uint8_t* first_flags;    // may be null
   int n_batch;
+  bool stochastic;                  // unbiased stochastic rounding instead of the interval number
+  unsigned long long seed, epoch;   // its generator key and the caller's call counter
 };
 
 struct DecodeArgs {
@@ -60,7 +62,8 @@ struct DecodeArgs {
 cudaError_t launch_encode(int dtype, int bits, const State& st, const EncodeArgs& a, cudaStream_t s);
 cudaError_t launch_decode(int dtype, int bits, const State& st, const DecodeArgs& a, cudaStream_t s);
 cudaError_t launch_quant_grad(int dtype, int bits, int lanes_per_group, const void* grad,
-                              long long n_elems, uint8_t* packed, float* scales, cudaStream_t s);
+                              long long n_elems, uint8_t* packed, float* scales, bool stochastic,
+                              unsigned long long seed, unsigned long long epoch, cudaStream_t s);
 cudaError_t launch_dequant_grad(int dtype, int bits, int lanes_per_group, const uint8_t* packed,
                                 const float* scales, long long n_elems, void* out, cudaStream_t s);
 // *sum_dev += digest of (m, seen); the caller zeroes *sum_dev first.

@@ -142,23 +142,36 @@ __device__ __forceinline__ uint32_t pack_fields(const uint32_t* tb) {
 //   reciprocal, |d * RN(1/delta)| < 2^(b-1) * (1 + 2^-24), which rounds to at most 2^(b-1).
 // * (k + 1/2) * delta, rounded once, is fma(k, delta, delta/2) whenever delta/2 is exact,
 //   i.e. delta >= 2^-125; the wide type falls back to add-then-multiply below that.
-template <typename T, int BITS>
-__device__ __forceinline__ void quantize8(const float (&d)[8], float s, float& delta,
+// STOCH (the unbiased quantizer that Theorem 3.1 assumes): delta = s / (2^(b-1) - 1/2), so that
+// the 2^b levels (k + 1/2) * delta reach from -s to +s, and k = floor(d / delta - 1/2 + r) with
+// r uniform in [0,1) from `noise`; both clamps are needed then.
+template <typename T, int BITS, bool STOCH>
+__device__ __forceinline__ void quantize8(const float (&d)[8], float s, const uint4& noise, float& delta,
                                           unsigned long long& codes, float (&q)[8]) {
   constexpr float kTwoPow = 1.0f / (float)(1 << (BITS - 1));
+  constexpr float kTop = (float)(1 << (BITS - 1)) - 0.5f;
   constexpr float kLo = -(float)(1 << (BITS - 1));
   constexpr float kHi = (float)(1 << (BITS - 1)) - 0.5f;
   constexpr float kMagic = 12582912.0f;                      // 1.5 * 2^23 = 0x4B400000
-  const float dl = __fmul_rn(s, kTwoPow);
+  const float dl = STOCH ? __fdiv_rn(s, kTop) : __fmul_rn(s, kTwoPow);
   const bool live = dl >= FLT_MIN;
   delta = live ? dl : 0.0f;
   const float inv = live ? __frcp_rn(dl) : 0.0f;             // IEEE 1/delta, one rounding
   const float half_delta = __fmul_rn(delta, 0.5f);
+  // stochastic rounding: r - 1/2 = (h - 32767.5) * 2^-16 for the element's 16 random bits h
+  // (a dead group gets no noise: its codes are 0).  2^22 + h + 1/2 is built in the mantissa.
+  const float noise_unit = live ? 1.52587890625e-05f : 0.0f;
+  const uint32_t nw[4] = {noise.x, noise.y, noise.z, noise.w};
   uint32_t tb[8];
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
     float u = __fmul_rn(d[j], inv);
-    if constexpr (Conv<T>::kWide) u = fmaxf(u, kLo);
+    if constexpr (STOCH) {
+      const uint32_t h = (j & 1) ? (nw[j >> 1] >> 16) : (nw[j >> 1] & 0xFFFFu);
+      const float hc = __fsub_rn(__uint_as_float(0x4A800001u | (h << 1)), 4227072.0f);   // h - 32767.5, exact
+      u = __fadd_rn(u, __fmul_rn(hc, noise_unit));
+    }
+    if constexpr (Conv<T>::kWide || STOCH) u = fmaxf(u, kLo);
     u = fminf(u, kHi);
     const float t = __fadd_rd(u, kMagic);
     tb[j] = __float_as_uint(t);
@@ -181,6 +194,28 @@ __device__ __forceinline__ void quantize8(const float (&d)[8], float s, float& d
     const uint32_t hi = pack_fields<BITS, 4>(tb + 4);
     codes = (unsigned long long)lo | ((unsigned long long)hi << (4 * BITS));
   }
+}
+
+// Philox4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw, SC 2011): the 128 random bits of one
+// chunk.  key = the seed's two words; counter = { chunk index in the stream, stream id (sample
+// id, or 0xFFFFFFFF for gradients), epoch low word, epoch high word }.  Element j of the chunk
+// uses bits [16*(j%2), 16*(j%2)+16) of word j/2.
+__device__ __forceinline__ uint4 chunk_noise(unsigned long long seed, unsigned long long epoch, uint32_t stream_id,
+                                             uint32_t chunk) {
+  uint32_t c0 = chunk, c1 = stream_id, c2 = (uint32_t)epoch, c3 = (uint32_t)(epoch >> 32);
+  uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
+#pragma unroll
+  for (int round = 0; round < 10; ++round) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    c0 = hi1 ^ c1 ^ k0;
+    c1 = lo1;
+    c2 = hi0 ^ c3 ^ k1;
+    c3 = lo0;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  return make_uint4(c0, c1, c2, c3);
 }
 
 // q = (k + 1/2) * delta from the b-bit fields.  The field, with its sign bit flipped, is
@@ -388,8 +423,9 @@ __device__ __forceinline__ Sample open_sample(const State& st, const LaunchPlan&
 
 // Delta visit of n rows starting at chunk c0 of one sample.  FULL: n == kRowsPerIter and every
 // chunk is inside the sample, so no bounds are checked.
-template <typename T, int BITS, int LPG, bool FULL>
-__device__ __forceinline__ void encode_rows(const State& st, const T* __restrict__ act, T* __restrict__ m,
+template <typename T, int BITS, int LPG, bool STOCH, bool FULL>
+__device__ __forceinline__ void encode_rows(const State& st, const EncodeArgs& a, uint32_t stream_id,
+                                            const T* __restrict__ act, T* __restrict__ m,
                                             uint8_t* __restrict__ stream, float* __restrict__ scales, int c0,
                                             int n, int lane, bool words_ok) {
   uint4 av[kRowsPerIter], mv[kRowsPerIter];
@@ -420,7 +456,9 @@ __device__ __forceinline__ void encode_rows(const State& st, const T* __restrict
       const float s = group_max<LPG>(abs_max8(d), st.lanes_per_group);
       float delta;
       unsigned long long codes;
-      quantize8<T, BITS>(d, s, delta, codes, q);
+      uint4 noise = make_uint4(0, 0, 0, 0);
+      if constexpr (STOCH) noise = chunk_noise(a.seed, a.epoch, stream_id, (uint32_t)c);
+      quantize8<T, BITS, STOCH>(d, s, noise, delta, codes, q);
 #pragma unroll
       for (int j = 0; j < 8; ++j) mf[j] = __fadd_rn(mf[j], q[j]);
       if (active) {
@@ -445,8 +483,8 @@ constexpr int decode_ctas_per_sm() {
   return (BITS == 1 || BITS == 2 || BITS == 4 || BITS == 8) ? 6 : (BITS == 3 ? 5 : 4);
 }
 
-template <typename T, int BITS, int LPG>
-__global__ void __launch_bounds__(kThreads, encode_ctas_per_sm<T, BITS>())
+template <typename T, int BITS, int LPG, bool STOCH>
+__global__ void __launch_bounds__(kThreads, STOCH ? 4 : encode_ctas_per_sm<T, BITS>())
     encode_kernel(const State st, const EncodeArgs a, const LaunchPlan plan) {
   const int tid = threadIdx.x;
   const int lane = tid & 31;
@@ -468,10 +506,11 @@ __global__ void __launch_bounds__(kThreads, encode_ctas_per_sm<T, BITS>())
     // whole iterations first (rows without a ragged end: no bounds to check), then the rest
     const int whole_end = min(r_end, st.chunks / kThreads);
     for (; r + kRowsPerIter <= whole_end; r += kRowsPerIter)
-      encode_rows<T, BITS, LPG, true>(st, act, m, stream, scales, r * kThreads + tid, kRowsPerIter, lane, words_ok);
+      encode_rows<T, BITS, LPG, STOCH, true>(st, a, (uint32_t)sample.id, act, m, stream, scales, r * kThreads + tid,
+                                             kRowsPerIter, lane, words_ok);
     for (; r < r_end; r += kRowsPerIter)
-      encode_rows<T, BITS, LPG, false>(st, act, m, stream, scales, r * kThreads + tid, min(kRowsPerIter, r_end - r),
-                                       lane, words_ok);
+      encode_rows<T, BITS, LPG, STOCH, false>(st, a, (uint32_t)sample.id, act, m, stream, scales, r * kThreads + tid,
+                                              min(kRowsPerIter, r_end - r), lane, words_ok);
   } else {
     // first visit: the activation itself becomes m(xi); skipped sample: nothing is stored.
     // Either way the sample's codes and scales are zero.
@@ -576,10 +615,11 @@ __global__ void __launch_bounds__(kThreads, decode_ctas_per_sm<BITS>()) decode_k
 
 // ------------------------------------------------------------------ backward direction: direct quantization
 
-template <typename T, int BITS, int LPG>
+template <typename T, int BITS, int LPG, bool STOCH>
 __global__ void __launch_bounds__(kThreads) quant_grad_kernel(const T* __restrict__ grad, long long n_chunks,
                                                               int lanes_per_group, uint8_t* __restrict__ packed,
-                                                              float* __restrict__ scales) {
+                                                              float* __restrict__ scales, unsigned long long seed,
+                                                              unsigned long long epoch) {
   const int lane = threadIdx.x & 31;
   const int lg_shift = __ffs(lanes_per_group) - 1;
   const long long c0 = (long long)blockIdx.x * kChunksPerCta + threadIdx.x;
@@ -599,7 +639,9 @@ __global__ void __launch_bounds__(kThreads) quant_grad_kernel(const T* __restric
     const float s = group_max<LPG>(abs_max8(d), lanes_per_group);
     float delta;
     unsigned long long codes;
-    quantize8<T, BITS>(d, s, delta, codes, q);
+    uint4 noise = make_uint4(0, 0, 0, 0);
+    if constexpr (STOCH) noise = chunk_noise(seed, epoch, 0xFFFFFFFFu, (uint32_t)c);
+    quantize8<T, BITS, STOCH>(d, s, noise, delta, codes, q);
     if (active && (lane & (lanes_per_group - 1)) == 0) scales[c >> lg_shift] = delta;
     store_codes<BITS>(packed, c, lane, active, c - lane + 32 <= n_chunks, codes);
   }
@@ -748,7 +790,9 @@ cudaError_t launch_rows(K kernel, const State& st, const Args& a, cudaStream_t s
 }  // namespace
 
 cudaError_t launch_encode(int dtype, int bits, const State& st, const EncodeArgs& a, cudaStream_t s) {
-#define AQ_CALL_LPG(L) return launch_rows(encode_kernel<T_, B_, L>, st, a, s)
+#define AQ_CALL_LPG(L)                                                         \
+  return a.stochastic ? launch_rows(encode_kernel<T_, B_, L, true>, st, a, s) \
+                      : launch_rows(encode_kernel<T_, B_, L, false>, st, a, s)
 #define AQ_CALL(T, B)                                      \
   {                                                        \
     using T_ = T;                                          \
@@ -769,12 +813,18 @@ cudaError_t launch_decode(int dtype, int bits, const State& st, const DecodeArgs
 }
 
 cudaError_t launch_quant_grad(int dtype, int bits, int lanes_per_group, const void* grad, long long n_elems,
-                              uint8_t* packed, float* scales, cudaStream_t s) {
+                              uint8_t* packed, float* scales, bool stochastic, unsigned long long seed,
+                              unsigned long long epoch, cudaStream_t s) {
   if (n_elems <= 0) return cudaSuccess;
   const long long chunks = n_elems / kChunk;
   const unsigned grid = grid_x(chunks);
-#define AQ_CALL_LPG(L) \
-  return launch_overlapped(quant_grad_kernel<T_, B_, L>, dim3(grid), s, reinterpret_cast<const T_*>(grad), chunks, lanes_per_group, packed, scales)
+#define AQ_CALL_LPG(L)                                                                                              \
+  return stochastic ? launch_overlapped(quant_grad_kernel<T_, B_, L, true>, dim3(grid), s,                          \
+                                        reinterpret_cast<const T_*>(grad), chunks, lanes_per_group, packed, scales, \
+                                        seed, epoch)                                                                \
+                    : launch_overlapped(quant_grad_kernel<T_, B_, L, false>, dim3(grid), s,                         \
+                                        reinterpret_cast<const T_*>(grad), chunks, lanes_per_group, packed, scales, \
+                                        seed, epoch)
 #define AQ_CALL(T, B)                                      \
   {                                                        \
     using T_ = T;                                          \

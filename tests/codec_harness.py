@@ -40,7 +40,7 @@ class GpuSide:
         return np.stack([self.m_row(i)[0] for i in range(self.cfg.n_samples)])
 
 
-def run_boundary(cfg, n_batch=None, epochs=None, check_all_m=True, order_fn=None, act_fn=None):
+def run_boundary(cfg, n_batch=None, epochs=None, check_all_m=True, order_fn=None, act_fn=None, stochastic_seed=None):
     """Every call of every epoch: GPU sender -> GPU receiver and oracle sender -> oracle
     receiver; packed, scales, first flags, out and (per epoch) both m arrays and the state
     digests must agree exactly."""
@@ -54,7 +54,13 @@ def run_boundary(cfg, n_batch=None, epochs=None, check_all_m=True, order_fn=None
     scales = torch.empty((nb, cfg.groups), dtype=torch.float32, device="cuda")
     out = torch.empty((nb, cfg.seq, cfg.hidden), dtype=cfg.torch_dtype, device="cuda")
     try:
+        if stochastic_seed is not None:                      # only the sender rounds; the receiver needs no setting
+            aq.aq_configure(gs.h, aq.AQ_ROUNDING, aq.AQ_ROUND_STOCHASTIC)
+            aq.aq_configure(gs.h, aq.AQ_SEED, stochastic_seed)
         for epoch in range(epochs):
+            if stochastic_seed is not None:
+                aq.aq_configure(gs.h, aq.AQ_EPOCH, (epoch << 33) | 5)          # both counter words in use
+                os_.set_rounding(True, stochastic_seed, (epoch << 33) | 5)
             order = order_fn(epoch) if order_fn else synth.epoch_order(cfg, epoch)
             for c in range(cfg.n_samples // nb):
                 ids = order[c * nb:(c + 1) * nb].contiguous()

@@ -315,3 +315,55 @@ def test_replayed_cuda_graph_counts_every_replay_as_a_call():
     finally:
         gs.close()
         gr.close()
+
+
+# ----------------------------------------------------------------- unbiased stochastic rounding (Philox4x32-10)
+
+def test_stochastic_rounding_tiny_boundary():
+    run_boundary(synth.TINY, stochastic_seed=0x1234567890ABCDEF)
+
+
+def test_stochastic_rounding_large_shapes_reduced_id_space():
+    run_boundary(synth.shrink(synth.GPT2_XL, 8, seq=160, epochs=3), n_batch=4, stochastic_seed=7)
+    run_boundary(synth.shrink(synth.DEBERTA_XXL, 16, seq=64), stochastic_seed=8)
+    run_boundary(synth.shrink(synth.SWEEP_FWD, 4, seq=96), stochastic_seed=9)
+
+
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+@pytest.mark.parametrize("bits", range(1, 9))
+def test_stochastic_rounding_every_bit_width_on_ragged_shapes(dtype, bits):
+    cfg = synth.Boundary("sr-ragged", 6, 3, 37, 136, dtype, bits, 8, 3, "outlier", 0.3, seed=70 + bits)
+    run_boundary(cfg, stochastic_seed=1000 + bits)
+    cfg = synth.Boundary("sr-groups", 4, 2, 3, 1024, dtype, bits, 256, 3, "student_t3", 0.2, seed=90 + bits)
+    run_boundary(cfg, stochastic_seed=2000 + bits)
+
+
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+@pytest.mark.parametrize("bits", [1, 3, 4, 6, 8])
+def test_stochastic_gradient_quantization_matches_oracle(dtype, bits):
+    td = torch.float16 if dtype == "fp16" else torch.bfloat16
+    group, n_groups = 64, 4097
+    n = group * n_groups
+    h = aq.aq_create(1, 1, group, 4, group)
+    try:
+        aq.aq_configure(h, aq.AQ_DTYPE, DT[dtype][0])
+        aq.aq_configure(h, aq.AQ_ROUNDING, aq.AQ_ROUND_STOCHASTIC)
+        aq.aq_configure(h, aq.AQ_SEED, 424242)
+        grad = _grad_input(n, group, td, 5000 + bits).cuda()
+        packed = torch.empty(n * bits // 8, dtype=torch.uint8, device="cuda")
+        scales = torch.empty(n // group, dtype=torch.float32, device="cuda")
+        out = torch.empty(n, dtype=td, device="cuda")
+        seen = []
+        for epoch in (3, (1 << 40) + 3):
+            aq.aq_configure(h, aq.AQ_EPOCH, epoch)
+            aq.aq_quant_grad(h, grad, n, bits, packed, scales)
+            aq.aq_dequant_grad(h, packed, scales, n, bits, out)
+            torch.cuda.synchronize()
+            p_o, s_o = oracle.quant_grad_stochastic(bits16(grad), bits, group, 424242, epoch, DT[dtype][1])
+            assert np.array_equal(packed.cpu().numpy(), p_o)
+            assert np.array_equal(scales.cpu().numpy().view(np.uint32), s_o.view(np.uint32))
+            assert np.array_equal(bits16(out), oracle.dequant_grad(p_o, s_o, n, bits, group, DT[dtype][1]))
+            seen.append(p_o)
+        assert not np.array_equal(seen[0], seen[1])
+    finally:
+        aq.aq_destroy(h)
