@@ -51,6 +51,8 @@ def parse_args():
     ap.add_argument("--workload", default="gpt2", choices=sorted(WORKLOADS))
     ap.add_argument("--per-launch", type=int, default=0, help="sequences handed to one aq_encode call (0 = the whole macro-batch)")
     ap.add_argument("--graph", action="store_true", help="replay each step as a captured CUDA graph")
+    ap.add_argument("--rounding", default="interval", choices=["interval", "stochastic"],
+                    help="quantizer of the sender: interval number (default) or unbiased stochastic rounding")
     ap.add_argument("--rows-per-cta", type=int, default=0, help="AQ_ROWS_PER_CTA of both handles (0 = library default)")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--skip-e2e", action="store_true")
@@ -268,6 +270,9 @@ def main():
         aq.aq_configure(h, aq.AQ_STREAM, stream.cuda_stream)
         if args.rows_per_cta:
             aq.aq_configure(h, aq.AQ_ROWS_PER_CTA, args.rows_per_cta)
+        if args.rounding == "stochastic":
+            aq.aq_configure(h, aq.AQ_ROUNDING, aq.AQ_ROUND_STOCHASTIC)
+            aq.aq_configure(h, aq.AQ_SEED, 20220601)
         handles.append(h)
     snd, rcv = handles
 
@@ -429,7 +434,7 @@ def main():
     launch_bytes = nb * cfg.elems * bpe
     enc_gbs = launch_bytes / (enc_ms * 1e-3) / 1e9
     dec_gbs = launch_bytes / (dec_ms * 1e-3) / 1e9
-    traffic = NCU_TRAFFIC_BYTES_PER_ELEMENT["encode"] if args.workload == NCU_TRAFFIC_WORKLOAD else None
+    traffic = NCU_TRAFFIC_BYTES_PER_ELEMENT["encode"] if (args.workload == NCU_TRAFFIC_WORKLOAD and args.rounding == "interval") else None
     value = replicas.whole_job_rate(args.steps * step_bytes, world, elapsed_ms) / 1e9
     line = {
         "metric": "activation encode+decode GB/s", "value": value, "unit": "GB/s",
@@ -437,7 +442,7 @@ def main():
         "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": label, "hidden": cfg.hidden, "seq": cfg.seq,
-                   "micro_batch": cfg.n_batch, "sequences_per_step": MACRO, "sequences_per_launch": nb, "cuda_graph": bool(args.graph),
+                   "micro_batch": cfg.n_batch, "sequences_per_step": MACRO, "sequences_per_launch": nb, "cuda_graph": bool(args.graph), "rounding": args.rounding,
                    "act_dtype": cfg.dtype, "bits": cfg.bits, "group": cfg.group, "n_samples_per_side": cfg.n_samples,
                    "m_bytes_per_side": cfg.n_samples * cfg.elems * 2, "steady_epochs_resident": n_arenas,
                    "l2": f"inputs larger than L2 (each step touches {int(MACRO * cfg.elems * 6 / 1e6)} MB of fresh HBM; no flush needed)",

@@ -169,7 +169,7 @@ __device__ __forceinline__ void quantize8(const float (&d)[8], float s, const ui
     if constexpr (STOCH) {
       const uint32_t h = (j & 1) ? (nw[j >> 1] >> 16) : (nw[j >> 1] & 0xFFFFu);
       const float hc = __fsub_rn(__uint_as_float(0x4A800001u | (h << 1)), 4227072.0f);   // h - 32767.5, exact
-      u = __fadd_rn(u, __fmul_rn(hc, noise_unit));
+      u = __fmaf_rn(hc, noise_unit, u);                      // hc * 2^-16 is exact: the same sum, one rounding
     }
     if constexpr (Conv<T>::kWide || STOCH) u = fmaxf(u, kLo);
     u = fminf(u, kHi);
