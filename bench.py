@@ -266,6 +266,7 @@ def main():
     handles = []
     for _ in range(2):
         h = aq.aq_create(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group)
+        aq.aq_configure(h, aq.AQ_DTYPE, aq.AQ_FP16 if cfg.dtype == "fp16" else aq.AQ_BF16)
         aq.aq_configure(h, aq.AQ_BATCH, nb)
         aq.aq_configure(h, aq.AQ_STREAM, stream.cuda_stream)
         if args.rows_per_cta:
@@ -335,6 +336,24 @@ def main():
         return e[0].elapsed_time(e[1]) / n, e[1].elapsed_time(e[2]) / n
 
     ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    # one throw-away visit on a small boundary of the same type, bit width and group: the first launch of a
+    # kernel loads its code (milliseconds), which must not count as first-visit time
+    warm = [aq.aq_create(2, 8, cfg.hidden, cfg.bits, cfg.group) for _ in range(2)]
+    for h in warm:
+        aq.aq_configure(h, aq.AQ_DTYPE, aq.AQ_FP16 if cfg.dtype == "fp16" else aq.AQ_BF16)
+        aq.aq_configure(h, aq.AQ_STREAM, stream.cuda_stream)
+        if args.rounding == "stochastic":
+            aq.aq_configure(h, aq.AQ_ROUNDING, aq.AQ_ROUND_STOCHASTIC)
+    w_act = torch.zeros((1, 8, cfg.hidden), dtype=cfg.torch_dtype, device="cuda")
+    w_ids = torch.zeros(1, dtype=torch.int32, device="cuda")
+    aq.aq_configure(warm[1], aq.AQ_RAW, w_act)
+    for _ in range(2):                                 # a first visit, then a delta visit
+        aq.aq_encode(warm[0], w_act, w_ids, packed[:1], scales[:1])
+        aq.aq_decode(warm[1], packed[:1], scales[:1], w_ids, out[:1])
+    torch.cuda.synchronize()
+    for h in warm:
+        aq.aq_destroy(h)
 
     # ---- epoch 0: first visits (uncompressed message), timed apart
     order0 = synth.epoch_order(cfg, 0)
