@@ -141,7 +141,8 @@ __device__ __forceinline__ uint32_t pack_fields(const uint32_t* tb) {
 // * The lower clamp is only compiled for the wide type: with |d| <= s and a normal
 //   reciprocal, |d * RN(1/delta)| < 2^(b-1) * (1 + 2^-24), which rounds to at most 2^(b-1).
 // * (k + 1/2) * delta, rounded once, is fma(k, delta, delta/2) whenever delta/2 is exact,
-//   i.e. delta >= 2^-125; the wide type falls back to add-then-multiply below that.
+//   i.e. delta >= 2^-125, which always holds for fp16 inputs; the wide type adds 1/2 to k
+//   (exact) and multiplies.
 // STOCH (the unbiased quantizer that Theorem 3.1 assumes): delta = s / (2^(b-1) - 1/2), so that
 // the 2^b levels (k + 1/2) * delta reach from -s to +s, and k = floor(d / delta - 1/2 + r) with
 // r uniform in [0,1) from `noise`; both clamps are needed then.
@@ -176,16 +177,10 @@ __device__ __forceinline__ void quantize8(const float (&d)[8], float s, const ui
     const float t = __fadd_rd(u, kMagic);
     tb[j] = __float_as_uint(t);
     const float kf = __fsub_rn(t, kMagic);                   // exact: (float)k
-    q[j] = __fmaf_rn(kf, delta, half_delta);
-  }
-  if constexpr (Conv<T>::kWide) {
-    if (live && delta < 2.3509887e-38f) {                    // 2^-125: delta/2 may have lost a bit
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const float kf = __fsub_rn(__uint_as_float(tb[j]), kMagic);
-        q[j] = __fmul_rn(__fadd_rn(kf, 0.5f), delta);
-      }
-    }
+    if constexpr (Conv<T>::kWide)
+      q[j] = __fmul_rn(__fadd_rn(kf, 0.5f), delta);          // delta / 2 may be inexact below 2^-125
+    else
+      q[j] = __fmaf_rn(kf, delta, half_delta);
   }
   if constexpr (BITS <= 4) {
     codes = pack_fields<BITS, 8>(tb);
@@ -476,7 +471,7 @@ __device__ __forceinline__ void encode_rows(const State& st, const EncodeArgs& a
 template <typename T, int BITS>
 constexpr int encode_ctas_per_sm() {
   const bool whole_words = BITS == 1 || BITS == 2 || BITS == 4;
-  return !whole_words ? (Conv<T>::kWide ? 3 : 4) : (Conv<T>::kWide ? 5 : 6);
+  return !whole_words ? (Conv<T>::kWide ? 3 : 4) : 6;
 }
 template <int BITS>
 constexpr int decode_ctas_per_sm() {
