@@ -513,34 +513,53 @@ def isolated_calls(aq, torch, stream, snd, rcv, cfg, arena, ids_dev, reps=40):
 
 def aux_kernels(aq, torch, synth, stream, h, cfg):
     """The remaining kernels of the path, each timed alone over rotating buffers larger than L2:
-    gradient quantize / dequantize (the 'Backward path' workload) and the state digest."""
+    gradient quantize / dequantize (the 'Backward path' workload: 4 x 1024 x 1600 per call, and the
+    same kernels on 16 such micro-batches handed over in one call) and the state digest.
+    Per call: CUDA events around 60 calls issued back to back through the binding ("stream"), and
+    around 5 replays of a CUDA graph of 12 calls ("graph": no host pacing between the launches)."""
+    from dataclasses import replace
     g = synth.BACKWARD
-    n = g.elems
-    grads = [synth.gradient(g, i, device="cuda") for i in range(12)]       # 12 x 13 MB > L2
     res = {}
     ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def timed(fn, reps):
+        a, b = ev(), ev()
+        a.record(stream)
+        for _ in range(reps):
+            fn()
+        b.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b)
+
     with torch.cuda.stream(stream):
-        for bits in g.bits:
-            packed = [torch.empty(n * bits // 8, dtype=torch.uint8, device="cuda") for _ in range(12)]
-            scales = [torch.empty(n // g.group, dtype=torch.float32, device="cuda") for _ in range(12)]
-            outs = [torch.empty(n, dtype=torch.float16, device="cuda") for _ in range(12)]
-            for name in ("quant", "dequant"):
-                def call(i):
-                    if name == "quant":
-                        aq.aq_quant_grad(h, grads[i], n, bits, packed[i], scales[i])
-                    else:
-                        aq.aq_dequant_grad(h, packed[i], scales[i], n, bits, outs[i])
-                for i in range(12):
-                    call(i)
-                a, b = ev(), ev()
-                a.record(stream)
-                for r in range(5):
-                    for i in range(12):
-                        call(i)
-                b.record(stream)
-                torch.cuda.synchronize()
-                ms = a.elapsed_time(b) / 60
-                res[f"{name}_grad_b{bits}"] = {"ms": ms, "GB/s": n * (2 + bits / 8 + 4 / g.group) / (ms * 1e-3) / 1e9}
+        for label, gw, sets in (("", g, 12), ("_x16", replace(g, n_batch=16 * g.n_batch), 3)):
+            n = gw.elems
+            grads = [synth.gradient(gw, i, device="cuda") for i in range(sets)]          # sets x n x 2 B > L2
+            for bits in g.bits:
+                packed = [torch.empty(n * bits // 8, dtype=torch.uint8, device="cuda") for _ in range(sets)]
+                scales = [torch.empty(n // g.group, dtype=torch.float32, device="cuda") for _ in range(sets)]
+                outs = [torch.empty(n, dtype=torch.float16, device="cuda") for _ in range(sets)]
+                for name in ("quant", "dequant"):
+                    def sweep():
+                        for i in range(sets):
+                            if name == "quant":
+                                aq.aq_quant_grad(h, grads[i], n, bits, packed[i], scales[i])
+                            else:
+                                aq.aq_dequant_grad(h, packed[i], scales[i], n, bits, outs[i])
+                    sweep()
+                    torch.cuda.synchronize()
+                    ms_stream = timed(sweep, 5) / (5 * sets)
+                    graph = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(graph, stream=stream):
+                        sweep()
+                    graph.replay()
+                    torch.cuda.synchronize()
+                    ms_graph = timed(graph.replay, 5) / (5 * sets)
+                    ms = min(ms_stream, ms_graph)
+                    res[f"{name}_grad_b{bits}{label}"] = {
+                        "ms": ms, "ms_stream": ms_stream, "ms_graph": ms_graph,
+                        "GB/s": n * (2 + bits / 8 + 4 / g.group) / (ms * 1e-3) / 1e9}
+            del grads
     t0 = time.perf_counter()
     aq.aq_state_checksum(h)
     dt = time.perf_counter() - t0
