@@ -68,6 +68,24 @@ def lib():
         L.aqo_quant_grad_stochastic.restype = None
         L.aqo_quant_grad_stochastic.argtypes = [u16p, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_uint64, C.c_uint64,
                                                 u8p, f32p]
+        L.aqo_low_create.restype = C.c_void_p
+        L.aqo_low_create.argtypes = [C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int]
+        L.aqo_low_destroy.restype = None
+        L.aqo_low_destroy.argtypes = [C.c_void_p]
+        L.aqo_low_m_codes.restype = u8p
+        L.aqo_low_m_codes.argtypes = [C.c_void_p]
+        L.aqo_low_m_scales.restype = f32p
+        L.aqo_low_m_scales.argtypes = [C.c_void_p]
+        L.aqo_low_seen.restype = u8p
+        L.aqo_low_seen.argtypes = [C.c_void_p]
+        L.aqo_low_status.restype = C.c_uint32
+        L.aqo_low_status.argtypes = [C.c_void_p]
+        L.aqo_low_encode.restype = None
+        L.aqo_low_encode.argtypes = [C.c_void_p, u16p, i32p, C.c_int, u8p, f32p, u8p]
+        L.aqo_low_decode.restype = None
+        L.aqo_low_decode.argtypes = [C.c_void_p, u8p, f32p, u16p, i32p, C.c_int, u16p, u8p]
+        L.aqo_low_state_checksum.restype = C.c_uint64
+        L.aqo_low_state_checksum.argtypes = [C.c_void_p]
         L.aqo_state_checksum.restype = C.c_uint64
         L.aqo_state_checksum.argtypes = [C.c_void_p]
         _lib = L
@@ -218,6 +236,79 @@ class Side:
 
     def checksum(self):
         return lib().aqo_state_checksum(self.h)
+
+
+class SideLow:
+    """One copy of m kept in m_bits bits per element (codes + one fp32 step per group)."""
+
+    def __init__(self, n_samples, seq, hidden, bits, group, dtype=FP16, m_bits=8):
+        self.n_samples, self.seq, self.hidden = n_samples, seq, hidden
+        self.bits, self.group, self.dtype, self.m_bits = bits, group, dtype, m_bits
+        self.h = lib().aqo_low_create(n_samples, seq, hidden, bits, group, dtype, m_bits)
+        if not self.h:
+            raise ValueError("aqo_low_create rejected the configuration")
+        self.E = seq * hidden
+        self.pbytes = self.E * bits // 8
+        self.ngroups = self.E // group
+        self.mbytes = self.E * m_bits // 8
+
+    def close(self):
+        if self.h:
+            lib().aqo_low_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        self.close()
+
+    def m_codes(self):
+        return np.ctypeslib.as_array(lib().aqo_low_m_codes(self.h), shape=(self.n_samples, self.mbytes))
+
+    def m_scales(self):
+        return np.ctypeslib.as_array(lib().aqo_low_m_scales(self.h), shape=(self.n_samples, self.ngroups))
+
+    def m_values(self):
+        """The dequantized store as float64 [n_samples, E]."""
+        out = np.empty((self.n_samples, self.E), np.float64)
+        for i in range(self.n_samples):
+            k = get_codes(self.m_codes()[i], self.E, self.m_bits).astype(np.float64)
+            out[i] = (k + 0.5) * np.repeat(self.m_scales()[i].astype(np.float64), self.group)
+        return out
+
+    def seen(self):
+        return np.ctypeslib.as_array(lib().aqo_low_seen(self.h), shape=(self.n_samples,))
+
+    def status(self):
+        return lib().aqo_low_status(self.h)
+
+    def encode(self, act, ids):
+        act = _c(act, np.uint16)
+        ids = _c(ids, np.int32)
+        nb = ids.shape[0]
+        assert act.size == nb * self.E
+        packed = np.empty((nb, self.pbytes), np.uint8)
+        scales = np.empty((nb, self.ngroups), np.float32)
+        first = np.zeros(nb, np.uint8)
+        lib().aqo_low_encode(self.h, _p(act, C.c_uint16), _p(ids, C.c_int32), nb,
+                             _p(packed, C.c_uint8), _p(scales, C.c_float), _p(first, C.c_uint8))
+        return packed, scales, first
+
+    def decode(self, packed, scales, ids, raw=None):
+        packed = _c(packed, np.uint8)
+        scales = _c(scales, np.float32)
+        ids = _c(ids, np.int32)
+        nb = ids.shape[0]
+        out = np.empty((nb, self.seq, self.hidden), np.uint16)
+        first = np.zeros(nb, np.uint8)
+        rawp = None
+        if raw is not None:
+            raw = _c(raw, np.uint16)
+            rawp = _p(raw, C.c_uint16)
+        lib().aqo_low_decode(self.h, _p(packed, C.c_uint8), _p(scales, C.c_float), rawp,
+                             _p(ids, C.c_int32), nb, _p(out, C.c_uint16), _p(first, C.c_uint8))
+        return out, first
+
+    def checksum(self):
+        return lib().aqo_low_state_checksum(self.h)
 
 
 def quant_grad(grad, bits, group, dtype=FP16):

@@ -310,6 +310,50 @@ uint64_t mix64(uint64_t index, uint64_t word) {
   return z ^ (z >> 31);
 }
 
+// ---------------------------------------------------------------------------
+// Previous messages kept at low precision (appendix "Number of Bits for
+// Previous Messages": "we perform quantization on m, where mz means that we
+// use z bits for previous messages").  The paper gives no formula; reading
+// fixed here: m is stored per group of G hidden elements as z-bit codes plus
+// one fp32 step, with the same Q as the messages (interval number, centre
+// reconstruction, max-abs normaliser), and every visit works on the
+// dequantized store:
+//
+//   m_deq  = (km + 1/2) * Delta_m                 (0 for a group with Delta_m = 0)
+//   sender: Delta_msg = Q_b(a - m_deq)            receiver: gets Delta_msg
+//   m_new  = m_deq + Delta_msg                    (fp32, one rounding; not rounded to T)
+//   store  <- Q_z(m_new);   the receiver's activation is T(m_new)
+//   first visit: m_new = a (resp. the raw message), store <- Q_z(m_new), activation = the raw message.
+//
+// Both sides run the same deterministic steps on the same numbers, so their
+// stores stay identical.
+// ---------------------------------------------------------------------------
+
+struct SideLow {
+  int64_t n_samples;
+  int seq, hidden, bits, group, dtype, m_bits;
+  std::vector<uint8_t> m_codes;   // [n_samples][seq*hidden*m_bits/8], bitstream layout of the messages
+  std::vector<float> m_scales;    // [n_samples][seq*hidden/group], Delta_m of every group
+  std::vector<uint8_t> seen;
+  uint32_t status;
+};
+
+int resolve_low(SideLow* S, const int32_t* ids, int y) {
+  const int64_t id = ids[y];
+  if (id < 0 || id >= S->n_samples) { S->status |= ST_BAD_ID; return 2; }
+  for (int p = 0; p < y; ++p)
+    if (ids[p] == ids[y]) { S->status |= ST_DUP_ID; return 2; }
+  return S->seen[id] ? 0 : 1;
+}
+
+// store <- Q_z(m_new) for one group
+void store_group(SideLow* S, uint8_t* MC, float* MS, int64_t g, const float* m_new, int32_t* km) {
+  float dm;
+  quantize_group(m_new, S->group, S->m_bits, km, &dm);
+  MS[g] = dm;
+  for (int j = 0; j < S->group; ++j) put_code(MC, g * S->group + j, S->m_bits, km[j]);
+}
+
 }  // namespace
 
 extern "C" {
@@ -504,6 +548,123 @@ uint64_t aqo_state_checksum(void* h) {
     const uint32_t w = (uint32_t)S->m[2 * i] | ((uint32_t)S->m[2 * i + 1] << 16);
     sum += mix64((uint64_t)i, w);
   }
+  for (int64_t x = 0; x < S->n_samples; ++x)
+    sum += mix64((1ull << 40) + (uint64_t)x, S->seen[x]);
+  return sum;
+}
+
+// ---- one side of one boundary, previous messages stored in m_bits bits per element
+
+void* aqo_low_create(int64_t n_samples, int seq, int hidden, int bits, int group, int dtype, int m_bits) {
+  if (n_samples <= 0 || seq <= 0 || hidden <= 0 || bits < 1 || bits > 8 || group <= 0) return nullptr;
+  if (m_bits < 1 || m_bits > 8 || hidden % group != 0 || (dtype != DT_FP16 && dtype != DT_BF16)) return nullptr;
+  const int64_t E = (int64_t)seq * hidden;
+  if ((E * bits) % 8 != 0 || (E * m_bits) % 8 != 0) return nullptr;
+  SideLow* S = new (std::nothrow) SideLow();
+  if (!S) return nullptr;
+  S->n_samples = n_samples; S->seq = seq; S->hidden = hidden; S->bits = bits; S->group = group;
+  S->dtype = dtype; S->m_bits = m_bits; S->status = 0;
+  S->m_codes.assign((size_t)(n_samples * E * m_bits / 8), 0);     // codes 0, steps 0: "initialized to 0"
+  S->m_scales.assign((size_t)(n_samples * E / group), 0.0f);
+  S->seen.assign((size_t)n_samples, 0);
+  return S;
+}
+void aqo_low_destroy(void* h) { delete (SideLow*)h; }
+const uint8_t* aqo_low_m_codes(void* h) { return ((SideLow*)h)->m_codes.data(); }
+const float* aqo_low_m_scales(void* h) { return ((SideLow*)h)->m_scales.data(); }
+const uint8_t* aqo_low_seen(void* h) { return ((SideLow*)h)->seen.data(); }
+uint32_t aqo_low_status(void* h) { SideLow* S = (SideLow*)h; uint32_t s = S->status; S->status = 0; return s; }
+
+void aqo_low_encode(void* h, const uint16_t* act, const int32_t* ids, int n_batch, uint8_t* packed, float* scales,
+                    uint8_t* first) {
+  SideLow* S = (SideLow*)h;
+  const int64_t E = (int64_t)S->seq * S->hidden, G = S->group;
+  const int64_t pbytes = E * S->bits / 8, ngroups = E / G, mbytes = E * S->m_bits / 8;
+  std::vector<float> d(G), m_deq(G), m_new(G);
+  std::vector<int32_t> k(G), km(G);
+  for (int y = 0; y < n_batch; ++y) {
+    const uint16_t* a = act + (int64_t)y * E;
+    uint8_t* P = packed + (int64_t)y * pbytes;
+    float* SC = scales + (int64_t)y * ngroups;
+    std::memset(P, 0, (size_t)pbytes);
+    for (int64_t g = 0; g < ngroups; ++g) SC[g] = 0.0f;
+    const int mode = resolve_low(S, ids, y);
+    if (first) first[y] = (uint8_t)(mode == 1);
+    if (mode == 2) continue;
+    uint8_t* MC = S->m_codes.data() + (int64_t)ids[y] * mbytes;
+    float* MS = S->m_scales.data() + (int64_t)ids[y] * ngroups;
+    for (int64_t g = 0; g < ngroups; ++g) {
+      const int64_t base = g * G;
+      if (mode == 1) {
+        for (int j = 0; j < G; ++j) m_new[j] = t_to_float(a[base + j], S->dtype);
+      } else {
+        for (int j = 0; j < G; ++j) {
+          m_deq[j] = reconstruct(get_code(MC, base + j, S->m_bits), MS[g]);
+          d[j] = t_to_float(a[base + j], S->dtype) - m_deq[j];
+        }
+        float delta;
+        quantize_group(d.data(), (int)G, S->bits, k.data(), &delta);
+        SC[g] = delta;
+        for (int j = 0; j < G; ++j) {
+          put_code(P, base + j, S->bits, k[j]);
+          m_new[j] = m_deq[j] + reconstruct(k[j], delta);
+        }
+      }
+      store_group(S, MC, MS, g, m_new.data(), km.data());
+    }
+    if (mode == 1) S->seen[ids[y]] = 1;
+  }
+}
+
+void aqo_low_decode(void* h, const uint8_t* packed, const float* scales, const uint16_t* raw, const int32_t* ids,
+                    int n_batch, uint16_t* out, uint8_t* first) {
+  SideLow* S = (SideLow*)h;
+  const int64_t E = (int64_t)S->seq * S->hidden, G = S->group;
+  const int64_t pbytes = E * S->bits / 8, ngroups = E / G, mbytes = E * S->m_bits / 8;
+  std::vector<float> m_new(G);
+  std::vector<int32_t> km(G);
+  for (int y = 0; y < n_batch; ++y) {
+    uint16_t* O = out + (int64_t)y * E;
+    int mode = resolve_low(S, ids, y);
+    if (mode == 1 && raw == nullptr) { S->status |= ST_NO_RAW; mode = 2; }
+    if (first) first[y] = (uint8_t)(mode == 1);
+    if (mode == 2) { for (int64_t i = 0; i < E; ++i) O[i] = 0; continue; }
+    uint8_t* MC = S->m_codes.data() + (int64_t)ids[y] * mbytes;
+    float* MS = S->m_scales.data() + (int64_t)ids[y] * ngroups;
+    const uint8_t* P = packed + (int64_t)y * pbytes;
+    const float* SC = scales + (int64_t)y * ngroups;
+    const uint16_t* R = raw ? raw + (int64_t)y * E : nullptr;
+    for (int64_t g = 0; g < ngroups; ++g) {
+      const int64_t base = g * G;
+      for (int j = 0; j < G; ++j) {
+        if (mode == 1) {
+          m_new[j] = t_to_float(R[base + j], S->dtype);
+          O[base + j] = R[base + j];
+        } else {
+          const float m_deq = reconstruct(get_code(MC, base + j, S->m_bits), MS[g]);
+          m_new[j] = m_deq + reconstruct(get_code(P, base + j, S->bits), SC[g]);
+          O[base + j] = float_to_t(m_new[j], S->dtype);
+        }
+      }
+      store_group(S, MC, MS, g, m_new.data(), km.data());
+    }
+    if (mode == 1) S->seen[ids[y]] = 1;
+  }
+}
+
+// Digest of a low-precision state: the code bytes read as little-endian 32-bit words, then the
+// steps' bit patterns (word index continuing), then the seen set as for the 16-bit state.
+uint64_t aqo_low_state_checksum(void* h) {
+  SideLow* S = (SideLow*)h;
+  uint64_t sum = 0;
+  const int64_t ncw = (int64_t)S->m_codes.size() / 4;
+  for (int64_t i = 0; i < ncw; ++i) {
+    uint32_t w;
+    std::memcpy(&w, S->m_codes.data() + 4 * i, 4);
+    sum += mix64((uint64_t)i, w);
+  }
+  for (int64_t i = 0; i < (int64_t)S->m_scales.size(); ++i)
+    sum += mix64((uint64_t)(ncw + i), f32_bits(S->m_scales[i]));
   for (int64_t x = 0; x < S->n_samples; ++x)
     sum += mix64((1ull << 40) + (uint64_t)x, S->seen[x]);
   return sum;
