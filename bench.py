@@ -53,6 +53,8 @@ def parse_args():
     ap.add_argument("--graph", action="store_true", help="replay each step as a captured CUDA graph")
     ap.add_argument("--rounding", default="interval", choices=["interval", "stochastic"],
                     help="quantizer of the sender: interval number (default) or unbiased stochastic rounding")
+    ap.add_argument("--m-bits", type=int, default=0, choices=[0, 2, 4, 8],
+                    help="keep the previous messages in this many bits per element (0 = the activation type)")
     ap.add_argument("--rows-per-cta", type=int, default=0, help="AQ_ROWS_PER_CTA of both handles (0 = library default)")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--skip-e2e", action="store_true")
@@ -62,9 +64,15 @@ def parse_args():
     return ap.parse_args()
 
 
+M_BITS = 0            # 0: m kept in the activation type; 2, 4, 8: low-precision store (--m-bits)
+
+
 def bytes_per_element(bits, group):
     """Algorithmic HBM bytes per element of a steady-state encode (= of a decode):
-    read a (2) + read m (2) + write m (2) + codes (b/8) + scale (4/G)."""
+    read a (2) + read m (2) + write m (2) + codes (b/8) + scale (4/G); with m kept in z bits:
+    a (2) + m read and written (2 * (z/8 + 4/G)) + codes (b/8) + scale (4/G)."""
+    if M_BITS:
+        return 2.0 + 2.0 * (M_BITS / 8.0 + 4.0 / group) + bits / 8.0 + 4.0 / group
     return 6.0 + bits / 8.0 + 4.0 / group
 
 
@@ -226,7 +234,8 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
 
     from paper_2206_01299_b200 import replicas, synth
-    global MACRO
+    global MACRO, M_BITS
+    M_BITS = args.m_bits
     recipe, MACRO, label = WORKLOADS[args.workload]
     cfg = getattr(synth, recipe)
     if args.n_samples:
@@ -265,7 +274,8 @@ def main():
 
     handles = []
     for _ in range(2):
-        h = aq.aq_create(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group)
+        h = (aq.aq_create_lowbit(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, args.m_bits) if args.m_bits
+             else aq.aq_create(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group))
         aq.aq_configure(h, aq.AQ_DTYPE, aq.AQ_FP16 if cfg.dtype == "fp16" else aq.AQ_BF16)
         aq.aq_configure(h, aq.AQ_BATCH, nb)
         aq.aq_configure(h, aq.AQ_STREAM, stream.cuda_stream)
@@ -339,7 +349,8 @@ def main():
 
     # one throw-away visit on a small boundary of the same type, bit width and group: the first launch of a
     # kernel loads its code (milliseconds), which must not count as first-visit time
-    warm = [aq.aq_create(2, 8, cfg.hidden, cfg.bits, cfg.group) for _ in range(2)]
+    warm = [aq.aq_create_lowbit(2, 8, cfg.hidden, cfg.bits, cfg.group, args.m_bits) if args.m_bits
+            else aq.aq_create(2, 8, cfg.hidden, cfg.bits, cfg.group) for _ in range(2)]
     for h in warm:
         aq.aq_configure(h, aq.AQ_DTYPE, aq.AQ_FP16 if cfg.dtype == "fp16" else aq.AQ_BF16)
         aq.aq_configure(h, aq.AQ_STREAM, stream.cuda_stream)
@@ -453,7 +464,8 @@ def main():
     launch_bytes = nb * cfg.elems * bpe
     enc_gbs = launch_bytes / (enc_ms * 1e-3) / 1e9
     dec_gbs = launch_bytes / (dec_ms * 1e-3) / 1e9
-    traffic = NCU_TRAFFIC_BYTES_PER_ELEMENT["encode"] if (args.workload == NCU_TRAFFIC_WORKLOAD and args.rounding == "interval") else None
+    traffic = NCU_TRAFFIC_BYTES_PER_ELEMENT["encode"] if (args.workload == NCU_TRAFFIC_WORKLOAD and args.rounding == "interval"
+                                                          and not args.m_bits) else None
     value = replicas.whole_job_rate(args.steps * step_bytes, world, elapsed_ms) / 1e9
     line = {
         "metric": "activation encode+decode GB/s", "value": value, "unit": "GB/s",
@@ -461,9 +473,9 @@ def main():
         "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": label, "hidden": cfg.hidden, "seq": cfg.seq,
-                   "micro_batch": cfg.n_batch, "sequences_per_step": MACRO, "sequences_per_launch": nb, "cuda_graph": bool(args.graph), "rounding": args.rounding,
+                   "micro_batch": cfg.n_batch, "sequences_per_step": MACRO, "sequences_per_launch": nb, "cuda_graph": bool(args.graph), "rounding": args.rounding, "m_bits": args.m_bits or 16,
                    "act_dtype": cfg.dtype, "bits": cfg.bits, "group": cfg.group, "n_samples_per_side": cfg.n_samples,
-                   "m_bytes_per_side": cfg.n_samples * cfg.elems * 2, "steady_epochs_resident": n_arenas,
+                   "m_bytes_per_side": cfg.n_samples * (cfg.elems * 2 if not args.m_bits else cfg.elems * args.m_bits // 8 + cfg.groups * 4), "steady_epochs_resident": n_arenas,
                    "l2": f"inputs larger than L2 (each step touches {int(MACRO * cfg.elems * 6 / 1e6)} MB of fresh HBM; no flush needed)",
                    "parallelism": f"dp{world} replicas, no collective"},
         "samples_per_s": replicas.whole_job_rate(args.steps * MACRO, world, elapsed_ms),

@@ -118,6 +118,20 @@ enum {
  */
 aq_handle* aq_create(int64_t n_samples, int seq, int hidden, int bits, int group);
 
+/*
+ * The same, with the previous messages kept at low precision (appendix "Number of Bits for
+ * Previous Messages": mz = z bits for m).  m is stored as m_bits-bit codes (2, 4 or 8) plus one
+ * fp32 step per group of `group` elements -- Q of this file applied to m -- and takes
+ * n_samples*seq*hidden*(m_bits/8 + 4/group) bytes.  Every visit works on the dequantized store:
+ *   m_deq = (km + 1/2) * Delta_m;  sender: Delta = Q_b(act - m_deq);  m_new = m_deq + Delta (binary32);
+ *   store <- Q_mbits(m_new);  the receiver's `out` is T(m_new);
+ *   first visit: m_new = act (resp. the raw message), out = the raw message.
+ * aq_encode / aq_decode and the host-buffer forms work as for aq_create; AQ_ROUND_STOCHASTIC and
+ * aq_state_checksum_noalloc answer AQ_EUNSUPPORTED on such a handle.  aq_state_checksum covers the
+ * code bytes (as 32-bit words), then the steps, then the seen-set.
+ */
+aq_handle* aq_create_lowbit(int64_t n_samples, int seq, int hidden, int bits, int group, int m_bits);
+
 /* Waits for the handle's stream, frees everything the handle owns.  NULL is allowed. */
 void aq_destroy(aq_handle* h);
 
@@ -194,6 +208,9 @@ const char* aq_last_error(aq_handle* h);
 /* Bytes of `packed` and floats of `scales` per sample for this handle's forward settings. */
 int64_t aq_packed_bytes_per_sample(aq_handle* h);
 int64_t aq_scales_per_sample(aq_handle* h);
+/* Bytes of one sample's stored m, the size of the host buffer of aq_export_sample / aq_import_sample:
+ * seq*hidden*2, or for a low-precision store the code bytes followed by the fp32 steps. */
+int64_t aq_m_bytes_per_sample(aq_handle* h);
 
 /*
  * Host-buffer forms: same operations, but every pointer is HOST memory (pinned memory
@@ -209,8 +226,9 @@ int aq_decode_host(aq_handle* h, const void* packed_host, const float* scales_ho
                    const void* raw_host, const int32_t* sample_ids_host, void* out_host);
 
 /*
- * State access for checkpoints and tests.  Copies one sample's m block (seq*hidden*2
- * bytes) and its seen flag between the handle and HOST memory; synchronises the stream.
+ * State access for checkpoints and tests.  Copies one sample's m block
+ * (aq_m_bytes_per_sample bytes) and its seen flag between the handle and HOST memory;
+ * synchronises the stream.
  */
 int aq_export_sample(aq_handle* h, int64_t sample_id, void* m_host, uint8_t* seen_host);
 int aq_import_sample(aq_handle* h, int64_t sample_id, const void* m_host, uint8_t seen);

@@ -21,6 +21,7 @@ AQ_ST_BAD_ID, AQ_ST_DUP_ID, AQ_ST_NO_RAW = 1, 2, 4
 # name -> (restype, argtypes); the load test checks these against the header
 SIGNATURES = {
     "aq_create": (C.c_void_p, [C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int]),
+    "aq_create_lowbit": (C.c_void_p, [C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int]),
     "aq_destroy": (None, [C.c_void_p]),
     "aq_configure": (C.c_int, [C.c_void_p, C.c_int, C.c_int64]),
     "aq_encode": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -33,6 +34,7 @@ SIGNATURES = {
     "aq_last_error": (C.c_char_p, [C.c_void_p]),
     "aq_packed_bytes_per_sample": (C.c_int64, [C.c_void_p]),
     "aq_scales_per_sample": (C.c_int64, [C.c_void_p]),
+    "aq_m_bytes_per_sample": (C.c_int64, [C.c_void_p]),
     "aq_encode_host": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "aq_decode_host": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "aq_export_sample": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]),
@@ -85,6 +87,13 @@ def _check(h, rc):
 
 def aq_create(n_samples, seq, hidden, bits, group):
     h = lib().aq_create(n_samples, seq, hidden, bits, group)
+    if not h:
+        raise AqError(AQ_EINVAL, aq_last_error(None))
+    return h
+
+
+def aq_create_lowbit(n_samples, seq, hidden, bits, group, m_bits):
+    h = lib().aq_create_lowbit(n_samples, seq, hidden, bits, group, m_bits)
     if not h:
         raise AqError(AQ_EINVAL, aq_last_error(None))
     return h
@@ -145,6 +154,10 @@ def aq_packed_bytes_per_sample(h):
 
 def aq_scales_per_sample(h):
     return lib().aq_scales_per_sample(h)
+
+
+def aq_m_bytes_per_sample(h):
+    return lib().aq_m_bytes_per_sample(h)
 
 
 def aq_encode_host(h, act_host, sample_ids_host, packed_host, scales_host):

@@ -96,7 +96,22 @@ int ensure_staging(aq_handle* h) {
 
 extern "C" {
 
+static aq_handle* create_handle(int64_t n_samples, int seq, int hidden, int bits, int group, int m_bits);
+
 aq_handle* aq_create(int64_t n_samples, int seq, int hidden, int bits, int group) {
+  return create_handle(n_samples, seq, hidden, bits, group, 0);
+}
+
+aq_handle* aq_create_lowbit(int64_t n_samples, int seq, int hidden, int bits, int group, int m_bits) {
+  if (m_bits != 2 && m_bits != 4 && m_bits != 8) {
+    g_create_err[0] = 0;
+    fail(nullptr, AQ_EINVAL, "m_bits must be 2, 4 or 8 (got %d)", m_bits);
+    return nullptr;
+  }
+  return create_handle(n_samples, seq, hidden, bits, group, m_bits);
+}
+
+static aq_handle* create_handle(int64_t n_samples, int seq, int hidden, int bits, int group, int m_bits) {
   g_create_err[0] = 0;
   const int lanes = lanes_for_group(group);
   if (n_samples <= 0 || seq <= 0 || hidden <= 0) { fail(nullptr, AQ_EINVAL, "n_samples, seq and hidden must be positive"); return nullptr; }
@@ -119,14 +134,19 @@ aq_handle* aq_create(int64_t n_samples, int seq, int hidden, int bits, int group
   st.lg_shift = __builtin_ctz((unsigned)lanes);
   cudaError_t e = cudaGetDevice(&h->device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&st.sms, cudaDevAttrMultiProcessorCount, h->device);
-  const size_t m_bytes = (size_t)n_samples * (size_t)st.elems * 2;
+  st.m_bits = m_bits;
+  st.m_bytes = m_bits ? st.elems * m_bits / 8 : st.elems * 2;
+  const size_t m_bytes = (size_t)n_samples * (size_t)st.m_bytes;
+  const size_t m_scale_bytes = m_bits ? (size_t)n_samples * (size_t)st.groups * sizeof(float) : 0;
   const size_t seen_bytes = (size_t)n_samples * sizeof(unsigned long long);
   if (e == cudaSuccess) e = cudaMalloc(&st.m, m_bytes);
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&st.seen), seen_bytes);
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&st.arrivals), sizeof(unsigned long long));
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&st.status), sizeof(uint32_t));
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&h->sum_dev), sizeof(unsigned long long));
+  if (e == cudaSuccess && m_bits) e = cudaMalloc(reinterpret_cast<void**>(&st.m_scales), m_scale_bytes);
   if (e == cudaSuccess) e = cudaMemset(st.m, 0, m_bytes);                      // "initialized to 0"
+  if (e == cudaSuccess && m_bits) e = cudaMemset(st.m_scales, 0, m_scale_bytes);
   if (e == cudaSuccess) e = cudaMemset(st.seen, 0, seen_bytes);
   if (e == cudaSuccess) e = cudaMemset(st.status, 0, sizeof(uint32_t));
   if (e == cudaSuccess) e = cudaMemset(st.arrivals, 0, sizeof(unsigned long long));
@@ -146,6 +166,7 @@ void aq_destroy(aq_handle* h) {
   cudaStreamSynchronize(h->stream);
   free_staging(h);
   cudaFree(h->st.m);
+  cudaFree(h->st.m_scales);
   cudaFree(h->st.seen);
   cudaFree(h->st.arrivals);
   cudaFree(h->st.status);
@@ -203,6 +224,11 @@ int aq_encode(aq_handle* h, const void* act, const int32_t* sample_ids, void* pa
   DeviceGuard g(h->device);
   aq::EncodeArgs a{act, sample_ids, static_cast<uint8_t*>(packed), scales, h->first_flags, h->n_batch,
                    h->rounding == AQ_ROUND_STOCHASTIC, h->seed, h->epoch};
+  if (h->st.m_bits) {
+    if (a.stochastic) return fail(h, AQ_EUNSUPPORTED, "aq_encode: stochastic rounding is not built for the low-precision store");
+    AQ_CUDA(h, aq::launch_encode_lowbit(h->dtype, h->bits, h->st, a, h->stream));
+    return AQ_OK;
+  }
   AQ_CUDA(h, aq::launch_encode(h->dtype, h->bits, h->st, a, h->stream));
   return AQ_OK;
 }
@@ -215,6 +241,10 @@ int aq_decode(aq_handle* h, const void* packed, const float* scales, const int32
     return fail(h, AQ_EINVAL, "aq_decode: packed, scales and out must be 16-byte aligned");
   DeviceGuard g(h->device);
   aq::DecodeArgs a{static_cast<const uint8_t*>(packed), scales, h->raw, sample_ids, out, h->first_flags, h->n_batch};
+  if (h->st.m_bits) {
+    AQ_CUDA(h, aq::launch_decode_lowbit(h->dtype, h->bits, h->st, a, h->stream));
+    return AQ_OK;
+  }
   AQ_CUDA(h, aq::launch_decode(h->dtype, h->bits, h->st, a, h->stream));
   return AQ_OK;
 }
@@ -279,6 +309,10 @@ const char* aq_last_error(aq_handle* h) { return h ? h->err : g_create_err; }
 
 int64_t aq_packed_bytes_per_sample(aq_handle* h) { return h ? h->st.packed_bytes : 0; }
 int64_t aq_scales_per_sample(aq_handle* h) { return h ? h->st.groups : 0; }
+int64_t aq_m_bytes_per_sample(aq_handle* h) {
+  if (!h) return 0;
+  return h->st.m_bytes + (h->st.m_bits ? h->st.groups * (int64_t)sizeof(float) : 0);
+}
 
 int aq_encode_host(aq_handle* h, const void* act_host, const int32_t* sample_ids_host, void* packed_host,
                    float* scales_host) {
@@ -330,10 +364,14 @@ int aq_export_sample(aq_handle* h, int64_t sample_id, void* m_host, uint8_t* see
   if (sample_id < 0 || sample_id >= h->st.n_samples) return fail(h, AQ_EINVAL, "sample id out of range");
   if (!m_host && !seen_host) return fail(h, AQ_EINVAL, "aq_export_sample: null pointers");
   DeviceGuard g(h->device);
-  const size_t bytes = (size_t)h->st.elems * 2;
-  if (m_host)
+  const size_t bytes = (size_t)h->st.m_bytes;
+  if (m_host) {
     AQ_CUDA(h, cudaMemcpyAsync(m_host, static_cast<const char*>(h->st.m) + (size_t)sample_id * bytes, bytes,
                                cudaMemcpyDeviceToHost, h->stream));
+    if (h->st.m_bits)                             // the steps follow the codes
+      AQ_CUDA(h, cudaMemcpyAsync(static_cast<char*>(m_host) + bytes, h->st.m_scales + (size_t)sample_id * h->st.groups,
+                                 (size_t)h->st.groups * sizeof(float), cudaMemcpyDeviceToHost, h->stream));
+  }
   unsigned long long stamp = 0;
   if (seen_host)
     AQ_CUDA(h, cudaMemcpyAsync(&stamp, h->st.seen + sample_id, sizeof(stamp), cudaMemcpyDeviceToHost, h->stream));
@@ -347,10 +385,13 @@ int aq_import_sample(aq_handle* h, int64_t sample_id, const void* m_host, uint8_
   if (sample_id < 0 || sample_id >= h->st.n_samples) return fail(h, AQ_EINVAL, "sample id out of range");
   if (!m_host) return fail(h, AQ_EINVAL, "aq_import_sample: null pointer");
   DeviceGuard g(h->device);
-  const size_t bytes = (size_t)h->st.elems * 2;
+  const size_t bytes = (size_t)h->st.m_bytes;
   const unsigned long long stamp = seen ? aq::kImportedStamp : 0ull;
   AQ_CUDA(h, cudaMemcpyAsync(static_cast<char*>(h->st.m) + (size_t)sample_id * bytes, m_host, bytes,
                              cudaMemcpyHostToDevice, h->stream));
+  if (h->st.m_bits)
+    AQ_CUDA(h, cudaMemcpyAsync(h->st.m_scales + (size_t)sample_id * h->st.groups, static_cast<const char*>(m_host) + bytes,
+                               (size_t)h->st.groups * sizeof(float), cudaMemcpyHostToDevice, h->stream));
   AQ_CUDA(h, cudaMemcpyAsync(h->st.seen + sample_id, &stamp, sizeof(stamp), cudaMemcpyHostToDevice, h->stream));
   AQ_CUDA(h, cudaStreamSynchronize(h->stream));
   return AQ_OK;

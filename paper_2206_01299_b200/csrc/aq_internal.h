@@ -22,7 +22,10 @@ constexpr unsigned long long kCallQuantum = 1ull << 20;
 
 // State of one side of a boundary, as the kernels see it.
 struct State {
-  void* m;                        // T[n_samples][elems]
+  void* m;                        // T[n_samples][elems]; low-precision store: uint8[n_samples][m_bytes] codes
+  float* m_scales;                // low-precision store: float[n_samples][groups] steps of m; else null
+  long long m_bytes;              // low-precision store: bytes of codes per sample (elems * m_bits / 8)
+  int m_bits;                     // 0: m kept in the activation type; 2, 4, 8: low-precision store
   unsigned long long* seen;       // [n_samples] stamps
   unsigned long long* arrivals;   // grows by kCallQuantum per encode / decode launch (starts at 0)
   uint32_t* status;               // sticky AQ_ST_* bits
@@ -61,6 +64,8 @@ struct DecodeArgs {
 
 cudaError_t launch_encode(int dtype, int bits, const State& st, const EncodeArgs& a, cudaStream_t s);
 cudaError_t launch_decode(int dtype, int bits, const State& st, const DecodeArgs& a, cudaStream_t s);
+cudaError_t launch_encode_lowbit(int dtype, int bits, const State& st, const EncodeArgs& a, cudaStream_t s);
+cudaError_t launch_decode_lowbit(int dtype, int bits, const State& st, const DecodeArgs& a, cudaStream_t s);
 cudaError_t launch_quant_grad(int dtype, int bits, int lanes_per_group, const void* grad,
                               long long n_elems, uint8_t* packed, float* scales, bool stochastic,
                               unsigned long long seed, unsigned long long epoch, cudaStream_t s);

@@ -138,6 +138,8 @@ __device__ __forceinline__ uint32_t pack_fields(const uint32_t* tb) {
 //   u + 1.5*2^23 rounded down is 1.5*2^23 + floor(u), whose low mantissa bits are the
 //   two's-complement code.  Clamping u to [-2^(b-1), 2^(b-1) - 1/2] before the floor equals
 //   clamping the integer afterwards.
+// * WIDE = false (differences of two fp16 values: every non-zero one is at least 2^-24 and the
+//   step is far from the ends of the binary32 range) drops two guards that WIDE = true keeps.
 // * The lower clamp is only compiled for the wide type: with |d| <= s and a normal
 //   reciprocal, |d * RN(1/delta)| < 2^(b-1) * (1 + 2^-24), which rounds to at most 2^(b-1).
 // * (k + 1/2) * delta, rounded once, is fma(k, delta, delta/2) whenever delta/2 is exact,
@@ -146,7 +148,7 @@ __device__ __forceinline__ uint32_t pack_fields(const uint32_t* tb) {
 // STOCH (the unbiased quantizer that Theorem 3.1 assumes): delta = s / (2^(b-1) - 1/2), so that
 // the 2^b levels (k + 1/2) * delta reach from -s to +s, and k = floor(d / delta - 1/2 + r) with
 // r uniform in [0,1) from `noise`; both clamps are needed then.
-template <typename T, int BITS, bool STOCH>
+template <int BITS, bool WIDE, bool STOCH>
 __device__ __forceinline__ void quantize8(const float (&d)[8], float s, const uint4& noise, float& delta,
                                           unsigned long long& codes, float (&q)[8]) {
   constexpr float kTwoPow = 1.0f / (float)(1 << (BITS - 1));
@@ -172,12 +174,12 @@ __device__ __forceinline__ void quantize8(const float (&d)[8], float s, const ui
       const float hc = __fsub_rn(__uint_as_float(0x4A800001u | (h << 1)), 4227072.0f);   // h - 32767.5, exact
       u = __fmaf_rn(hc, noise_unit, u);                      // hc * 2^-16 is exact: the same sum, one rounding
     }
-    if constexpr (Conv<T>::kWide || STOCH) u = fmaxf(u, kLo);
+    if constexpr (WIDE || STOCH) u = fmaxf(u, kLo);
     u = fminf(u, kHi);
     const float t = __fadd_rd(u, kMagic);
     tb[j] = __float_as_uint(t);
     const float kf = __fsub_rn(t, kMagic);                   // exact: (float)k
-    if constexpr (Conv<T>::kWide)
+    if constexpr (WIDE)
       q[j] = __fmul_rn(__fadd_rn(kf, 0.5f), delta);          // delta / 2 may be inexact below 2^-125
     else
       q[j] = __fmaf_rn(kf, delta, half_delta);
@@ -453,7 +455,7 @@ __device__ __forceinline__ void encode_rows(const State& st, const EncodeArgs& a
       unsigned long long codes;
       uint4 noise = make_uint4(0, 0, 0, 0);
       if constexpr (STOCH) noise = chunk_noise(a.seed, a.epoch, stream_id, (uint32_t)c);
-      quantize8<T, BITS, STOCH>(d, s, noise, delta, codes, q);
+      quantize8<BITS, Conv<T>::kWide, STOCH>(d, s, noise, delta, codes, q);
 #pragma unroll
       for (int j = 0; j < 8; ++j) mf[j] = __fadd_rn(mf[j], q[j]);
       if (active) {
@@ -608,6 +610,100 @@ __global__ void __launch_bounds__(kThreads, decode_ctas_per_sm<BITS>()) decode_k
   }
 }
 
+// ------------------------------------------------------------------ previous messages kept in MBITS bits per element
+//
+// The store holds Q(m) instead of m: MBITS-bit codes in the messages' bitstream layout plus one
+// fp32 step per group, and every visit works on the dequantized store (the paper's "mz"
+// ablation; reading: the same Q as for the messages):
+//   m_deq = (km + 1/2) * Delta_m;  sender: Delta_msg = Q_b(a - m_deq);  m_new = m_deq + Delta_msg
+//   (fp32);  store <- Q_z(m_new);  the receiver's activation is T(m_new).
+// A first visit is the same pass with m_deq = 0 and the activation (the raw message) as the
+// update, so both branches end in the same re-quantization.  Differences against an fp32 store
+// are not differences of two 16-bit values, hence the guarded (WIDE) quantizer arithmetic.
+
+template <typename T, int BITS, int MBITS, bool SENDER>
+__global__ void __launch_bounds__(kThreads, 4)
+    lowbit_kernel(const State st, const EncodeArgs ea, const DecodeArgs da, const LaunchPlan plan) {
+  const int tid = threadIdx.x;
+  const int lane = tid & 31;
+  const int y = blockIdx.y;
+  overlap_with_neighbours();
+  const Sample sample = SENDER ? open_sample(st, plan, ea.ids, y, false, false, ea.first_flags)
+                               : open_sample(st, plan, da.ids, y, true, da.raw != nullptr, da.first_flags);
+  const int mode = sample.mode;
+  const unsigned elems = (unsigned)st.elems;
+  const unsigned long long row = (unsigned long long)(unsigned)y;
+  const T* in = SENDER ? reinterpret_cast<const T*>(ea.act) + row * elems
+                       : (mode == kModeFirst ? reinterpret_cast<const T*>(da.raw) + row * elems : nullptr);
+  uint8_t* wire_w = SENDER ? ea.packed + row * (unsigned)st.packed_bytes : nullptr;
+  float* scale_w = SENDER ? ea.scales + row * (unsigned)st.groups : nullptr;
+  const uint8_t* wire_r = SENDER ? nullptr : da.packed + row * (unsigned)st.packed_bytes;
+  const float* scale_r = SENDER ? nullptr : da.scales + row * (unsigned)st.groups;
+  T* out = SENDER ? nullptr : reinterpret_cast<T*>(da.out) + row * elems;
+  const bool words_ok = (st.packed_bytes & 3) == 0;
+  const bool touch = mode != kModeSkip;
+  const unsigned long long sid = touch ? (unsigned long long)(unsigned)sample.id : 0ull;
+  uint8_t* m_codes = static_cast<uint8_t*>(st.m) + sid * (unsigned long long)st.m_bytes;
+  float* m_scales = st.m_scales + sid * (unsigned)st.groups;
+  const uint4 no_noise = make_uint4(0, 0, 0, 0);
+
+  const int r_end = min(st.rows, (int)(blockIdx.x + 1) * plan.rows_per_cta);
+  for (int r = blockIdx.x * plan.rows_per_cta; r < r_end; ++r) {
+    const int c = r * kThreads + tid;
+    const bool active = c < st.chunks;
+    const bool whole_warp = c - lane + 32 <= st.chunks;
+    const int g = c >> st.lg_shift;
+    float m_new[8];
+    unsigned long long codes = 0ull;
+    float delta = 0.0f;
+    if (mode == kModeDelta) {                                   // uniform over the CTA
+      unsigned long long km = 0ull, kw = 0ull;
+      float dm = 0.0f;
+      uint4 av = make_uint4(0, 0, 0, 0);
+      if (active) {
+        dm = m_scales[g];
+        if (SENDER) av = ld_stream(in + (unsigned)c * (unsigned)kChunk);
+        else delta = __ldg(scale_r + g);
+      }
+      km = load_codes<MBITS>(m_codes, c, lane, active, false);
+      if (!SENDER) kw = load_codes<BITS>(wire_r, c, lane, active, words_ok && whole_warp);
+      float m_deq[8], q[8];
+      dequantize8<MBITS>(km, dm, m_deq);
+      if (SENDER) {
+        float af[8], d[8];
+        Conv<T>::unpack(av, af);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) d[j] = __fsub_rn(af[j], m_deq[j]);
+        const float s = group_max<0>(abs_max8(d), st.lanes_per_group);
+        quantize8<BITS, true, false>(d, s, no_noise, delta, codes, q);
+      } else {
+        dequantize8<BITS>(kw, delta, q);
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j) m_new[j] = __fadd_rn(m_deq[j], q[j]);
+    } else {
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (mode == kModeFirst && active) v = ld_stream(in + (unsigned)c * (unsigned)kChunk);
+      Conv<T>::unpack(v, m_new);
+    }
+    // store <- Q_z(m_new)
+    {
+      const float s2 = group_max<0>(abs_max8(m_new), st.lanes_per_group);
+      unsigned long long km2;
+      float dm2, unused[8];
+      quantize8<MBITS, true, false>(m_new, s2, no_noise, dm2, km2, unused);
+      store_codes<MBITS>(m_codes, c, lane, active && touch, false, km2);
+      if (active && touch && (lane & (st.lanes_per_group - 1)) == 0) m_scales[g] = dm2;
+    }
+    if (SENDER) {
+      store_codes<BITS>(wire_w, c, lane, active, words_ok && whole_warp, codes);
+      if (active && (lane & (st.lanes_per_group - 1)) == 0) scale_w[g] = delta;
+    } else if (active) {
+      st_stream(out + (unsigned)c * (unsigned)kChunk, Conv<T>::pack(m_new));     // zeros for a skipped sample
+    }
+  }
+}
+
 // ------------------------------------------------------------------ backward direction: direct quantization
 
 template <typename T, int BITS, int LPG, bool STOCH>
@@ -636,7 +732,7 @@ __global__ void __launch_bounds__(kThreads) quant_grad_kernel(const T* __restric
     unsigned long long codes;
     uint4 noise = make_uint4(0, 0, 0, 0);
     if constexpr (STOCH) noise = chunk_noise(seed, epoch, 0xFFFFFFFFu, (uint32_t)c);
-    quantize8<T, BITS, STOCH>(d, s, noise, delta, codes, q);
+    quantize8<BITS, Conv<T>::kWide, STOCH>(d, s, noise, delta, codes, q);
     if (active && (lane & (lanes_per_group - 1)) == 0) scales[c >> lg_shift] = delta;
     store_codes<BITS>(packed, c, lane, active, c - lane + 32 <= n_chunks, codes);
   }
@@ -690,6 +786,29 @@ __global__ void __launch_bounds__(kThreads) checksum_kernel(const State st, unsi
     acc += mix64(i, w.x) + mix64(i + 1, w.y) + mix64(i + 2, w.z) + mix64(i + 3, w.w);
   }
   for (long long x = (long long)blockIdx.x * kThreads + threadIdx.x; x < st.n_samples; x += stride)
+    acc += mix64((1ull << 40) + (unsigned long long)x, st.seen[x] != 0ull ? 1ull : 0ull);
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(kFullMask, acc, o);
+  __shared__ unsigned long long part[kThreads / 32];
+  if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned long long t = 0ull;
+    for (int w = 0; w < kThreads / 32; ++w) t += part[w];
+    atomicAdd(sum_out, t);
+  }
+}
+
+__global__ void __launch_bounds__(kThreads) checksum_lowbit_kernel(const State st, unsigned long long* sum_out) {
+  const long long n_code_words = st.n_samples * st.m_bytes / 4;      // the code bytes of all samples as one array
+  const long long n_scale_words = st.n_samples * st.groups;
+  const uint32_t* cw = static_cast<const uint32_t*>(st.m);
+  const uint32_t* sw = reinterpret_cast<const uint32_t*>(st.m_scales);
+  const long long stride = (long long)gridDim.x * kThreads;
+  const long long first = (long long)blockIdx.x * kThreads + threadIdx.x;
+  unsigned long long acc = 0ull;
+  for (long long i = first; i < n_code_words; i += stride) acc += mix64((unsigned long long)i, cw[i]);
+  for (long long i = first; i < n_scale_words; i += stride) acc += mix64((unsigned long long)(n_code_words + i), sw[i]);
+  for (long long x = first; x < st.n_samples; x += stride)
     acc += mix64((1ull << 40) + (unsigned long long)x, st.seen[x] != 0ull ? 1ull : 0ull);
   for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(kFullMask, acc, o);
   __shared__ unsigned long long part[kThreads / 32];
@@ -807,6 +926,53 @@ cudaError_t launch_decode(int dtype, int bits, const State& st, const DecodeArgs
   return cudaErrorInvalidValue;
 }
 
+// one launch shape for both directions of the low-precision store
+template <typename K>
+cudaError_t launch_lowbit(K kernel, const State& st, const EncodeArgs& ea, const DecodeArgs& da, int n_batch,
+                          cudaStream_t s) {
+  if (n_batch <= 0) return cudaSuccess;
+  long long per = st.rows_per_cta > 0 ? st.rows_per_cta : kRowsPerCta;
+  if (per > st.rows) per = st.rows;
+  long long gx = (st.rows + per - 1) / per;
+  if (gx * n_batch > (long long)kCallQuantum) {
+    gx = (long long)kCallQuantum / n_batch;
+    per = (st.rows + gx - 1) / gx;
+    gx = (st.rows + per - 1) / per;
+  }
+  const unsigned long long ctas = (unsigned long long)gx * (unsigned long long)n_batch;
+  LaunchPlan plan;
+  plan.rows_per_cta = (int)per;
+  plan.share = (unsigned)(kCallQuantum / ctas);
+  plan.first_share = (unsigned)(kCallQuantum - (unsigned long long)plan.share * (ctas - 1ull));
+  return launch_overlapped(kernel, dim3((unsigned)gx, (unsigned)n_batch), s, st, ea, da, plan);
+}
+
+#define AQ_DISPATCH_MBITS(T, B, SENDER)                                                             \
+  switch (st.m_bits) {                                                                              \
+    case 2: return launch_lowbit(lowbit_kernel<T, B, 2, SENDER>, st, ea, da, n_batch, s);           \
+    case 4: return launch_lowbit(lowbit_kernel<T, B, 4, SENDER>, st, ea, da, n_batch, s);           \
+    case 8: return launch_lowbit(lowbit_kernel<T, B, 8, SENDER>, st, ea, da, n_batch, s);           \
+    default: return cudaErrorInvalidValue;                                                          \
+  }
+
+cudaError_t launch_encode_lowbit(int dtype, int bits, const State& st, const EncodeArgs& ea, cudaStream_t s) {
+  const DecodeArgs da{};
+  const int n_batch = ea.n_batch;
+#define AQ_CALL(T, B) AQ_DISPATCH_MBITS(T, B, true)
+  AQ_DISPATCH(dtype, bits, AQ_CALL)
+#undef AQ_CALL
+  return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_decode_lowbit(int dtype, int bits, const State& st, const DecodeArgs& da, cudaStream_t s) {
+  const EncodeArgs ea{};
+  const int n_batch = da.n_batch;
+#define AQ_CALL(T, B) AQ_DISPATCH_MBITS(T, B, false)
+  AQ_DISPATCH(dtype, bits, AQ_CALL)
+#undef AQ_CALL
+  return cudaErrorInvalidValue;
+}
+
 cudaError_t launch_quant_grad(int dtype, int bits, int lanes_per_group, const void* grad, long long n_elems,
                               uint8_t* packed, float* scales, bool stochastic, unsigned long long seed,
                               unsigned long long epoch, cudaStream_t s) {
@@ -845,6 +1011,13 @@ cudaError_t launch_dequant_grad(int dtype, int bits, int lanes_per_group, const 
 }
 
 cudaError_t launch_checksum(const State& st, unsigned long long* sum_dev, cudaStream_t s) {
+  if (st.m_bits) {
+    const long long words = st.n_samples * st.m_bytes / 4;
+    long long want = (words + kThreads - 1) / kThreads;
+    const long long cap = (long long)st.sms * 8;
+    checksum_lowbit_kernel<<<(unsigned)(want < 1 ? 1 : (want > cap ? cap : want)), kThreads, 0, s>>>(st, sum_dev);
+    return cudaGetLastError();
+  }
   const long long n_vec = st.n_samples * (long long)st.chunks;
   long long want = (n_vec + kThreads - 1) / kThreads;
   const long long cap = (long long)st.sms * 8;

@@ -1,0 +1,151 @@
+"""The low-precision store of previous messages (aq_create_lowbit: m kept in 2, 4 or 8 bits per
+element) against the CPU oracle, element by element, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2206_01299_b200 as aq
+from paper_2206_01299_b200 import synth
+from codec_harness import DT, bits16
+
+pytestmark = pytest.mark.gpu
+
+
+class LowSide:
+    def __init__(self, cfg, n_batch, m_bits):
+        self.cfg, self.m_bits = cfg, m_bits
+        self.h = aq.aq_create_lowbit(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, m_bits)
+        aq.aq_configure(self.h, aq.AQ_DTYPE, DT[cfg.dtype][0])
+        aq.aq_configure(self.h, aq.AQ_BATCH, n_batch)
+        self.first = torch.zeros(n_batch, dtype=torch.uint8, device="cuda")
+        aq.aq_configure(self.h, aq.AQ_FIRST_FLAGS, self.first)
+        self.code_bytes = cfg.elems * m_bits // 8
+        assert aq.aq_m_bytes_per_sample(self.h) == self.code_bytes + cfg.groups * 4
+
+    def close(self):
+        aq.aq_destroy(self.h)
+
+    def state(self):
+        """(codes uint8[n, code_bytes], steps float32[n, groups], seen uint8[n])"""
+        n = self.cfg.n_samples
+        codes = np.empty((n, self.code_bytes), np.uint8)
+        steps = np.empty((n, self.cfg.groups), np.float32)
+        seen = np.empty(n, np.uint8)
+        buf = np.empty(self.code_bytes + self.cfg.groups * 4, np.uint8)
+        for i in range(n):
+            seen[i] = aq.aq_export_sample(self.h, i, buf)
+            codes[i] = buf[:self.code_bytes]
+            steps[i] = buf[self.code_bytes:].view(np.float32)
+        return codes, steps, seen
+
+
+def run_lowbit(cfg, m_bits, n_batch=None):
+    nb = n_batch or cfg.n_batch
+    gs, gr = LowSide(cfg, nb, m_bits), LowSide(cfg, nb, m_bits)
+    od = DT[cfg.dtype][1]
+    os_, or_ = (oracle.SideLow(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, od, m_bits) for _ in range(2))
+    packed = torch.empty((nb, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
+    scales = torch.empty((nb, cfg.groups), dtype=torch.float32, device="cuda")
+    out = torch.empty((nb, cfg.seq, cfg.hidden), dtype=cfg.torch_dtype, device="cuda")
+    try:
+        for epoch in range(cfg.epochs):
+            order = synth.epoch_order(cfg, epoch)
+            for c in range(cfg.n_samples // nb):
+                ids = order[c * nb:(c + 1) * nb].contiguous()
+                act = synth.activation(cfg, ids, epoch, device="cuda")
+                packed.fill_(0xAB)
+                scales.fill_(-7.0)
+                out.fill_(3.0)
+                aq.aq_encode(gs.h, act, ids.cuda(), packed, scales)
+                aq.aq_configure(gr.h, aq.AQ_RAW, act)
+                aq.aq_decode(gr.h, packed, scales, ids.cuda(), out)
+                torch.cuda.synchronize()
+                a_np = bits16(act)
+                p_o, s_o, f_o = os_.encode(a_np, ids.numpy())
+                out_o, fr_o = or_.decode(p_o, s_o, ids.numpy(), raw=a_np)
+                assert np.array_equal(packed.cpu().numpy(), p_o), (epoch, c, "packed")
+                assert np.array_equal(scales.cpu().numpy().view(np.uint32), s_o.view(np.uint32)), (epoch, c, "scales")
+                assert np.array_equal(gs.first.cpu().numpy(), f_o) and np.array_equal(gr.first.cpu().numpy(), fr_o)
+                assert np.array_equal(bits16(out), out_o), (epoch, c, "out")
+            for g_side, o_side in ((gs, os_), (gr, or_)):
+                codes, steps, seen = g_side.state()
+                assert np.array_equal(codes, o_side.m_codes()), (epoch, "stored codes")
+                assert np.array_equal(steps.view(np.uint32), o_side.m_scales().view(np.uint32)), (epoch, "stored steps")
+                assert np.array_equal(seen, o_side.seen())
+            assert aq.aq_state_checksum(gs.h) == aq.aq_state_checksum(gr.h) == os_.checksum() == or_.checksum()
+            assert aq.aq_status(gs.h) == 0 and aq.aq_status(gr.h) == 0
+    finally:
+        gs.close()
+        gr.close()
+        os_.close()
+        or_.close()
+
+
+@pytest.mark.parametrize("m_bits", [2, 4, 8])
+def test_tiny_boundary_with_a_low_precision_store(m_bits):
+    run_lowbit(synth.TINY, m_bits)
+
+
+@pytest.mark.parametrize("m_bits", [2, 8])
+def test_large_shapes_reduced_id_space(m_bits):
+    run_lowbit(synth.shrink(synth.GPT2_XL, 8, seq=96, epochs=3), m_bits, n_batch=4)
+    run_lowbit(synth.shrink(synth.DEBERTA_XXL, 16, seq=40), m_bits)
+    run_lowbit(synth.shrink(synth.SWEEP_FWD, 4, seq=64), m_bits)
+
+
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+@pytest.mark.parametrize("bits", range(1, 9))
+def test_every_message_width_on_ragged_shapes(dtype, bits):
+    m_bits = (2, 4, 8)[bits % 3]
+    cfg = synth.Boundary("low-ragged", 6, 3, 37, 136, dtype, bits, 8, 3, "outlier", 0.3, seed=120 + bits)
+    run_lowbit(cfg, m_bits)
+    cfg = synth.Boundary("low-groups", 4, 2, 3, 1024, dtype, bits, 256, 3, "student_t3", 0.2, seed=140 + bits)
+    run_lowbit(cfg, m_bits)
+    cfg = synth.Boundary("low-one-chunk", 4, 2, 1, 8, dtype, bits, 8, 3, "normal", 0.5, seed=160 + bits)
+    run_lowbit(cfg, m_bits)
+
+
+def test_bad_ids_import_export_and_unsupported_calls():
+    cfg = synth.Boundary("low-err", 5, 4, 2, 64, "fp16", 2, 64, 1, "normal", 0.1, seed=5)
+    gs, gr = LowSide(cfg, 4, 8), LowSide(cfg, 4, 8)
+    os_, or_ = (oracle.SideLow(5, 2, 64, 2, 64, oracle.FP16, 8) for _ in range(2))
+    try:
+        packed = torch.empty((4, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
+        scales = torch.empty((4, cfg.groups), dtype=torch.float32, device="cuda")
+        out = torch.empty((4, 2, 64), dtype=torch.float16, device="cuda")
+        for step, id_list in enumerate([[1, 7, 1, 3], [3, -1, 1, 3], [0, 1, 2, 3]]):
+            ids = torch.tensor(id_list, dtype=torch.int32)
+            act = synth.activation(cfg, torch.tensor([10, 11, 12, 13]), step, device="cuda")
+            aq.aq_encode(gs.h, act, ids.cuda(), packed, scales)
+            raw = act if step != 2 else None
+            aq.aq_configure(gr.h, aq.AQ_RAW, raw)
+            aq.aq_decode(gr.h, packed, scales, ids.cuda(), out)
+            torch.cuda.synchronize()
+            p_o, s_o, _ = os_.encode(bits16(act), ids.numpy())
+            out_o, _ = or_.decode(p_o, s_o, ids.numpy(), raw=bits16(act) if raw is not None else None)
+            assert np.array_equal(packed.cpu().numpy(), p_o) and np.array_equal(scales.cpu().numpy(), s_o)
+            assert np.array_equal(bits16(out), out_o)
+            assert aq.aq_status(gs.h) == os_.status() and aq.aq_status(gr.h) == or_.status()
+            assert aq.aq_state_checksum(gs.h) == os_.checksum() and aq.aq_state_checksum(gr.h) == or_.checksum()
+        # checkpoint: export every sample of one handle into a fresh one
+        fresh = LowSide(cfg, 4, 8)
+        buf = np.empty(aq.aq_m_bytes_per_sample(gs.h), np.uint8)
+        for i in range(cfg.n_samples):
+            seen = aq.aq_export_sample(gs.h, i, buf)
+            aq.aq_import_sample(fresh.h, i, buf, seen)
+        assert aq.aq_state_checksum(fresh.h) == aq.aq_state_checksum(gs.h)
+        fresh.close()
+        # what is not built for this store says so
+        aq.aq_configure(gs.h, aq.AQ_ROUNDING, aq.AQ_ROUND_STOCHASTIC)
+        with pytest.raises(aq.AqError) as e:
+            aq.aq_encode(gs.h, act, ids.cuda(), packed, scales)
+        assert e.value.code == aq.AQ_EUNSUPPORTED
+        with pytest.raises(aq.AqError) as e:
+            aq.aq_state_checksum_noalloc(gs.h)
+        assert e.value.code == aq.AQ_EUNSUPPORTED
+        with pytest.raises(aq.AqError):
+            aq.aq_create_lowbit(4, 2, 64, 4, 64, 3)
+    finally:
+        gs.close()
+        gr.close()
