@@ -32,6 +32,7 @@ constexpr int kChunksPerThread = 2;                      // grad kernels: chunks
 constexpr int kChunksPerCta = kThreads * kChunksPerThread;
 
 enum { kModeDelta = 0, kModeFirst = 1, kModeSkip = 2 };
+enum { kStBadId = 1, kStDupId = 2, kStNoRaw = 4 };
 
 // What the launch layer decides for one encode / decode launch.
 struct LaunchPlan {
@@ -39,7 +40,6 @@ struct LaunchPlan {
   unsigned share;          // what a CTA adds to the arrival counter ...
   unsigned first_share;    // ... and what CTA (0,0) adds, so that the grid adds kCallQuantum in all
 };
-enum { kStBadId = 1, kStDupId = 2, kStNoRaw = 4 };
 
 // ------------------------------------------------------------------ 16-bit types
 

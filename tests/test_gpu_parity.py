@@ -367,3 +367,90 @@ def test_stochastic_gradient_quantization_matches_oracle(dtype, bits):
         assert not np.array_equal(seen[0], seen[1])
     finally:
         aq.aq_destroy(h)
+
+
+# ----------------------------------------------------------------- limits, overrides and random configurations
+
+def test_largest_batch_of_small_samples():
+    """4096 samples in one call (the limit of AQ_BATCH), ids in random order with one repeat and
+    one out of range: grid of 4096 samples, the repeat check scans up to 4095 earlier ids."""
+    cfg = synth.Boundary("wide", 4096, 4096, 1, 64, "fp16", 4, 64, 2, "normal", 0.1, seed=201)
+    gs, gr = GpuSide(cfg, 4096), GpuSide(cfg, 4096)
+    os_, or_ = (oracle.Side(4096, 1, 64, 4, 64, oracle.FP16) for _ in range(2))
+    try:
+        packed = torch.empty((4096, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
+        scales = torch.empty((4096, cfg.groups), dtype=torch.float32, device="cuda")
+        out = torch.empty((4096, 1, 64), dtype=torch.float16, device="cuda")
+        for epoch in range(3):
+            ids = synth.epoch_order(cfg, epoch).clone()
+            ids[4000] = ids[17]                       # a repeat far into the call
+            ids[123] = 5000                           # out of range
+            act = synth.activation(cfg, torch.arange(4096), epoch, device="cuda")
+            aq.aq_encode(gs.h, act, ids.cuda(), packed, scales)
+            aq.aq_configure(gr.h, aq.AQ_RAW, act)
+            aq.aq_decode(gr.h, packed, scales, ids.cuda(), out)
+            torch.cuda.synchronize()
+            p_o, s_o, f_o = os_.encode(bits16(act), ids.numpy())
+            out_o, fr_o = or_.decode(p_o, s_o, ids.numpy(), raw=bits16(act))
+            assert np.array_equal(packed.cpu().numpy(), p_o) and np.array_equal(scales.cpu().numpy(), s_o)
+            assert np.array_equal(bits16(out), out_o)
+            assert np.array_equal(gs.first.cpu().numpy(), f_o) and np.array_equal(gr.first.cpu().numpy(), fr_o)
+            assert aq.aq_status(gs.h) == os_.status() == (aq.AQ_ST_BAD_ID | aq.AQ_ST_DUP_ID)
+            assert aq.aq_status(gr.h) == or_.status()
+            assert aq.aq_state_checksum(gs.h) == aq.aq_state_checksum(gr.h) == os_.checksum() == or_.checksum()
+        with pytest.raises(aq.AqError):
+            aq.aq_configure(gs.h, aq.AQ_BATCH, 4097)
+    finally:
+        gs.close()
+        gr.close()
+
+
+def test_one_large_sample():
+    """A single sequence of 2^24 elements (32 MB): 8192 rows, far more CTAs per sample than any workload."""
+    cfg = synth.Boundary("long", 2, 1, 8192, 2048, "bf16", 3, 128, 2, "normal", 0.05, seed=202)
+    run_boundary(cfg, check_all_m=True)
+
+
+@pytest.mark.parametrize("rows_per_cta", [1, 3, 7, 1 << 20])
+def test_rows_per_cta_override_does_not_change_results(rows_per_cta):
+    cfg = synth.Boundary("rows", 4, 2, 21, 1000, "fp16", 4, 8, 2, "outlier", 0.2, seed=203)   # 2625 chunks: 11 rows, ragged
+    gs, gr = GpuSide(cfg, 2), GpuSide(cfg, 2)
+    os_, or_ = (oracle.Side(4, 21, 1000, 4, 8, oracle.FP16) for _ in range(2))
+    try:
+        for h in (gs.h, gr.h):
+            aq.aq_configure(h, aq.AQ_ROWS_PER_CTA, rows_per_cta)
+        packed = torch.empty((2, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
+        scales = torch.empty((2, cfg.groups), dtype=torch.float32, device="cuda")
+        out = torch.empty((2, 21, 1000), dtype=torch.float16, device="cuda")
+        for epoch in range(3):
+            ids = torch.tensor([3, 1], dtype=torch.int32)
+            act = synth.activation(cfg, ids, epoch, device="cuda")
+            aq.aq_encode(gs.h, act, ids.cuda(), packed, scales)
+            aq.aq_configure(gr.h, aq.AQ_RAW, act)
+            aq.aq_decode(gr.h, packed, scales, ids.cuda(), out)
+            torch.cuda.synchronize()
+            p_o, s_o, _ = os_.encode(bits16(act), ids.numpy())
+            out_o, _ = or_.decode(p_o, s_o, ids.numpy(), raw=bits16(act))
+            assert np.array_equal(packed.cpu().numpy(), p_o) and np.array_equal(scales.cpu().numpy(), s_o)
+            assert np.array_equal(bits16(out), out_o)
+        assert aq.aq_state_checksum(gs.h) == os_.checksum() and aq.aq_state_checksum(gr.h) == or_.checksum()
+    finally:
+        gs.close()
+        gr.close()
+
+
+def test_random_configurations():
+    """Seeded random shapes, widths, groups, types, batch sizes and rounding modes."""
+    rng = np.random.default_rng(2206)
+    for trial in range(24):
+        group = int(rng.choice([8, 16, 32, 64, 128, 256]))
+        hidden = group * int(rng.integers(1, 9))
+        seq = int(rng.integers(1, 70))
+        bits = int(rng.integers(1, 9))
+        nb = int(rng.choice([1, 2, 3, 5]))
+        n_samples = nb * int(rng.integers(1, 4))
+        dtype = str(rng.choice(["fp16", "bf16"]))
+        kind = str(rng.choice(["normal", "outlier", "student_t3"]))
+        cfg = synth.Boundary(f"rnd{trial}", n_samples, nb, seq, hidden, dtype, bits, group, 3, kind,
+                             float(rng.choice([0.0, 0.01, 0.5])), seed=300 + trial)
+        run_boundary(cfg, stochastic_seed=(int(rng.integers(1 << 40)) if trial % 3 == 0 else None))
