@@ -55,6 +55,7 @@ def parse_args():
                     help="quantizer of the sender: interval number (default) or unbiased stochastic rounding")
     ap.add_argument("--m-bits", type=int, default=0, choices=[0, 2, 4, 8],
                     help="keep the previous messages in this many bits per element (0 = the activation type)")
+    ap.add_argument("--hosted", action="store_true", help="keep m in page-locked host memory (aq_create_hosted)")
     ap.add_argument("--rows-per-cta", type=int, default=0, help="AQ_ROWS_PER_CTA of both handles (0 = library default)")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--skip-e2e", action="store_true")
@@ -275,6 +276,7 @@ def main():
     handles = []
     for _ in range(2):
         h = (aq.aq_create_lowbit(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, args.m_bits) if args.m_bits
+             else aq.aq_create_hosted(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group) if args.hosted
              else aq.aq_create(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group))
         aq.aq_configure(h, aq.AQ_DTYPE, aq.AQ_FP16 if cfg.dtype == "fp16" else aq.AQ_BF16)
         aq.aq_configure(h, aq.AQ_BATCH, nb)
@@ -465,7 +467,7 @@ def main():
     enc_gbs = launch_bytes / (enc_ms * 1e-3) / 1e9
     dec_gbs = launch_bytes / (dec_ms * 1e-3) / 1e9
     traffic = NCU_TRAFFIC_BYTES_PER_ELEMENT["encode"] if (args.workload == NCU_TRAFFIC_WORKLOAD and args.rounding == "interval"
-                                                          and not args.m_bits) else None
+                                                          and not args.m_bits and not args.hosted) else None
     value = replicas.whole_job_rate(args.steps * step_bytes, world, elapsed_ms) / 1e9
     line = {
         "metric": "activation encode+decode GB/s", "value": value, "unit": "GB/s",
@@ -474,6 +476,7 @@ def main():
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": label, "hidden": cfg.hidden, "seq": cfg.seq,
                    "micro_batch": cfg.n_batch, "sequences_per_step": MACRO, "sequences_per_launch": nb, "cuda_graph": bool(args.graph), "rounding": args.rounding, "m_bits": args.m_bits or 16,
+                   "m_in": "host memory (page-locked, mapped)" if args.hosted else "HBM",
                    "act_dtype": cfg.dtype, "bits": cfg.bits, "group": cfg.group, "n_samples_per_side": cfg.n_samples,
                    "m_bytes_per_side": cfg.n_samples * (cfg.elems * 2 if not args.m_bits else cfg.elems * args.m_bits // 8 + cfg.groups * 4), "steady_epochs_resident": n_arenas,
                    "l2": f"inputs larger than L2 (each step touches {int(MACRO * cfg.elems * 6 / 1e6)} MB of fresh HBM; no flush needed)",

@@ -119,6 +119,17 @@ enum {
 aq_handle* aq_create(int64_t n_samples, int seq, int hidden, int bits, int group);
 
 /*
+ * The same, with m in page-locked host memory instead of device memory (Section 3.3: the
+ * previous messages can live in host memory; the appendix on offloading measures no loss of
+ * throughput).  The GPU addresses that memory directly, so aq_encode / aq_decode and every other
+ * call work unchanged and give the same results; they then run at the speed of the host link
+ * (each element of m crosses it once in each direction) and the state is bounded by host
+ * memory, not by the 180 GB of the GPU.  Run such a handle on its own stream beside the stage's
+ * compute, as the paper hides the transfers behind the forward pass.
+ */
+aq_handle* aq_create_hosted(int64_t n_samples, int seq, int hidden, int bits, int group);
+
+/*
  * The same, with the previous messages kept at low precision (appendix "Number of Bits for
  * Previous Messages": mz = z bits for m).  m is stored as m_bits-bit codes (2, 4 or 8) plus one
  * fp32 step per group of `group` elements -- Q of this file applied to m -- and takes

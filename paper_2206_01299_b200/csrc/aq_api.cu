@@ -21,6 +21,7 @@ struct aq_handle {
   const void* raw = nullptr;
   uint8_t* first_flags = nullptr;
   unsigned long long* sum_dev = nullptr;     // scratch of aq_state_checksum
+  void* m_host = nullptr;                    // hosted store: the pinned host block that st.m maps
   // staging for the host-buffer entry points, sized for staged_batch samples
   int staged_batch = 0;
   void* d_act = nullptr;      // also raw / out
@@ -96,10 +97,15 @@ int ensure_staging(aq_handle* h) {
 
 extern "C" {
 
-static aq_handle* create_handle(int64_t n_samples, int seq, int hidden, int bits, int group, int m_bits);
+static aq_handle* create_handle(int64_t n_samples, int seq, int hidden, int bits, int group, int m_bits,
+                                bool hosted = false);
 
 aq_handle* aq_create(int64_t n_samples, int seq, int hidden, int bits, int group) {
   return create_handle(n_samples, seq, hidden, bits, group, 0);
+}
+
+aq_handle* aq_create_hosted(int64_t n_samples, int seq, int hidden, int bits, int group) {
+  return create_handle(n_samples, seq, hidden, bits, group, 0, true);
 }
 
 aq_handle* aq_create_lowbit(int64_t n_samples, int seq, int hidden, int bits, int group, int m_bits) {
@@ -111,7 +117,8 @@ aq_handle* aq_create_lowbit(int64_t n_samples, int seq, int hidden, int bits, in
   return create_handle(n_samples, seq, hidden, bits, group, m_bits);
 }
 
-static aq_handle* create_handle(int64_t n_samples, int seq, int hidden, int bits, int group, int m_bits) {
+static aq_handle* create_handle(int64_t n_samples, int seq, int hidden, int bits, int group, int m_bits,
+                                bool hosted) {
   g_create_err[0] = 0;
   const int lanes = lanes_for_group(group);
   if (n_samples <= 0 || seq <= 0 || hidden <= 0) { fail(nullptr, AQ_EINVAL, "n_samples, seq and hidden must be positive"); return nullptr; }
@@ -139,13 +146,19 @@ static aq_handle* create_handle(int64_t n_samples, int seq, int hidden, int bits
   const size_t m_bytes = (size_t)n_samples * (size_t)st.m_bytes;
   const size_t m_scale_bytes = m_bits ? (size_t)n_samples * (size_t)st.groups * sizeof(float) : 0;
   const size_t seen_bytes = (size_t)n_samples * sizeof(unsigned long long);
-  if (e == cudaSuccess) e = cudaMalloc(&st.m, m_bytes);
+  if (e == cudaSuccess && !hosted) e = cudaMalloc(&st.m, m_bytes);
+  if (e == cudaSuccess && hosted) {
+    // page-locked host memory that the GPU addresses directly: the kernels stream m over the bus
+    e = cudaHostAlloc(&h->m_host, m_bytes, cudaHostAllocMapped | cudaHostAllocPortable);
+    if (e == cudaSuccess) e = cudaHostGetDevicePointer(&st.m, h->m_host, 0);
+  }
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&st.seen), seen_bytes);
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&st.arrivals), sizeof(unsigned long long));
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&st.status), sizeof(uint32_t));
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&h->sum_dev), sizeof(unsigned long long));
   if (e == cudaSuccess && m_bits) e = cudaMalloc(reinterpret_cast<void**>(&st.m_scales), m_scale_bytes);
-  if (e == cudaSuccess) e = cudaMemset(st.m, 0, m_bytes);                      // "initialized to 0"
+  if (e == cudaSuccess && !hosted) e = cudaMemset(st.m, 0, m_bytes);           // "initialized to 0"
+  if (e == cudaSuccess && hosted) memset(h->m_host, 0, m_bytes);
   if (e == cudaSuccess && m_bits) e = cudaMemset(st.m_scales, 0, m_scale_bytes);
   if (e == cudaSuccess) e = cudaMemset(st.seen, 0, seen_bytes);
   if (e == cudaSuccess) e = cudaMemset(st.status, 0, sizeof(uint32_t));
@@ -165,7 +178,8 @@ void aq_destroy(aq_handle* h) {
   DeviceGuard g(h->device);
   cudaStreamSynchronize(h->stream);
   free_staging(h);
-  cudaFree(h->st.m);
+  if (h->m_host) cudaFreeHost(h->m_host);
+  else cudaFree(h->st.m);
   cudaFree(h->st.m_scales);
   cudaFree(h->st.seen);
   cudaFree(h->st.arrivals);

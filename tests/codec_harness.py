@@ -16,9 +16,10 @@ def bits16(t: torch.Tensor) -> np.ndarray:
 
 
 class GpuSide:
-    def __init__(self, cfg, n_batch, stream=None):
+    def __init__(self, cfg, n_batch, stream=None, hosted=False):
         self.cfg = cfg
-        self.h = aq.aq_create(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group)
+        create = aq.aq_create_hosted if hosted else aq.aq_create
+        self.h = create(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group)
         aq.aq_configure(self.h, aq.AQ_DTYPE, DT[cfg.dtype][0])
         aq.aq_configure(self.h, aq.AQ_BATCH, n_batch)
         if stream is not None:
@@ -40,14 +41,15 @@ class GpuSide:
         return np.stack([self.m_row(i)[0] for i in range(self.cfg.n_samples)])
 
 
-def run_boundary(cfg, n_batch=None, epochs=None, check_all_m=True, order_fn=None, act_fn=None, stochastic_seed=None):
+def run_boundary(cfg, n_batch=None, epochs=None, check_all_m=True, order_fn=None, act_fn=None, stochastic_seed=None,
+                 hosted=False):
     """Every call of every epoch: GPU sender -> GPU receiver and oracle sender -> oracle
     receiver; packed, scales, first flags, out and (per epoch) both m arrays and the state
     digests must agree exactly."""
     nb = n_batch or cfg.n_batch
     epochs = epochs or cfg.epochs
     assert cfg.n_samples % nb == 0
-    gs, gr = GpuSide(cfg, nb), GpuSide(cfg, nb)
+    gs, gr = GpuSide(cfg, nb, hosted=hosted), GpuSide(cfg, nb, hosted=hosted)
     od = DT[cfg.dtype][1]
     os_, or_ = (oracle.Side(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, od) for _ in range(2))
     packed = torch.empty((nb, cfg.packed_bytes), dtype=torch.uint8, device="cuda")

@@ -454,3 +454,31 @@ def test_random_configurations():
         cfg = synth.Boundary(f"rnd{trial}", n_samples, nb, seq, hidden, dtype, bits, group, 3, kind,
                              float(rng.choice([0.0, 0.01, 0.5])), seed=300 + trial)
         run_boundary(cfg, stochastic_seed=(int(rng.integers(1 << 40)) if trial % 3 == 0 else None))
+
+
+# ----------------------------------------------------------------- m in page-locked host memory
+
+def test_hosted_store_gives_the_same_results():
+    run_boundary(synth.TINY, hosted=True)
+    run_boundary(synth.shrink(synth.GPT2_XL, 8, seq=128, epochs=3), n_batch=4, hosted=True)
+    run_boundary(synth.shrink(synth.DEBERTA_XXL, 16, seq=32), hosted=True, stochastic_seed=5)
+    cfg = synth.Boundary("hosted-ragged", 6, 3, 37, 136, "bf16", 3, 8, 3, "outlier", 0.3, seed=411)
+    run_boundary(cfg, hosted=True)
+
+
+def test_hosted_store_checkpoint_and_digest():
+    cfg = synth.Boundary("hosted-ckpt", 3, 1, 4, 64, "fp16", 4, 64, 1, "normal", 0.1, seed=412)
+    a, b = GpuSide(cfg, 1, hosted=True), GpuSide(cfg, 1)
+    try:
+        ids = torch.tensor([2], dtype=torch.int32, device="cuda")
+        act = synth.activation(cfg, [2], 0, device="cuda")
+        p = torch.empty((1, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
+        s = torch.empty((1, cfg.groups), dtype=torch.float32, device="cuda")
+        aq.aq_encode(a.h, act, ids, p, s)
+        for i in range(3):
+            row, seen = a.m_row(i)
+            aq.aq_import_sample(b.h, i, row, seen)
+        assert aq.aq_state_checksum(a.h) == aq.aq_state_checksum(b.h) == aq.aq_state_checksum_noalloc(a.h)
+    finally:
+        a.close()
+        b.close()
