@@ -237,6 +237,19 @@ int aq_decode_host(aq_handle* h, const void* packed_host, const float* scales_ho
                    const void* raw_host, const int32_t* sample_ids_host, void* out_host);
 
 /*
+ * The wire between the two sides of a boundary when both live in one process: copies what
+ * aq_encode produced for the handle's n_batch sequences -- the codes, the steps and, when
+ * raw_src is given (a call with first visits; Algorithm 1: the first message of a sample is
+ * the activation itself), the uncompressed block -- from the sender's device to buffers on
+ * dst_device (the same device, or a peer over NVLink; plain copies into the receiver's own
+ * memory, after which aq_decode reads locally).  Queued on the sender handle's stream `h`; the
+ * receiver's stream has to wait for it (an event, or the same stream).  All pointers are device
+ * pointers; *_dst live on dst_device.
+ */
+int aq_wire_copy(aq_handle* h, int dst_device, void* packed_dst, float* scales_dst, void* raw_dst,
+                 const void* packed_src, const float* scales_src, const void* raw_src);
+
+/*
  * State access for checkpoints and tests.  Copies one sample's m block
  * (aq_m_bytes_per_sample bytes) and its seen flag between the handle and HOST memory;
  * synchronises the stream.

@@ -38,6 +38,8 @@ SIGNATURES = {
     "aq_m_bytes_per_sample": (C.c_int64, [C.c_void_p]),
     "aq_encode_host": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "aq_decode_host": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "aq_wire_copy": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                               C.c_void_p]),
     "aq_export_sample": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]),
     "aq_import_sample": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p, C.c_uint8]),
 }
@@ -176,6 +178,11 @@ def aq_encode_host(h, act_host, sample_ids_host, packed_host, scales_host):
 def aq_decode_host(h, packed_host, scales_host, raw_host, sample_ids_host, out_host):
     return _check(h, lib().aq_decode_host(h, _ptr(packed_host), _ptr(scales_host), _ptr(raw_host),
                                           _ptr(sample_ids_host), _ptr(out_host)))
+
+
+def aq_wire_copy(h, dst_device, packed_dst, scales_dst, raw_dst, packed_src, scales_src, raw_src):
+    return _check(h, lib().aq_wire_copy(h, dst_device, _ptr(packed_dst), _ptr(scales_dst), _ptr(raw_dst),
+                                        _ptr(packed_src), _ptr(scales_src), _ptr(raw_src)))
 
 
 def aq_export_sample(h, sample_id, m_host):

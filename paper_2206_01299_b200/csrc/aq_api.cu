@@ -373,6 +373,25 @@ int aq_decode_host(aq_handle* h, const void* packed_host, const float* scales_ho
   return AQ_OK;
 }
 
+int aq_wire_copy(aq_handle* h, int dst_device, void* packed_dst, float* scales_dst, void* raw_dst,
+                 const void* packed_src, const float* scales_src, const void* raw_src) {
+  if (!h) return fail(nullptr, AQ_EINVAL, "null handle");
+  if (h->n_batch == 0) return AQ_OK;
+  if (!packed_dst || !scales_dst || !packed_src || !scales_src) return fail(h, AQ_EINVAL, "aq_wire_copy: null pointer");
+  if ((raw_dst == nullptr) != (raw_src == nullptr)) return fail(h, AQ_EINVAL, "aq_wire_copy: raw_dst and raw_src go together");
+  int n_dev = 0;
+  AQ_CUDA(h, cudaGetDeviceCount(&n_dev));
+  if (dst_device < 0 || dst_device >= n_dev) return fail(h, AQ_EINVAL, "aq_wire_copy: no device %d", dst_device);
+  DeviceGuard g(h->device);
+  const size_t nb = (size_t)h->n_batch;
+  AQ_CUDA(h, cudaMemcpyPeerAsync(packed_dst, dst_device, packed_src, h->device, nb * (size_t)h->st.packed_bytes, h->stream));
+  AQ_CUDA(h, cudaMemcpyPeerAsync(scales_dst, dst_device, scales_src, h->device,
+                                 nb * (size_t)h->st.groups * sizeof(float), h->stream));
+  if (raw_src)
+    AQ_CUDA(h, cudaMemcpyPeerAsync(raw_dst, dst_device, raw_src, h->device, nb * (size_t)h->st.elems * 2, h->stream));
+  return AQ_OK;
+}
+
 int aq_export_sample(aq_handle* h, int64_t sample_id, void* m_host, uint8_t* seen_host) {
   if (!h) return fail(nullptr, AQ_EINVAL, "null handle");
   if (sample_id < 0 || sample_id >= h->st.n_samples) return fail(h, AQ_EINVAL, "sample id out of range");

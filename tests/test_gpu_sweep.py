@@ -54,10 +54,9 @@ def test_pipeline_sweep_boundary_major():
                         act = synth.activation(cfg, ids, epoch, device="cuda")
                         # forward: sender -> channel -> receiver
                         aq.aq_encode(gs.h, act, ids_d, tx_p, tx_s)
-                        rx_p.copy_(tx_p)
-                        rx_s.copy_(tx_s)
-                        if epoch == 0:
-                            rx_raw.copy_(act)                       # first visit: the message is the activation
+                        # the channel (same stream as both handles): on a first visit the message is the activation
+                        aq.aq_wire_copy(gs.h, 0, rx_p, rx_s, rx_raw if epoch == 0 else None,
+                                        tx_p, tx_s, act if epoch == 0 else None)
                         aq.aq_decode(gr.h, rx_p, rx_s, ids_d, out)
                         # backward: receiver -> channel -> sender
                         grad = synth.gradient(bwd, call, device="cuda", stream=boundary)
