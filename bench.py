@@ -31,7 +31,10 @@ if ROOT not in sys.path:
 MACRO = 32            # sequences per step: the macro-batch (32 x micro-batch 1 in the paper's GPT2 runs)
 # name -> (recipe in synth, sequences per macro-batch, label); the paper's DeBERTa/QNLI runs use macro-batch 64
 WORKLOADS = {"gpt2": ("GPT2_XL", 32, "GPT2-1.5B-shaped boundary (configs[1])"),
-             "deberta": ("DEBERTA_XXL", 64, "DeBERTa-1.5B-shaped boundary (configs[2])")}
+             "deberta": ("DEBERTA_XXL", 64, "DeBERTa-1.5B-shaped boundary (configs[2])"),
+             # one of the 8 boundaries of the pipeline sweep (they are independent and alike): per macro-batch of 16
+             # micro-batches, forward 3-bit deltas and backward 6-bit gradients, each over a device-to-device wire
+             "sweep": ("SWEEP_FWD", 16, "one boundary of the pipeline sweep (configs[4]): fwd 3-bit delta + bwd 6-bit direct + wire copies")}
 FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one delta-visit launch of 32 GPT2-shaped sequences
@@ -234,6 +237,7 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
 
+    from dataclasses import replace
     from paper_2206_01299_b200 import replicas, synth
     global MACRO, M_BITS
     M_BITS = args.m_bits
@@ -289,12 +293,19 @@ def main():
         handles.append(h)
     snd, rcv = handles
 
-    # fp32 running sum A_e of every sample in id order (the recipe's state), advanced one epoch at a time
-    running = torch.empty((cfg.n_samples, cfg.elems), dtype=torch.float32, device="cuda")
+    # fp32 running sum A_e of every sample in id order (the recipe's state), advanced one epoch at a time;
+    # id spaces too large for that (4 B per element beside the two m arrays) recompute A_e per chunk instead
+    keep_running = cfg.n_samples * cfg.elems * 4 < 40e9
+    running = torch.empty((cfg.n_samples, cfg.elems), dtype=torch.float32, device="cuda") if keep_running else None
     all_ids = torch.arange(cfg.n_samples)
 
     def gen_arena(epoch, order):
         """Activations of one epoch in visiting order: arena[p] = a(order[p]) at that epoch."""
+        if not keep_running:
+            arena = torch.empty((cfg.n_samples, cfg.seq, cfg.hidden), dtype=cfg.torch_dtype, device="cuda")
+            for c in range(0, cfg.n_samples, 16):
+                arena[c:c + 16] = synth.activation(cfg, order[c:c + 16], epoch, device="cuda")
+            return arena
         for c in range(0, cfg.n_samples, 16):
             ids = all_ids[c:c + 16]
             if epoch == 0:
@@ -311,8 +322,23 @@ def main():
     scales = torch.empty((MACRO, cfg.groups), dtype=torch.float32, device="cuda")
     out = torch.empty((MACRO, cfg.seq, cfg.hidden), dtype=cfg.torch_dtype, device="cuda")
 
+    sweep = args.workload == "sweep"
+    if sweep:
+        # receiver's ends of the forward wire, both ends of the backward wire, rotating gradients (4 x 52 MB > L2)
+        bw = synth.SWEEP_BWD
+        bbits, n_grad = bw.bits[0], MACRO * cfg.elems
+        rx_packed, rx_scales = torch.empty_like(packed), torch.empty_like(scales)
+        grads = [synth.gradient(replace(bw, n_batch=MACRO), i, device="cuda") for i in range(4)]
+        g_tx = (torch.empty(n_grad * bbits // 8, dtype=torch.uint8, device="cuda"), torch.empty(n_grad // bw.group, dtype=torch.float32, device="cuda"))
+        g_rx = (torch.empty_like(g_tx[0]), torch.empty_like(g_tx[1]))
+        g_out = torch.empty(n_grad, dtype=cfg.torch_dtype, device="cuda")
+        step_bytes += (2 * n_grad * (2 + bbits / 8 + 4 / bw.group)                      # quantize + dequantize
+                       + 2 * (MACRO * (cfg.packed_bytes + cfg.groups * 4))             # forward wire: read + write
+                       + 2 * (n_grad * bbits // 8 + n_grad // bw.group * 4))           # backward wire
+
     def run_step(arena, ids_dev, s, raw=False):
-        """One macro-batch: MACRO micro-batches in launches of nb, each encoded then decoded."""
+        """One macro-batch: MACRO micro-batches in launches of nb, each encoded then decoded (the pipeline
+        sweep: encode, wire, decode, then the gradient of the macro-batch quantized, wired and dequantized)."""
         for l in range(launches_per_step):
             lo = s * MACRO + l * nb
             a, i = arena[lo:lo + nb], ids_dev[lo:lo + nb]
@@ -320,7 +346,17 @@ def main():
             aq.aq_encode(snd, a, i, p, sc)
             if raw:
                 aq.aq_configure(rcv, aq.AQ_RAW, a)
-            aq.aq_decode(rcv, p, sc, i, o)
+            if sweep:
+                rp, rs = rx_packed[l * nb:(l + 1) * nb], rx_scales[l * nb:(l + 1) * nb]
+                aq.aq_wire_copy(snd, local_rank, rp, rs, None, p, sc, None)
+                aq.aq_decode(rcv, rp, rs, i, o)
+            else:
+                aq.aq_decode(rcv, p, sc, i, o)
+        if sweep:
+            aq.aq_quant_grad(rcv, grads[s % 4], n_grad, bbits, g_tx[0], g_tx[1])
+            g_rx[0].copy_(g_tx[0], non_blocking=True)    # the backward wire (same stream as the handles)
+            g_rx[1].copy_(g_tx[1], non_blocking=True)
+            aq.aq_dequant_grad(snd, g_rx[0], g_rx[1], n_grad, bbits, g_out)
 
     def kernel_pass(first_step, window):
         """Average duration of one encode launch and of one decode launch: `window` steps whose
@@ -490,7 +526,7 @@ def main():
                      "timing": f"CUDA events around {window * launches_per_step} back-to-back launches of the kernel, 3 passes right after the timed steps",
                      "decode_kernel": {"achieved": dec_gbs, "frac": dec_gbs / peak, "avg_launch_ms": dec_ms}},
         "first_visit_epoch": {"ms": first_ms, "GB/s": first_bytes / (first_ms * 1e-3) / 1e9},
-        "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": args.steps * launches_per_step * 2,
+        "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": args.steps * (launches_per_step * 2 + (2 if sweep else 0)),
         "clocks": clocks.summary(),
     }
     line.update(result_extra)

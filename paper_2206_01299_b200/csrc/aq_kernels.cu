@@ -468,16 +468,17 @@ __device__ __forceinline__ void encode_rows(const State& st, const EncodeArgs& a
   }
 }
 
-// CTAs per multiprocessor that the register budget is cut for: the most that compile without
-// spilling (the wide type carries two more guards; fields that straddle words need shuffles).
+// CTAs per multiprocessor that the register budget is cut for: measured, the most that pays
+// (the 3-bit kernels spill a few bytes at six and are still 3 % faster than at four; fields
+// that straddle words need shuffles and more registers).
 template <typename T, int BITS>
 constexpr int encode_ctas_per_sm() {
-  const bool whole_words = BITS == 1 || BITS == 2 || BITS == 4;
-  return !whole_words ? (Conv<T>::kWide ? 3 : 4) : 6;
+  const bool light = BITS <= 4;                 // codes of a chunk fit one word (3 bits: with a few spilled bytes)
+  return !light ? (Conv<T>::kWide ? 3 : 4) : 6;
 }
 template <int BITS>
 constexpr int decode_ctas_per_sm() {
-  return (BITS == 1 || BITS == 2 || BITS == 4 || BITS == 8) ? 6 : (BITS == 3 ? 5 : 4);
+  return (BITS <= 4 || BITS == 8) ? 6 : 4;
 }
 
 template <typename T, int BITS, int LPG, bool STOCH>
