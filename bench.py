@@ -56,8 +56,8 @@ def parse_args():
     ap.add_argument("--graph", action="store_true", help="replay each step as a captured CUDA graph")
     ap.add_argument("--rounding", default="interval", choices=["interval", "stochastic"],
                     help="quantizer of the sender: interval number (default) or unbiased stochastic rounding")
-    ap.add_argument("--m-bits", type=int, default=0, choices=[0, 2, 4, 8],
-                    help="keep the previous messages in this many bits per element (0 = the activation type)")
+    ap.add_argument("--m-bits", type=int, default=0, choices=[0, 2, 4, 8, 32],
+                    help="keep the previous messages in this many bits per element (0 = the activation type, 32 = binary32)")
     ap.add_argument("--hosted", action="store_true", help="keep m in page-locked host memory (aq_create_hosted)")
     ap.add_argument("--rows-per-cta", type=int, default=0, help="AQ_ROWS_PER_CTA of both handles (0 = library default)")
     ap.add_argument("--skip-cpu", action="store_true")
@@ -75,6 +75,8 @@ def bytes_per_element(bits, group):
     """Algorithmic HBM bytes per element of a steady-state encode (= of a decode):
     read a (2) + read m (2) + write m (2) + codes (b/8) + scale (4/G); with m kept in z bits:
     a (2) + m read and written (2 * (z/8 + 4/G)) + codes (b/8) + scale (4/G)."""
+    if M_BITS == 32:                                  # binary32 store: no steps
+        return 2.0 + 8.0 + bits / 8.0 + 4.0 / group
     if M_BITS:
         return 2.0 + 2.0 * (M_BITS / 8.0 + 4.0 / group) + bits / 8.0 + 4.0 / group
     return 6.0 + bits / 8.0 + 4.0 / group
@@ -279,7 +281,8 @@ def main():
 
     handles = []
     for _ in range(2):
-        h = (aq.aq_create_lowbit(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, args.m_bits) if args.m_bits
+        h = (aq.aq_create_fp32(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group) if args.m_bits == 32
+             else aq.aq_create_lowbit(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, args.m_bits) if args.m_bits
              else aq.aq_create_hosted(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group) if args.hosted
              else aq.aq_create(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group))
         aq.aq_configure(h, aq.AQ_DTYPE, aq.AQ_FP16 if cfg.dtype == "fp16" else aq.AQ_BF16)
@@ -387,7 +390,8 @@ def main():
 
     # one throw-away visit on a small boundary of the same type, bit width and group: the first launch of a
     # kernel loads its code (milliseconds), which must not count as first-visit time
-    warm = [aq.aq_create_lowbit(2, 8, cfg.hidden, cfg.bits, cfg.group, args.m_bits) if args.m_bits
+    warm = [aq.aq_create_fp32(2, 8, cfg.hidden, cfg.bits, cfg.group) if args.m_bits == 32
+            else aq.aq_create_lowbit(2, 8, cfg.hidden, cfg.bits, cfg.group, args.m_bits) if args.m_bits
             else aq.aq_create(2, 8, cfg.hidden, cfg.bits, cfg.group) for _ in range(2)]
     for h in warm:
         aq.aq_configure(h, aq.AQ_DTYPE, aq.AQ_FP16 if cfg.dtype == "fp16" else aq.AQ_BF16)
@@ -514,7 +518,7 @@ def main():
                    "micro_batch": cfg.n_batch, "sequences_per_step": MACRO, "sequences_per_launch": nb, "cuda_graph": bool(args.graph), "rounding": args.rounding, "m_bits": args.m_bits or 16,
                    "m_in": "host memory (page-locked, mapped)" if args.hosted else "HBM",
                    "act_dtype": cfg.dtype, "bits": cfg.bits, "group": cfg.group, "n_samples_per_side": cfg.n_samples,
-                   "m_bytes_per_side": cfg.n_samples * (cfg.elems * 2 if not args.m_bits else cfg.elems * args.m_bits // 8 + cfg.groups * 4), "steady_epochs_resident": n_arenas,
+                   "m_bytes_per_side": cfg.n_samples * (cfg.elems * 2 if not args.m_bits else cfg.elems * args.m_bits // 8 + (0 if args.m_bits == 32 else cfg.groups * 4)), "steady_epochs_resident": n_arenas,
                    "l2": f"inputs larger than L2 (each step touches {int(MACRO * cfg.elems * 6 / 1e6)} MB of fresh HBM; no flush needed)",
                    "parallelism": f"dp{world} replicas, no collective"},
         "samples_per_s": replicas.whole_job_rate(args.steps * MACRO, world, elapsed_ms),

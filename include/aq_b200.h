@@ -143,6 +143,14 @@ aq_handle* aq_create_hosted(int64_t n_samples, int seq, int hidden, int bits, in
  */
 aq_handle* aq_create_lowbit(int64_t n_samples, int seq, int hidden, int bits, int group, int m_bits);
 
+/*
+ * The same, with the previous messages kept in binary32 (the precision of the paper's own runs:
+ * 6.4 MB per 1024 x 1600 example): m_new = m + Delta is neither rounded to T nor re-quantized,
+ * the receiver's `out` is T(m_new); 4 bytes per element of state.  Same restrictions as
+ * aq_create_lowbit; aq_state_checksum covers the float words and the seen-set.
+ */
+aq_handle* aq_create_fp32(int64_t n_samples, int seq, int hidden, int bits, int group);
+
 /* Waits for the handle's stream, frees everything the handle owns.  NULL is allowed. */
 void aq_destroy(aq_handle* h);
 

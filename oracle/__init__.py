@@ -264,10 +264,14 @@ class SideLow:
         return np.ctypeslib.as_array(lib().aqo_low_m_codes(self.h), shape=(self.n_samples, self.mbytes))
 
     def m_scales(self):
+        if self.m_bits == 32:
+            return np.zeros((self.n_samples, 0), np.float32)
         return np.ctypeslib.as_array(lib().aqo_low_m_scales(self.h), shape=(self.n_samples, self.ngroups))
 
     def m_values(self):
         """The dequantized store as float64 [n_samples, E]."""
+        if self.m_bits == 32:
+            return self.m_codes().view(np.float32).astype(np.float64)
         out = np.empty((self.n_samples, self.E), np.float64)
         for i in range(self.n_samples):
             k = get_codes(self.m_codes()[i], self.E, self.m_bits).astype(np.float64)

@@ -346,8 +346,19 @@ int resolve_low(SideLow* S, const int32_t* ids, int y) {
   return S->seen[id] ? 0 : 1;
 }
 
+// m_bits == 32: the store is m_new itself, binary32, no steps (the precision of the paper's own
+// runs, 6.4 MB per 1024 x 1600 example); the "codes" array then holds the floats.
+float load_m(const SideLow* S, const uint8_t* MC, const float* MS, int64_t g, int64_t i) {
+  if (S->m_bits == 32) { float v; std::memcpy(&v, MC + 4 * i, 4); return v; }
+  return reconstruct(get_code(MC, i, S->m_bits), MS[g]);
+}
+
 // store <- Q_z(m_new) for one group
 void store_group(SideLow* S, uint8_t* MC, float* MS, int64_t g, const float* m_new, int32_t* km) {
+  if (S->m_bits == 32) {
+    std::memcpy(MC + 4 * g * S->group, m_new, 4 * (size_t)S->group);
+    return;
+  }
   float dm;
   quantize_group(m_new, S->group, S->m_bits, km, &dm);
   MS[g] = dm;
@@ -557,7 +568,7 @@ uint64_t aqo_state_checksum(void* h) {
 
 void* aqo_low_create(int64_t n_samples, int seq, int hidden, int bits, int group, int dtype, int m_bits) {
   if (n_samples <= 0 || seq <= 0 || hidden <= 0 || bits < 1 || bits > 8 || group <= 0) return nullptr;
-  if (m_bits < 1 || m_bits > 8 || hidden % group != 0 || (dtype != DT_FP16 && dtype != DT_BF16)) return nullptr;
+  if (((m_bits < 1 || m_bits > 8) && m_bits != 32) || hidden % group != 0 || (dtype != DT_FP16 && dtype != DT_BF16)) return nullptr;
   const int64_t E = (int64_t)seq * hidden;
   if ((E * bits) % 8 != 0 || (E * m_bits) % 8 != 0) return nullptr;
   SideLow* S = new (std::nothrow) SideLow();
@@ -565,7 +576,7 @@ void* aqo_low_create(int64_t n_samples, int seq, int hidden, int bits, int group
   S->n_samples = n_samples; S->seq = seq; S->hidden = hidden; S->bits = bits; S->group = group;
   S->dtype = dtype; S->m_bits = m_bits; S->status = 0;
   S->m_codes.assign((size_t)(n_samples * E * m_bits / 8), 0);     // codes 0, steps 0: "initialized to 0"
-  S->m_scales.assign((size_t)(n_samples * E / group), 0.0f);
+  S->m_scales.assign(m_bits == 32 ? 0 : (size_t)(n_samples * E / group), 0.0f);
   S->seen.assign((size_t)n_samples, 0);
   return S;
 }
@@ -592,14 +603,14 @@ void aqo_low_encode(void* h, const uint16_t* act, const int32_t* ids, int n_batc
     if (first) first[y] = (uint8_t)(mode == 1);
     if (mode == 2) continue;
     uint8_t* MC = S->m_codes.data() + (int64_t)ids[y] * mbytes;
-    float* MS = S->m_scales.data() + (int64_t)ids[y] * ngroups;
+    float* MS = S->m_bits == 32 ? nullptr : S->m_scales.data() + (int64_t)ids[y] * ngroups;
     for (int64_t g = 0; g < ngroups; ++g) {
       const int64_t base = g * G;
       if (mode == 1) {
         for (int j = 0; j < G; ++j) m_new[j] = t_to_float(a[base + j], S->dtype);
       } else {
         for (int j = 0; j < G; ++j) {
-          m_deq[j] = reconstruct(get_code(MC, base + j, S->m_bits), MS[g]);
+          m_deq[j] = load_m(S, MC, MS, g, base + j);
           d[j] = t_to_float(a[base + j], S->dtype) - m_deq[j];
         }
         float delta;
@@ -630,7 +641,7 @@ void aqo_low_decode(void* h, const uint8_t* packed, const float* scales, const u
     if (first) first[y] = (uint8_t)(mode == 1);
     if (mode == 2) { for (int64_t i = 0; i < E; ++i) O[i] = 0; continue; }
     uint8_t* MC = S->m_codes.data() + (int64_t)ids[y] * mbytes;
-    float* MS = S->m_scales.data() + (int64_t)ids[y] * ngroups;
+    float* MS = S->m_bits == 32 ? nullptr : S->m_scales.data() + (int64_t)ids[y] * ngroups;
     const uint8_t* P = packed + (int64_t)y * pbytes;
     const float* SC = scales + (int64_t)y * ngroups;
     const uint16_t* R = raw ? raw + (int64_t)y * E : nullptr;
@@ -641,7 +652,7 @@ void aqo_low_decode(void* h, const uint8_t* packed, const float* scales, const u
           m_new[j] = t_to_float(R[base + j], S->dtype);
           O[base + j] = R[base + j];
         } else {
-          const float m_deq = reconstruct(get_code(MC, base + j, S->m_bits), MS[g]);
+          const float m_deq = load_m(S, MC, MS, g, base + j);
           m_new[j] = m_deq + reconstruct(get_code(P, base + j, S->bits), SC[g]);
           O[base + j] = float_to_t(m_new[j], S->dtype);
         }

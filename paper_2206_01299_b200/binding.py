@@ -22,6 +22,7 @@ AQ_ST_BAD_ID, AQ_ST_DUP_ID, AQ_ST_NO_RAW = 1, 2, 4
 SIGNATURES = {
     "aq_create": (C.c_void_p, [C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int]),
     "aq_create_hosted": (C.c_void_p, [C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int]),
+    "aq_create_fp32": (C.c_void_p, [C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int]),
     "aq_create_lowbit": (C.c_void_p, [C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int]),
     "aq_destroy": (None, [C.c_void_p]),
     "aq_configure": (C.c_int, [C.c_void_p, C.c_int, C.c_int64]),
@@ -97,6 +98,13 @@ def aq_create(n_samples, seq, hidden, bits, group):
 
 def aq_create_hosted(n_samples, seq, hidden, bits, group):
     h = lib().aq_create_hosted(n_samples, seq, hidden, bits, group)
+    if not h:
+        raise AqError(AQ_EINVAL, aq_last_error(None))
+    return h
+
+
+def aq_create_fp32(n_samples, seq, hidden, bits, group):
+    h = lib().aq_create_fp32(n_samples, seq, hidden, bits, group)
     if not h:
         raise AqError(AQ_EINVAL, aq_last_error(None))
     return h

@@ -108,6 +108,10 @@ aq_handle* aq_create_hosted(int64_t n_samples, int seq, int hidden, int bits, in
   return create_handle(n_samples, seq, hidden, bits, group, 0, true);
 }
 
+aq_handle* aq_create_fp32(int64_t n_samples, int seq, int hidden, int bits, int group) {
+  return create_handle(n_samples, seq, hidden, bits, group, 32);
+}
+
 aq_handle* aq_create_lowbit(int64_t n_samples, int seq, int hidden, int bits, int group, int m_bits) {
   if (m_bits != 2 && m_bits != 4 && m_bits != 8) {
     g_create_err[0] = 0;
@@ -144,7 +148,8 @@ static aq_handle* create_handle(int64_t n_samples, int seq, int hidden, int bits
   st.m_bits = m_bits;
   st.m_bytes = m_bits ? st.elems * m_bits / 8 : st.elems * 2;
   const size_t m_bytes = (size_t)n_samples * (size_t)st.m_bytes;
-  const size_t m_scale_bytes = m_bits ? (size_t)n_samples * (size_t)st.groups * sizeof(float) : 0;
+  const bool m_steps = m_bits == 2 || m_bits == 4 || m_bits == 8;
+  const size_t m_scale_bytes = m_steps ? (size_t)n_samples * (size_t)st.groups * sizeof(float) : 0;
   const size_t seen_bytes = (size_t)n_samples * sizeof(unsigned long long);
   if (e == cudaSuccess && !hosted) e = cudaMalloc(&st.m, m_bytes);
   if (e == cudaSuccess && hosted) {
@@ -156,10 +161,10 @@ static aq_handle* create_handle(int64_t n_samples, int seq, int hidden, int bits
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&st.arrivals), sizeof(unsigned long long));
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&st.status), sizeof(uint32_t));
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&h->sum_dev), sizeof(unsigned long long));
-  if (e == cudaSuccess && m_bits) e = cudaMalloc(reinterpret_cast<void**>(&st.m_scales), m_scale_bytes);
+  if (e == cudaSuccess && m_steps) e = cudaMalloc(reinterpret_cast<void**>(&st.m_scales), m_scale_bytes);
   if (e == cudaSuccess && !hosted) e = cudaMemset(st.m, 0, m_bytes);           // "initialized to 0"
   if (e == cudaSuccess && hosted) memset(h->m_host, 0, m_bytes);
-  if (e == cudaSuccess && m_bits) e = cudaMemset(st.m_scales, 0, m_scale_bytes);
+  if (e == cudaSuccess && m_steps) e = cudaMemset(st.m_scales, 0, m_scale_bytes);
   if (e == cudaSuccess) e = cudaMemset(st.seen, 0, seen_bytes);
   if (e == cudaSuccess) e = cudaMemset(st.status, 0, sizeof(uint32_t));
   if (e == cudaSuccess) e = cudaMemset(st.arrivals, 0, sizeof(unsigned long long));
@@ -239,7 +244,7 @@ int aq_encode(aq_handle* h, const void* act, const int32_t* sample_ids, void* pa
   aq::EncodeArgs a{act, sample_ids, static_cast<uint8_t*>(packed), scales, h->first_flags, h->n_batch,
                    h->rounding == AQ_ROUND_STOCHASTIC, h->seed, h->epoch};
   if (h->st.m_bits) {
-    if (a.stochastic) return fail(h, AQ_EUNSUPPORTED, "aq_encode: stochastic rounding is not built for the low-precision store");
+    if (a.stochastic) return fail(h, AQ_EUNSUPPORTED, "aq_encode: stochastic rounding is not built for the low-precision and binary32 stores");
     AQ_CUDA(h, aq::launch_encode_lowbit(h->dtype, h->bits, h->st, a, h->stream));
     return AQ_OK;
   }
@@ -325,7 +330,7 @@ int64_t aq_packed_bytes_per_sample(aq_handle* h) { return h ? h->st.packed_bytes
 int64_t aq_scales_per_sample(aq_handle* h) { return h ? h->st.groups : 0; }
 int64_t aq_m_bytes_per_sample(aq_handle* h) {
   if (!h) return 0;
-  return h->st.m_bytes + (h->st.m_bits ? h->st.groups * (int64_t)sizeof(float) : 0);
+  return h->st.m_bytes + (h->st.m_scales ? h->st.groups * (int64_t)sizeof(float) : 0);
 }
 
 int aq_encode_host(aq_handle* h, const void* act_host, const int32_t* sample_ids_host, void* packed_host,
@@ -401,7 +406,7 @@ int aq_export_sample(aq_handle* h, int64_t sample_id, void* m_host, uint8_t* see
   if (m_host) {
     AQ_CUDA(h, cudaMemcpyAsync(m_host, static_cast<const char*>(h->st.m) + (size_t)sample_id * bytes, bytes,
                                cudaMemcpyDeviceToHost, h->stream));
-    if (h->st.m_bits)                             // the steps follow the codes
+    if (h->st.m_scales)                           // the steps follow the codes
       AQ_CUDA(h, cudaMemcpyAsync(static_cast<char*>(m_host) + bytes, h->st.m_scales + (size_t)sample_id * h->st.groups,
                                  (size_t)h->st.groups * sizeof(float), cudaMemcpyDeviceToHost, h->stream));
   }
@@ -422,7 +427,7 @@ int aq_import_sample(aq_handle* h, int64_t sample_id, const void* m_host, uint8_
   const unsigned long long stamp = seen ? aq::kImportedStamp : 0ull;
   AQ_CUDA(h, cudaMemcpyAsync(static_cast<char*>(h->st.m) + (size_t)sample_id * bytes, m_host, bytes,
                              cudaMemcpyHostToDevice, h->stream));
-  if (h->st.m_bits)
+  if (h->st.m_scales)
     AQ_CUDA(h, cudaMemcpyAsync(h->st.m_scales + (size_t)sample_id * h->st.groups, static_cast<const char*>(m_host) + bytes,
                                (size_t)h->st.groups * sizeof(float), cudaMemcpyHostToDevice, h->stream));
   AQ_CUDA(h, cudaMemcpyAsync(h->st.seen + sample_id, &stamp, sizeof(stamp), cudaMemcpyHostToDevice, h->stream));

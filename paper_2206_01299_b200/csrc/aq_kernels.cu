@@ -645,7 +645,8 @@ __global__ void __launch_bounds__(kThreads, 4)
   const bool touch = mode != kModeSkip;
   const unsigned long long sid = touch ? (unsigned long long)(unsigned)sample.id : 0ull;
   uint8_t* m_codes = static_cast<uint8_t*>(st.m) + sid * (unsigned long long)st.m_bytes;
-  float* m_scales = st.m_scales + sid * (unsigned)st.groups;
+  float* m_scales = (MBITS == 32) ? nullptr : st.m_scales + sid * (unsigned)st.groups;
+  uint4* m_f32 = reinterpret_cast<uint4*>(m_codes);              // MBITS == 32: the store is binary32, two pieces per chunk
   const uint4 no_noise = make_uint4(0, 0, 0, 0);
 
   const int r_end = min(st.rows, (int)(blockIdx.x + 1) * plan.rows_per_cta);
@@ -661,15 +662,27 @@ __global__ void __launch_bounds__(kThreads, 4)
       unsigned long long km = 0ull, kw = 0ull;
       float dm = 0.0f;
       uint4 av = make_uint4(0, 0, 0, 0);
+      float m_deq[8], q[8];
+      uint4 mlo = make_uint4(0, 0, 0, 0), mhi = make_uint4(0, 0, 0, 0);
       if (active) {
-        dm = m_scales[g];
+        if constexpr (MBITS == 32) {
+          mlo = ld_stream(m_f32 + 2 * c);
+          mhi = ld_stream(m_f32 + 2 * c + 1);
+        } else {
+          dm = m_scales[g];
+        }
         if (SENDER) av = ld_stream(in + (unsigned)c * (unsigned)kChunk);
         else delta = __ldg(scale_r + g);
       }
-      km = load_codes<MBITS>(m_codes, c, lane, active, false);
+      if constexpr (MBITS != 32) km = load_codes<MBITS>(m_codes, c, lane, active, false);
       if (!SENDER) kw = load_codes<BITS>(wire_r, c, lane, active, words_ok && whole_warp);
-      float m_deq[8], q[8];
-      dequantize8<MBITS>(km, dm, m_deq);
+      if constexpr (MBITS == 32) {
+        const uint32_t w[8] = {mlo.x, mlo.y, mlo.z, mlo.w, mhi.x, mhi.y, mhi.z, mhi.w};
+#pragma unroll
+        for (int j = 0; j < 8; ++j) m_deq[j] = __uint_as_float(w[j]);
+      } else {
+        dequantize8<MBITS>(km, dm, m_deq);
+      }
       if (SENDER) {
         float af[8], d[8];
         Conv<T>::unpack(av, af);
@@ -687,8 +700,15 @@ __global__ void __launch_bounds__(kThreads, 4)
       if (mode == kModeFirst && active) v = ld_stream(in + (unsigned)c * (unsigned)kChunk);
       Conv<T>::unpack(v, m_new);
     }
-    // store <- Q_z(m_new)
-    {
+    // store <- Q_z(m_new), or m_new itself
+    if constexpr (MBITS == 32) {
+      if (active && touch) {
+        st_stream(m_f32 + 2 * c, make_uint4(__float_as_uint(m_new[0]), __float_as_uint(m_new[1]), __float_as_uint(m_new[2]),
+                                            __float_as_uint(m_new[3])));
+        st_stream(m_f32 + 2 * c + 1, make_uint4(__float_as_uint(m_new[4]), __float_as_uint(m_new[5]),
+                                                __float_as_uint(m_new[6]), __float_as_uint(m_new[7])));
+      }
+    } else {
       const float s2 = group_max<0>(abs_max8(m_new), st.lanes_per_group);
       unsigned long long km2;
       float dm2, unused[8];
@@ -801,7 +821,7 @@ __global__ void __launch_bounds__(kThreads) checksum_kernel(const State st, unsi
 
 __global__ void __launch_bounds__(kThreads) checksum_lowbit_kernel(const State st, unsigned long long* sum_out) {
   const long long n_code_words = st.n_samples * st.m_bytes / 4;      // the code bytes of all samples as one array
-  const long long n_scale_words = st.n_samples * st.groups;
+  const long long n_scale_words = st.m_scales ? st.n_samples * st.groups : 0;
   const uint32_t* cw = static_cast<const uint32_t*>(st.m);
   const uint32_t* sw = reinterpret_cast<const uint32_t*>(st.m_scales);
   const long long stride = (long long)gridDim.x * kThreads;
@@ -953,6 +973,7 @@ cudaError_t launch_lowbit(K kernel, const State& st, const EncodeArgs& ea, const
     case 2: return launch_lowbit(lowbit_kernel<T, B, 2, SENDER>, st, ea, da, n_batch, s);           \
     case 4: return launch_lowbit(lowbit_kernel<T, B, 4, SENDER>, st, ea, da, n_batch, s);           \
     case 8: return launch_lowbit(lowbit_kernel<T, B, 8, SENDER>, st, ea, da, n_batch, s);           \
+    case 32: return launch_lowbit(lowbit_kernel<T, B, 32, SENDER>, st, ea, da, n_batch, s);         \
     default: return cudaErrorInvalidValue;                                                          \
   }
 

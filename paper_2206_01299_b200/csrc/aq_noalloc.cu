@@ -100,7 +100,7 @@ extern "C" int aq_state_checksum_noalloc(aq_handle* h, uint64_t* out_host) {
   if (!out_host) return aq::handle_fail(h, AQ_EINVAL, "aq_state_checksum_noalloc: null pointer");
   const aq::State& st = *aq::handle_state(h);
   if (st.m_bits)
-    return aq::handle_fail(h, AQ_EUNSUPPORTED, "aq_state_checksum_noalloc: not built for the low-precision store");
+    return aq::handle_fail(h, AQ_EUNSUPPORTED, "aq_state_checksum_noalloc: not built for the low-precision and binary32 stores");
   const long long n_vec = st.n_samples * (long long)st.chunks;
   const long long n_slots = (n_vec + kSlabVecs - 1) / kSlabVecs;
   if (n_slots > kSlots)

@@ -15,13 +15,15 @@ pytestmark = pytest.mark.gpu
 class LowSide:
     def __init__(self, cfg, n_batch, m_bits):
         self.cfg, self.m_bits = cfg, m_bits
-        self.h = aq.aq_create_lowbit(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, m_bits)
+        self.h = (aq.aq_create_fp32(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group) if m_bits == 32
+                  else aq.aq_create_lowbit(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, m_bits))
         aq.aq_configure(self.h, aq.AQ_DTYPE, DT[cfg.dtype][0])
         aq.aq_configure(self.h, aq.AQ_BATCH, n_batch)
         self.first = torch.zeros(n_batch, dtype=torch.uint8, device="cuda")
         aq.aq_configure(self.h, aq.AQ_FIRST_FLAGS, self.first)
         self.code_bytes = cfg.elems * m_bits // 8
-        assert aq.aq_m_bytes_per_sample(self.h) == self.code_bytes + cfg.groups * 4
+        self.n_steps = 0 if m_bits == 32 else cfg.groups
+        assert aq.aq_m_bytes_per_sample(self.h) == self.code_bytes + self.n_steps * 4
 
     def close(self):
         aq.aq_destroy(self.h)
@@ -30,9 +32,9 @@ class LowSide:
         """(codes uint8[n, code_bytes], steps float32[n, groups], seen uint8[n])"""
         n = self.cfg.n_samples
         codes = np.empty((n, self.code_bytes), np.uint8)
-        steps = np.empty((n, self.cfg.groups), np.float32)
+        steps = np.empty((n, self.n_steps), np.float32)
         seen = np.empty(n, np.uint8)
-        buf = np.empty(self.code_bytes + self.cfg.groups * 4, np.uint8)
+        buf = np.empty(self.code_bytes + self.n_steps * 4, np.uint8)
         for i in range(n):
             seen[i] = aq.aq_export_sample(self.h, i, buf)
             codes[i] = buf[:self.code_bytes]
@@ -82,12 +84,12 @@ def run_lowbit(cfg, m_bits, n_batch=None):
         or_.close()
 
 
-@pytest.mark.parametrize("m_bits", [2, 4, 8])
+@pytest.mark.parametrize("m_bits", [2, 4, 8, 32])
 def test_tiny_boundary_with_a_low_precision_store(m_bits):
     run_lowbit(synth.TINY, m_bits)
 
 
-@pytest.mark.parametrize("m_bits", [2, 8])
+@pytest.mark.parametrize("m_bits", [2, 8, 32])
 def test_large_shapes_reduced_id_space(m_bits):
     run_lowbit(synth.shrink(synth.GPT2_XL, 8, seq=96, epochs=3), m_bits, n_batch=4)
     run_lowbit(synth.shrink(synth.DEBERTA_XXL, 16, seq=40), m_bits)
@@ -97,7 +99,7 @@ def test_large_shapes_reduced_id_space(m_bits):
 @pytest.mark.parametrize("dtype", ["fp16", "bf16"])
 @pytest.mark.parametrize("bits", range(1, 9))
 def test_every_message_width_on_ragged_shapes(dtype, bits):
-    m_bits = (2, 4, 8)[bits % 3]
+    m_bits = (2, 4, 8, 32)[bits % 4]
     cfg = synth.Boundary("low-ragged", 6, 3, 37, 136, dtype, bits, 8, 3, "outlier", 0.3, seed=120 + bits)
     run_lowbit(cfg, m_bits)
     cfg = synth.Boundary("low-groups", 4, 2, 3, 1024, dtype, bits, 256, 3, "student_t3", 0.2, seed=140 + bits)

@@ -131,3 +131,47 @@ def test_low_precision_bad_ids():
     assert snd.status() == (oracle.ST_BAD_ID | oracle.ST_DUP_ID) and list(snd.seen()) == [0, 1, 0, 0]
     out, _ = rcv.decode(p, s, np.array([1, 2], np.int32), raw=None)
     assert rcv.status() == oracle.ST_NO_RAW and not out.any() and not rcv.seen().any()
+
+
+@pytest.mark.parametrize("dtype", [FP16, BF16])
+def test_binary32_store(dtype):
+    """m kept in binary32 (m_bits = 32): m_new = m + Q(a - m) is stored as it is, the receiver's
+    activation is T(m_new); wiring against the separately pinned bare quantizer, the message
+    bound, identity of the two sides, and geometric decay of the error of a halted activation
+    without the floor that a 16-bit store has."""
+    rng = np.random.default_rng(41)
+    N, seq, hidden, bits, group = 3, 2, 64, 3, 16
+    E = seq * hidden
+    snd = oracle.SideLow(N, seq, hidden, bits, group, dtype, 32)
+    rcv = oracle.SideLow(N, seq, hidden, bits, group, dtype, 32)
+    ids = np.array([2, 0], np.int32)
+    a0 = _rand_act(rng, (2, seq, hidden), dtype)
+    p, s, first = snd.encode(a0, ids)
+    out, _ = rcv.decode(p, s, ids, raw=a0)
+    assert first.all() and np.array_equal(out, a0) and snd.m_codes().shape == (N, E * 4)
+    assert np.array_equal(snd.m_codes()[ids].view(np.float32), _f32(a0.reshape(2, E), dtype))     # stored exactly
+    a1 = _rand_act(rng, (2, seq, hidden), dtype)
+    for visit in range(1, 6):
+        before = snd.m_codes()[ids].view(np.float32).copy()
+        p, s, first = snd.encode(a1, ids)
+        out, _ = rcv.decode(p, s, ids)
+        assert not first.any()
+        assert np.array_equal(snd.m_codes(), rcv.m_codes()) and snd.checksum() == rcv.checksum()
+        a = _f32(a1.reshape(2, E), dtype)
+        for y in range(2):
+            d = a[y] - before[y]
+            m_new = np.empty(E, np.float32)
+            for g in range(E // group):
+                sl = slice(g * group, (g + 1) * group)
+                k, delta = oracle.quantize_group(d[sl], bits)
+                assert np.array_equal(oracle.get_codes(p[y], E, bits)[sl], k) and s[y, g] == delta
+                m_new[sl] = before[y][sl] + np.array([oracle.reconstruct(kk, delta) for kk in k], np.float32)
+            assert np.array_equal(snd.m_codes()[ids[y]].view(np.float32), m_new)
+            want_out = m_new.astype(np.float16).view(np.uint16) if dtype == FP16 else \
+                torch.tensor(m_new).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+            assert np.array_equal(out[y].reshape(-1), want_out)
+        # the error of the store against the halted activation shrinks by 2^-b per visit, with no 16-bit floor
+        D = np.abs(a - _f32(a0.reshape(2, E), dtype)).reshape(2, -1, group).max(-1)
+        err = np.abs(a - snd.m_codes()[ids].view(np.float32)).reshape(2, -1, group).max(-1)
+        assert (err <= D * 2.0 ** (-bits * visit) * (1 + 1e-4) + np.abs(a).reshape(2, -1, group).max(-1) * 2.0 ** -21).all()
+    assert err.max() < 1e-3 * D.max()                      # far below what fp16 / bf16 storage could hold
