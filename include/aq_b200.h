@@ -157,7 +157,7 @@ void aq_destroy(aq_handle* h);
 int aq_configure(aq_handle* h, int key, int64_t value);
 
 /*
- * Sender side (Algorithm 2, "on network a"; Algorithm 1 lines 4-9).  For each
+ * Sender side (Algorithm 2, "on network a"; Algorithm 1, the branch on "xi not seen before").  For each
  * of the n_batch samples, in one fused pass over the data:
  *   first visit  m(xi) <- act (bit copy; the full-precision activation itself is the
  *                message, the caller forwards `act`), codes and scales of the sample = 0;

@@ -416,7 +416,7 @@ const uint16_t* aqo_m(void* h) { return ((Side*)h)->m.data(); }
 const uint8_t* aqo_seen(void* h) { return ((Side*)h)->seen.data(); }
 uint32_t aqo_status(void* h) { Side* S = (Side*)h; uint32_t s = S->status; S->status = 0; return s; }
 
-// Sender (Algorithm 2, "on network a"; Algorithm 1 lines 4-9).
+// Sender (Algorithm 2, "on network a"; Algorithm 1, the branch on "xi not seen before").
 //   act     [n_batch][seq][hidden]  activation a(xi)
 //   ids     [n_batch]               sample ids xi
 //   packed  [n_batch][seq*hidden*bits/8]   out: bitstream of codes
