@@ -40,7 +40,8 @@
  * the work queued on the handle's stream has finished.  The functions only
  * enqueue work on that stream and return; they do not synchronise unless they
  * say so.  Calls on one handle must not overlap on the GPU (use one stream per
- * handle, or order the streams).
+ * handle, or order the streams), and a handle is not thread-safe: one host thread at a
+ * time.  Change AQ_STREAM only while the handle has no work in flight.
  *
  * Errors: functions returning int give AQ_OK or a negative AQ_E* code and leave
  * a message for aq_last_error().  Conditions only the GPU can see (a sample id
