@@ -40,7 +40,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one delta-visit launch of 32 GPT2-shaped sequences
 # (52,428,800 elements), from the ncu capture summarised in profiles/encode_decode_gpt2_boundary_ncu.md;
 # scaled by the elements of a launch.  Set to None when the kernels change after the capture.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = {"encode": 288901632 / 52428800, "decode": 287772928 / 52428800}
+NCU_TRAFFIC_BYTES_PER_ELEMENT = {"encode": 290332160 / 52428800, "decode": 286967040 / 52428800}
 NCU_TRAFFIC_WORKLOAD = "gpt2"
 
 
@@ -59,6 +59,9 @@ def parse_args():
     ap.add_argument("--m-bits", type=int, default=0, choices=[0, 2, 4, 8, 32],
                     help="keep the previous messages in this many bits per element (0 = the activation type, 32 = binary32)")
     ap.add_argument("--hosted", action="store_true", help="keep m in page-locked host memory (aq_create_hosted)")
+    ap.add_argument("--prefetch", action="store_true",
+                    help="with --hosted: fetch every call's previous messages ahead of it (aq_prefetch); the calls "
+                         "then run on staged rows in HBM and write them back behind the caller")
     ap.add_argument("--rows-per-cta", type=int, default=0, help="AQ_ROWS_PER_CTA of both handles (0 = library default)")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--skip-e2e", action="store_true")
@@ -279,6 +282,8 @@ def main():
     bpe = bytes_per_element(cfg.bits, cfg.group)
     step_bytes = 2 * MACRO * cfg.elems * bpe          # encode + decode
 
+    if args.prefetch and not args.hosted:
+        raise SystemExit("--prefetch needs --hosted")
     handles = []
     for _ in range(2):
         h = (aq.aq_create_fp32(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group) if args.m_bits == 32
@@ -339,6 +344,8 @@ def main():
                        + 2 * (MACRO * (cfg.packed_bytes + cfg.groups * 4))             # forward wire: read + write
                        + 2 * (n_grad * bbits // 8 + n_grad // bw.group * 4))           # backward wire
 
+    host_ids = {}                                      # device id list -> its host copy (aq_prefetch reads ids on the host)
+
     def run_step(arena, ids_dev, s, raw=False):
         """One macro-batch: MACRO micro-batches in launches of nb, each encoded then decoded (the pipeline
         sweep: encode, wire, decode, then the gradient of the macro-batch quantized, wired and dequantized)."""
@@ -346,6 +353,10 @@ def main():
             lo = s * MACRO + l * nb
             a, i = arena[lo:lo + nb], ids_dev[lo:lo + nb]
             p, sc, o = packed[l * nb:(l + 1) * nb], scales[l * nb:(l + 1) * nb], out[l * nb:(l + 1) * nb]
+            if args.prefetch:
+                ih = host_ids.setdefault(ids_dev.data_ptr(), ids_dev.cpu())[lo:lo + nb]
+                aq.aq_prefetch(snd, ih)
+                aq.aq_prefetch(rcv, ih)
             aq.aq_encode(snd, a, i, p, sc)
             if raw:
                 aq.aq_configure(rcv, aq.AQ_RAW, a)
@@ -455,6 +466,7 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
         with ClockSampler(local_rank) as clocks:
+            wall0 = time.perf_counter()
             t_begin.record(stream)
             for t in range(args.steps):
                 if graphs:
@@ -463,10 +475,33 @@ def main():
                     run_step(*step_source(args.warmup + t))
             t_end.record(stream)
             torch.cuda.synchronize()
+            wall_ms = (time.perf_counter() - wall0) * 1e3
         if dist:
             dist.barrier()
         torch.cuda.synchronize()
-    elapsed_ms = t_begin.elapsed_time(t_end)
+    # staged calls end with copies on the handles' own copy streams, which the event on `stream` does
+    # not cover: there the step time is the host's, taken between two whole-device synchronisations
+    elapsed_ms = wall_ms if args.prefetch else t_begin.elapsed_time(t_end)
+    staged_call_us = None
+    if args.prefetch:
+        # the calls' time once their rows have arrived: what stays on the critical path of a pipeline stage
+        lat = []
+        with torch.cuda.stream(stream):
+            for r in range(8):
+                arena, ids_dev, sidx = step_source(total_steps + r)
+                lo = sidx * MACRO
+                ih = host_ids.setdefault(ids_dev.data_ptr(), ids_dev.cpu())[lo:lo + nb]
+                aq.aq_prefetch(snd, ih)
+                aq.aq_prefetch(rcv, ih)
+                torch.cuda.synchronize()
+                a0, a1 = ev(), ev()
+                a0.record(stream)
+                aq.aq_encode(snd, arena[lo:lo + nb], ids_dev[lo:lo + nb], packed[:nb], scales[:nb])
+                aq.aq_decode(rcv, packed[:nb], scales[:nb], ids_dev[lo:lo + nb], out[:nb])
+                a1.record(stream)
+                torch.cuda.synchronize()
+                lat.append(a0.elapsed_time(a1) * 1e3)
+        staged_call_us = statistics.median(lat)
     # per-kernel durations: the steps that follow the timed ones, same handles, same data
     window = min(32, steps_per_epoch)
     with torch.cuda.stream(stream):
@@ -516,7 +551,8 @@ def main():
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": label, "hidden": cfg.hidden, "seq": cfg.seq,
                    "micro_batch": cfg.n_batch, "sequences_per_step": MACRO, "sequences_per_launch": nb, "cuda_graph": bool(args.graph), "rounding": args.rounding, "m_bits": args.m_bits or 16,
-                   "m_in": "host memory (page-locked, mapped)" if args.hosted else "HBM",
+                   "m_in": ("host memory (page-locked), staged through HBM by aq_prefetch, written back on a copy stream; step time by the host clock" if args.prefetch
+                            else "host memory (page-locked, mapped)" if args.hosted else "HBM"),
                    "act_dtype": cfg.dtype, "bits": cfg.bits, "group": cfg.group, "n_samples_per_side": cfg.n_samples,
                    "m_bytes_per_side": cfg.n_samples * (cfg.elems * 2 if not args.m_bits else cfg.elems * args.m_bits // 8 + (0 if args.m_bits == 32 else cfg.groups * 4)), "steady_epochs_resident": n_arenas,
                    "l2": f"inputs larger than L2 (each step touches {int(MACRO * cfg.elems * 6 / 1e6)} MB of fresh HBM; no flush needed)",
@@ -533,6 +569,8 @@ def main():
         "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": args.steps * (launches_per_step * 2 + (2 if sweep else 0)),
         "clocks": clocks.summary(),
     }
+    if staged_call_us is not None:
+        line["staged_encode_plus_decode_us"] = staged_call_us
     line.update(result_extra)
     print(json.dumps(line))
 

@@ -108,7 +108,9 @@ enum { AQ_ROUND_INTERVAL = 0, AQ_ROUND_STOCHASTIC = 1 };
 enum {
   AQ_ST_BAD_ID = 1,      /* a sample id was < 0 or >= n_samples */
   AQ_ST_DUP_ID = 2,      /* an id appeared twice in one call; every occurrence after the first is skipped */
-  AQ_ST_NO_RAW = 4       /* aq_decode met a first-visit sample while AQ_RAW was 0 */
+  AQ_ST_NO_RAW = 4,      /* aq_decode met a first-visit sample while AQ_RAW was 0 */
+  AQ_ST_STAGED = 8       /* a call after aq_prefetch brought another id at some position than the one
+                            prefetched for it; that sample is skipped */
 };
 
 /*
@@ -129,6 +131,30 @@ aq_handle* aq_create(int64_t n_samples, int seq, int hidden, int bits, int group
  * compute, as the paper hides the transfers behind the forward pass.
  */
 aq_handle* aq_create_hosted(int64_t n_samples, int seq, int hidden, int bits, int group);
+
+/*
+ * Hosted handles only (AQ_EUNSUPPORTED otherwise): fetch m(xi) of the NEXT aq_encode / aq_decode
+ * call ahead of time (Section 3.3 and the appendix on offloading: the previous messages are
+ * prefetched from host memory while the preceding stages compute, so the transfer is off the
+ * critical path).  sample_ids_host int32[n] (host; copied before the call returns), n must equal
+ * AQ_BATCH now and at that call.  The call returns at once; on a copy stream of the handle's
+ * own, behind everything issued so far on the handle's stream, each sample's row of m is copied
+ * into a staging block in device memory (n rows, allocated at the first use and when n grows).
+ * The next aq_encode / aq_decode (aq_encode_host / aq_decode_host too) then
+ *   - waits on the device, not on the host, until the rows have arrived,
+ *   - runs the same kernel on the staged rows at device-memory speed, with the same results as
+ *     on the host block in place, and
+ *   - starts the copy of the rows back to host memory on the copy stream, again without
+ *     blocking the caller; every later call that touches m waits for it on the device.
+ * That call must bring the prefetched ids, position by position: a sample whose id differs is
+ * skipped (codes and scales zero, m untouched, as for a bad id) and AQ_ST_STAGED is set.  Ids
+ * out of range and repeated ids are not fetched and the call reports them as always.  Between
+ * aq_prefetch and the call that uses it, aq_import_sample of one of its samples is not seen by
+ * that call.  A second aq_prefetch before the call replaces the first.  Calls with no prefetch
+ * pending work on the host block in place.  Staged calls use events between two streams and
+ * cannot be captured into a CUDA graph.
+ */
+int aq_prefetch(aq_handle* h, const int32_t* sample_ids_host, int n);
 
 /*
  * The same, with the previous messages kept at low precision (appendix "Number of Bits for

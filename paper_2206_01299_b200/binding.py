@@ -16,7 +16,7 @@ AQ_DTYPE, AQ_BATCH, AQ_STREAM, AQ_RAW, AQ_FIRST_FLAGS, AQ_ROWS_PER_CTA = 1, 2, 3
 AQ_ROUNDING, AQ_SEED, AQ_EPOCH = 7, 8, 9
 AQ_FP16, AQ_BF16 = 0, 1
 AQ_ROUND_INTERVAL, AQ_ROUND_STOCHASTIC = 0, 1
-AQ_ST_BAD_ID, AQ_ST_DUP_ID, AQ_ST_NO_RAW = 1, 2, 4
+AQ_ST_BAD_ID, AQ_ST_DUP_ID, AQ_ST_NO_RAW, AQ_ST_STAGED = 1, 2, 4, 8
 
 # name -> (restype, argtypes); the load test checks these against the header
 SIGNATURES = {
@@ -41,6 +41,7 @@ SIGNATURES = {
     "aq_decode_host": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "aq_wire_copy": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                C.c_void_p]),
+    "aq_prefetch": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int]),
     "aq_export_sample": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]),
     "aq_import_sample": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p, C.c_uint8]),
 }
@@ -191,6 +192,12 @@ def aq_decode_host(h, packed_host, scales_host, raw_host, sample_ids_host, out_h
 def aq_wire_copy(h, dst_device, packed_dst, scales_dst, raw_dst, packed_src, scales_src, raw_src):
     return _check(h, lib().aq_wire_copy(h, dst_device, _ptr(packed_dst), _ptr(scales_dst), _ptr(raw_dst),
                                         _ptr(packed_src), _ptr(scales_src), _ptr(raw_src)))
+
+
+def aq_prefetch(h, sample_ids_host):
+    """sample_ids_host: int32 CPU tensor / numpy array of AQ_BATCH ids."""
+    return _check(h, lib().aq_prefetch(h, _ptr(sample_ids_host), int(sample_ids_host.numel()
+                                       if hasattr(sample_ids_host, "numel") else sample_ids_host.size)))
 
 
 def aq_export_sample(h, sample_id, m_host):

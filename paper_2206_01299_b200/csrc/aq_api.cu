@@ -8,6 +8,8 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <unordered_set>
+#include <vector>
 
 struct aq_handle {
   aq::State st{};
@@ -22,6 +24,25 @@ struct aq_handle {
   uint8_t* first_flags = nullptr;
   unsigned long long* sum_dev = nullptr;     // scratch of aq_state_checksum
   void* m_host = nullptr;                    // hosted store: the pinned host block that st.m maps
+  // hosted store, staged visits: aq_prefetch copies the next call's m(xi) into `slots` on
+  // copy_stream, the call works there and copies the rows back on copy_stream afterwards
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t ev_settled = nullptr;          // the handle's stream, when aq_prefetch was called
+  cudaEvent_t ev_staged = nullptr;           // copy_stream: the prefetched rows are in HBM
+  cudaEvent_t ev_computed = nullptr;         // the handle's stream: the call that used them is done
+  cudaEvent_t ev_written = nullptr;          // copy_stream: its rows are back in host memory
+  void* slots = nullptr;                     // T[slots_batch][elems]
+  int32_t* d_slot_ids = nullptr;             // [slots_batch] ids as given to aq_prefetch
+  int slots_batch = 0;
+  std::vector<int32_t> staged_ids;           // per slot: the sample whose row it holds, -1 = nothing to copy
+  // the ids travel to d_slot_ids from page-locked blocks used in turn (a pageable source would
+  // make the copy wait on the host for copy_stream to drain); an event says when one is free again
+  static constexpr int kIdRing = 4;
+  int32_t* ids_pinned[kIdRing] = {nullptr, nullptr, nullptr, nullptr};
+  cudaEvent_t ev_ids_sent[kIdRing] = {nullptr, nullptr, nullptr, nullptr};
+  unsigned prefetches = 0;
+  bool prefetch_pending = false;
+  bool writeback_issued = false;
   // staging for the host-buffer entry points, sized for staged_batch samples
   int staged_batch = 0;
   void* d_act = nullptr;      // also raw / out
@@ -93,6 +114,38 @@ int ensure_staging(aq_handle* h) {
   return AQ_OK;
 }
 
+// Hosted store: rows that a staged call updated travel back to host memory on copy_stream.
+// Whatever touches the host block next on the handle's stream waits for them on the device.
+cudaError_t settle(aq_handle* h) {
+  if (!h->writeback_issued) return cudaSuccess;
+  return cudaStreamWaitEvent(h->stream, h->ev_written, 0);
+}
+
+// A staged call: `launch` runs on the prefetched rows in HBM, then the rows go home.
+template <typename Launch>
+int run_staged(aq_handle* h, Launch launch) {
+  h->prefetch_pending = false;
+  if ((int)h->staged_ids.size() != h->n_batch)
+    return fail(h, AQ_EINVAL, "the pending aq_prefetch was for %d samples, AQ_BATCH is %d", (int)h->staged_ids.size(), h->n_batch);
+  aq::State st = h->st;
+  st.m = h->slots;
+  st.slot_ids = h->d_slot_ids;
+  AQ_CUDA(h, cudaStreamWaitEvent(h->stream, h->ev_staged, 0));
+  AQ_CUDA(h, launch(st));
+  AQ_CUDA(h, cudaEventRecord(h->ev_computed, h->stream));
+  AQ_CUDA(h, cudaStreamWaitEvent(h->copy_stream, h->ev_computed, 0));
+  const size_t bytes = (size_t)h->st.m_bytes;
+  for (size_t j = 0; j < h->staged_ids.size(); ++j) {
+    const int32_t id = h->staged_ids[j];
+    if (id < 0) continue;
+    AQ_CUDA(h, cudaMemcpyAsync(static_cast<char*>(h->m_host) + (size_t)id * bytes,
+                               static_cast<const char*>(h->slots) + j * bytes, bytes, cudaMemcpyDeviceToHost, h->copy_stream));
+  }
+  AQ_CUDA(h, cudaEventRecord(h->ev_written, h->copy_stream));
+  h->writeback_issued = true;
+  return AQ_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -156,6 +209,13 @@ static aq_handle* create_handle(int64_t n_samples, int seq, int hidden, int bits
     // page-locked host memory that the GPU addresses directly: the kernels stream m over the bus
     e = cudaHostAlloc(&h->m_host, m_bytes, cudaHostAllocMapped | cudaHostAllocPortable);
     if (e == cudaSuccess) e = cudaHostGetDevicePointer(&st.m, h->m_host, 0);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking);
+    for (cudaEvent_t* ev : {&h->ev_settled, &h->ev_staged, &h->ev_computed, &h->ev_written})
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming);
+    for (int i = 0; i < aq_handle::kIdRing; ++i) {
+      if (e == cudaSuccess) e = cudaHostAlloc(reinterpret_cast<void**>(&h->ids_pinned[i]), aq::kMaxBatch * sizeof(int32_t), cudaHostAllocPortable);
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_ids_sent[i], cudaEventDisableTiming);
+    }
   }
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&st.seen), seen_bytes);
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&st.arrivals), sizeof(unsigned long long));
@@ -183,6 +243,17 @@ void aq_destroy(aq_handle* h) {
   DeviceGuard g(h->device);
   cudaStreamSynchronize(h->stream);
   free_staging(h);
+  if (h->copy_stream) {
+    cudaStreamSynchronize(h->copy_stream);
+    cudaStreamDestroy(h->copy_stream);
+    cudaEventDestroy(h->ev_settled); cudaEventDestroy(h->ev_staged);
+    cudaEventDestroy(h->ev_computed); cudaEventDestroy(h->ev_written);
+    cudaFree(h->slots); cudaFree(h->d_slot_ids);
+    for (int i = 0; i < aq_handle::kIdRing; ++i) {
+      cudaFreeHost(h->ids_pinned[i]);
+      cudaEventDestroy(h->ev_ids_sent[i]);
+    }
+  }
   if (h->m_host) cudaFreeHost(h->m_host);
   else cudaFree(h->st.m);
   cudaFree(h->st.m_scales);
@@ -248,6 +319,9 @@ int aq_encode(aq_handle* h, const void* act, const int32_t* sample_ids, void* pa
     AQ_CUDA(h, aq::launch_encode_lowbit(h->dtype, h->bits, h->st, a, h->stream));
     return AQ_OK;
   }
+  if (h->prefetch_pending)
+    return run_staged(h, [&](const aq::State& st) { return aq::launch_encode(h->dtype, h->bits, st, a, h->stream); });
+  AQ_CUDA(h, settle(h));
   AQ_CUDA(h, aq::launch_encode(h->dtype, h->bits, h->st, a, h->stream));
   return AQ_OK;
 }
@@ -264,6 +338,9 @@ int aq_decode(aq_handle* h, const void* packed, const float* scales, const int32
     AQ_CUDA(h, aq::launch_decode_lowbit(h->dtype, h->bits, h->st, a, h->stream));
     return AQ_OK;
   }
+  if (h->prefetch_pending)
+    return run_staged(h, [&](const aq::State& st) { return aq::launch_decode(h->dtype, h->bits, st, a, h->stream); });
+  AQ_CUDA(h, settle(h));
   AQ_CUDA(h, aq::launch_decode(h->dtype, h->bits, h->st, a, h->stream));
   return AQ_OK;
 }
@@ -303,6 +380,7 @@ int aq_state_checksum(aq_handle* h, uint64_t* out_host) {
   if (!h) return fail(nullptr, AQ_EINVAL, "null handle");
   if (!out_host) return fail(h, AQ_EINVAL, "aq_state_checksum: null pointer");
   DeviceGuard g(h->device);
+  AQ_CUDA(h, settle(h));
   AQ_CUDA(h, cudaMemsetAsync(h->sum_dev, 0, sizeof(unsigned long long), h->stream));
   AQ_CUDA(h, aq::launch_checksum(h->st, h->sum_dev, h->stream));
   unsigned long long v = 0;
@@ -378,6 +456,49 @@ int aq_decode_host(aq_handle* h, const void* packed_host, const float* scales_ho
   return AQ_OK;
 }
 
+int aq_prefetch(aq_handle* h, const int32_t* sample_ids_host, int n) {
+  if (!h) return fail(nullptr, AQ_EINVAL, "null handle");
+  if (!h->m_host) return fail(h, AQ_EUNSUPPORTED, "aq_prefetch: the handle keeps m in device memory (see aq_create_hosted)");
+  if (n != h->n_batch) return fail(h, AQ_EINVAL, "aq_prefetch: n must equal AQ_BATCH (%d), got %d", h->n_batch, n);
+  if (n == 0) return AQ_OK;
+  if (!sample_ids_host) return fail(h, AQ_EINVAL, "aq_prefetch: null pointer");
+  DeviceGuard g(h->device);
+  const size_t bytes = (size_t)h->st.m_bytes;
+  if (h->slots_batch < n) {
+    AQ_CUDA(h, cudaStreamSynchronize(h->copy_stream));
+    AQ_CUDA(h, cudaStreamSynchronize(h->stream));
+    cudaFree(h->slots); cudaFree(h->d_slot_ids);
+    h->slots = nullptr; h->d_slot_ids = nullptr; h->slots_batch = 0;
+    AQ_CUDA(h, cudaMalloc(&h->slots, (size_t)n * bytes));
+    AQ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&h->d_slot_ids), (size_t)n * sizeof(int32_t)));
+    h->slots_batch = n;
+  }
+  // rows to move: every id once (the kernels skip an id's later occurrences and ids out of range)
+  h->staged_ids.assign(sample_ids_host, sample_ids_host + n);
+  std::unordered_set<int32_t> taken;
+  for (int32_t& id : h->staged_ids)
+    if (id < 0 || (long long)id >= h->st.n_samples || !taken.insert(id).second) id = -1;
+  // the copies start once everything issued so far on the handle's stream is done (it may
+  // write the host block in place, and an earlier staged call still owns the slots until
+  // its write-back, which copy_stream runs first)
+  AQ_CUDA(h, cudaEventRecord(h->ev_settled, h->stream));
+  AQ_CUDA(h, cudaStreamWaitEvent(h->copy_stream, h->ev_settled, 0));
+  const int ring = (int)(h->prefetches++ % aq_handle::kIdRing);
+  AQ_CUDA(h, cudaEventSynchronize(h->ev_ids_sent[ring]));      // long done, unless kIdRing prefetches are queued
+  memcpy(h->ids_pinned[ring], sample_ids_host, (size_t)n * sizeof(int32_t));
+  AQ_CUDA(h, cudaMemcpyAsync(h->d_slot_ids, h->ids_pinned[ring], (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice, h->copy_stream));
+  AQ_CUDA(h, cudaEventRecord(h->ev_ids_sent[ring], h->copy_stream));
+  for (int j = 0; j < n; ++j) {
+    const int32_t id = h->staged_ids[j];
+    if (id < 0) continue;
+    AQ_CUDA(h, cudaMemcpyAsync(static_cast<char*>(h->slots) + (size_t)j * bytes,
+                               static_cast<const char*>(h->m_host) + (size_t)id * bytes, bytes, cudaMemcpyHostToDevice, h->copy_stream));
+  }
+  AQ_CUDA(h, cudaEventRecord(h->ev_staged, h->copy_stream));
+  h->prefetch_pending = true;
+  return AQ_OK;
+}
+
 int aq_wire_copy(aq_handle* h, int dst_device, void* packed_dst, float* scales_dst, void* raw_dst,
                  const void* packed_src, const float* scales_src, const void* raw_src) {
   if (!h) return fail(nullptr, AQ_EINVAL, "null handle");
@@ -402,6 +523,7 @@ int aq_export_sample(aq_handle* h, int64_t sample_id, void* m_host, uint8_t* see
   if (sample_id < 0 || sample_id >= h->st.n_samples) return fail(h, AQ_EINVAL, "sample id out of range");
   if (!m_host && !seen_host) return fail(h, AQ_EINVAL, "aq_export_sample: null pointers");
   DeviceGuard g(h->device);
+  AQ_CUDA(h, settle(h));
   const size_t bytes = (size_t)h->st.m_bytes;
   if (m_host) {
     AQ_CUDA(h, cudaMemcpyAsync(m_host, static_cast<const char*>(h->st.m) + (size_t)sample_id * bytes, bytes,
@@ -423,6 +545,7 @@ int aq_import_sample(aq_handle* h, int64_t sample_id, const void* m_host, uint8_
   if (sample_id < 0 || sample_id >= h->st.n_samples) return fail(h, AQ_EINVAL, "sample id out of range");
   if (!m_host) return fail(h, AQ_EINVAL, "aq_import_sample: null pointer");
   DeviceGuard g(h->device);
+  AQ_CUDA(h, settle(h));
   const size_t bytes = (size_t)h->st.m_bytes;
   const unsigned long long stamp = seen ? aq::kImportedStamp : 0ull;
   AQ_CUDA(h, cudaMemcpyAsync(static_cast<char*>(h->st.m) + (size_t)sample_id * bytes, m_host, bytes,
@@ -446,6 +569,7 @@ cudaStream_t handle_stream(aq_handle* h) { return h->stream; }
 int handle_device(aq_handle* h) { return h->device; }
 
 int handle_fail(aq_handle* h, int code, const char* msg) { return fail(h, code, "%s", msg); }
+cudaError_t handle_settle(aq_handle* h) { return settle(h); }
 
 }  // namespace aq
 

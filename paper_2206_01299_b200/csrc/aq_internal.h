@@ -39,6 +39,8 @@ struct State {
   int lg_shift;                   // log2(lanes_per_group)
   int sms;                        // multiprocessors of the handle's device
   int rows_per_cta;               // 0 = chosen by the launch layer (default); > 0 = fixed rows per CTA
+  const int32_t* slot_ids;        // null: row xi of m belongs to sample xi.  Else m is a staging block of the
+                                  // running call: row y holds m of sample slot_ids[y] (hosted store, prefetched)
 };
 
 struct EncodeArgs {
@@ -83,4 +85,5 @@ const State* handle_state(aq_handle* h);
 cudaStream_t handle_stream(aq_handle* h);
 int handle_device(aq_handle* h);
 int handle_fail(aq_handle* h, int code, const char* msg);   // records msg for aq_last_error, returns code
+cudaError_t handle_settle(aq_handle* h);   // hosted store: makes the handle's stream wait for write-backs in flight
 }  // namespace aq

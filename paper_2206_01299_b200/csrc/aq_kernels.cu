@@ -32,7 +32,7 @@ constexpr int kChunksPerThread = 2;                      // grad kernels: chunks
 constexpr int kChunksPerCta = kThreads * kChunksPerThread;
 
 enum { kModeDelta = 0, kModeFirst = 1, kModeSkip = 2 };
-enum { kStBadId = 1, kStDupId = 2, kStNoRaw = 4 };
+enum { kStBadId = 1, kStDupId = 2, kStNoRaw = 4, kStStaged = 8 };
 
 // What the launch layer decides for one encode / decode launch.
 struct LaunchPlan {
@@ -365,6 +365,7 @@ __device__ __forceinline__ void overlap_with_neighbours() {
 struct Sample {
   int mode;
   int32_t id;
+  unsigned row;   // the sample's row of st.m: its id, or its position in the call when m(xi) was staged
 };
 
 // Sample y of the call, resolved by warp 0 for the whole CTA (one barrier): its id, whether it
@@ -372,6 +373,8 @@ struct Sample {
 // earlier ids), its "seen" stamp and the call number -- four independent memory operations in
 // flight together, the stamp one step behind the id.  Lane 0 of the CTA that owns the sample's
 // first row also records the visit: status bit of a skipped sample, first-visit flag, stamp.
+// With staged messages (st.slot_ids set) row y of st.m holds m of sample slot_ids[y]; a call
+// that brings another id to that position skips the sample.
 __device__ __forceinline__ Sample open_sample(const State& st, const LaunchPlan& plan,
                                               const int32_t* __restrict__ ids, int y, bool need_raw,
                                               bool have_raw, uint8_t* first_flags) {
@@ -385,6 +388,7 @@ __device__ __forceinline__ Sample open_sample(const State& st, const LaunchPlan&
     int dup = 0;
     for (int q = lane; q < y; q += 32) dup |= (ids[q] == id);
     const unsigned long long stamp = (lane == 0 && in_range) ? __ldcg(st.seen + id) : 0ull;
+    const int32_t staged = (lane == 0 && st.slot_ids) ? st.slot_ids[y] : id;
     dup = __any_sync(kFullMask, dup);
     if (lane == 0) {
       int mode;
@@ -395,6 +399,9 @@ __device__ __forceinline__ Sample open_sample(const State& st, const LaunchPlan&
       } else if (dup) {
         mode = kModeSkip;
         why = kStDupId;
+      } else if (staged != id) {
+        mode = kModeSkip;
+        why = kStStaged;
       } else if (stamp != 0ull && stamp != call) {
         mode = kModeDelta;
       } else if (need_raw && !have_raw) {
@@ -405,6 +412,7 @@ __device__ __forceinline__ Sample open_sample(const State& st, const LaunchPlan&
       }
       s_sample.mode = mode;
       s_sample.id = id;
+      s_sample.row = st.slot_ids ? (unsigned)y : (unsigned)id;
       if (blockIdx.x == 0) {                     // once per sample and call
         if (why) atomicOr(st.status, why);
         if (first_flags) first_flags[y] = (uint8_t)(mode == kModeFirst);
@@ -500,7 +508,7 @@ __global__ void __launch_bounds__(kThreads, STOCH ? 4 : encode_ctas_per_sm<T, BI
   const int r_end = min(st.rows, r + plan.rows_per_cta);
 
   if (mode == kModeDelta) {
-    T* m = reinterpret_cast<T*>(st.m) + (unsigned long long)(unsigned)sample.id * elems;
+    T* m = reinterpret_cast<T*>(st.m) + (unsigned long long)sample.row * elems;
     // whole iterations first (rows without a ragged end: no bounds to check), then the rest
     const int whole_end = min(r_end, st.chunks / kThreads);
     for (; r + kRowsPerIter <= whole_end; r += kRowsPerIter)
@@ -512,7 +520,7 @@ __global__ void __launch_bounds__(kThreads, STOCH ? 4 : encode_ctas_per_sm<T, BI
   } else {
     // first visit: the activation itself becomes m(xi); skipped sample: nothing is stored.
     // Either way the sample's codes and scales are zero.
-    T* m = (mode == kModeFirst) ? reinterpret_cast<T*>(st.m) + (unsigned long long)(unsigned)sample.id * elems : nullptr;
+    T* m = (mode == kModeFirst) ? reinterpret_cast<T*>(st.m) + (unsigned long long)sample.row * elems : nullptr;
     for (; r < r_end; ++r) {
       const int c = r * kThreads + tid;
       const bool active = c < st.chunks;
@@ -582,7 +590,7 @@ __global__ void __launch_bounds__(kThreads, decode_ctas_per_sm<BITS>()) decode_k
   const int r_end = min(st.rows, r + plan.rows_per_cta);
 
   if (mode == kModeDelta) {
-    T* m = reinterpret_cast<T*>(st.m) + (unsigned long long)(unsigned)sample.id * elems;
+    T* m = reinterpret_cast<T*>(st.m) + (unsigned long long)sample.row * elems;
     const uint8_t* stream = a.packed + (unsigned long long)(unsigned)y * (unsigned)st.packed_bytes;
     const float* scales = a.scales + (unsigned long long)(unsigned)y * (unsigned)st.groups;
     const bool words_ok = (st.packed_bytes & 3) == 0;
@@ -595,7 +603,7 @@ __global__ void __launch_bounds__(kThreads, decode_ctas_per_sm<BITS>()) decode_k
   } else {
     // first visit: the raw message becomes m(xi) and the activation; skipped sample: zeros out.
     const bool first = mode == kModeFirst;
-    T* m = first ? reinterpret_cast<T*>(st.m) + (unsigned long long)(unsigned)sample.id * elems : nullptr;
+    T* m = first ? reinterpret_cast<T*>(st.m) + (unsigned long long)sample.row * elems : nullptr;
     const T* raw = first ? reinterpret_cast<const T*>(a.raw) + (unsigned long long)(unsigned)y * elems : nullptr;
     for (; r < r_end; ++r) {
       const int c = r * kThreads + tid;

@@ -116,6 +116,7 @@ extern "C" int aq_state_checksum_noalloc(aq_handle* h, uint64_t* out_host) {
   cudaError_t e = scratch_address(device, &scratch);
   const cudaStream_t stream = aq::handle_stream(h);
   unsigned long long v = 0;
+  if (e == cudaSuccess) e = aq::handle_settle(h);
   if (e == cudaSuccess) {
     digest_slabs_kernel<<<(unsigned)n_slots, aq::kThreads, 0, stream>>>(static_cast<const uint4*>(st.m), n_vec, scratch);
     digest_finish_kernel<<<1, aq::kThreads, 0, stream>>>(st.seen, st.n_samples, (int)n_slots, scratch);

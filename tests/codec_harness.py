@@ -42,10 +42,11 @@ class GpuSide:
 
 
 def run_boundary(cfg, n_batch=None, epochs=None, check_all_m=True, order_fn=None, act_fn=None, stochastic_seed=None,
-                 hosted=False):
+                 hosted=False, prefetch=None):
     """Every call of every epoch: GPU sender -> GPU receiver and oracle sender -> oracle
     receiver; packed, scales, first flags, out and (per epoch) both m arrays and the state
-    digests must agree exactly."""
+    digests must agree exactly.  prefetch (hosted handles): a function of the call's running
+    number saying whether the two sides fetch that call's previous messages ahead of it."""
     nb = n_batch or cfg.n_batch
     epochs = epochs or cfg.epochs
     assert cfg.n_samples % nb == 0
@@ -55,6 +56,7 @@ def run_boundary(cfg, n_batch=None, epochs=None, check_all_m=True, order_fn=None
     packed = torch.empty((nb, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
     scales = torch.empty((nb, cfg.groups), dtype=torch.float32, device="cuda")
     out = torch.empty((nb, cfg.seq, cfg.hidden), dtype=cfg.torch_dtype, device="cuda")
+    calls = 0
     try:
         if stochastic_seed is not None:                      # only the sender rounds; the receiver needs no setting
             aq.aq_configure(gs.h, aq.AQ_ROUNDING, aq.AQ_ROUND_STOCHASTIC)
@@ -71,6 +73,10 @@ def run_boundary(cfg, n_batch=None, epochs=None, check_all_m=True, order_fn=None
                 packed.fill_(0xAB)
                 scales.fill_(-7.0)
                 out.fill_(3.0)
+                if prefetch and prefetch(calls):
+                    aq.aq_prefetch(gs.h, ids)
+                    aq.aq_prefetch(gr.h, ids)
+                calls += 1
                 aq.aq_encode(gs.h, act, ids_d, packed, scales)
                 aq.aq_configure(gr.h, aq.AQ_RAW, act)        # first visits: the raw message is the activation
                 aq.aq_decode(gr.h, packed, scales, ids_d, out)
