@@ -1,5 +1,5 @@
 // C ABI of the codec: handle, argument checks, stream plumbing.  All arithmetic lives in
-// aq_kernels.cu; nothing here computes on the CPU and there is no CPU fallback.
+// aq_kernels.cu and aq_lowbit.cu; nothing here computes on the CPU and there is no CPU fallback.
 
 #include "../../include/aq_b200.h"
 #include "aq_internal.h"

@@ -1,4 +1,4 @@
-// Launch-layer interface between the C ABI (aq_api.cu) and the kernels (aq_kernels.cu).
+// Launch-layer interface between the C ABI (aq_api.cu) and the kernels (aq_kernels.cu, aq_lowbit.cu).
 #pragma once
 
 #include <cuda_runtime.h>
