@@ -70,6 +70,8 @@ def lib():
                                                 u8p, f32p]
         L.aqo_low_create.restype = C.c_void_p
         L.aqo_low_create.argtypes = [C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int]
+        L.aqo_low_set_rounding.restype = None
+        L.aqo_low_set_rounding.argtypes = [C.c_void_p, C.c_int, C.c_uint64, C.c_uint64]
         L.aqo_low_destroy.restype = None
         L.aqo_low_destroy.argtypes = [C.c_void_p]
         L.aqo_low_m_codes.restype = u8p
@@ -259,6 +261,10 @@ class SideLow:
 
     def __del__(self):
         self.close()
+
+    def set_rounding(self, stochastic, seed=0, epoch=0):
+        """Rounding of the messages; the store's own re-quantization stays deterministic."""
+        lib().aqo_low_set_rounding(self.h, int(bool(stochastic)), seed, epoch)
 
     def m_codes(self):
         return np.ctypeslib.as_array(lib().aqo_low_m_codes(self.h), shape=(self.n_samples, self.mbytes))

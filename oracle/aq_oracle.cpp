@@ -336,6 +336,8 @@ struct SideLow {
   std::vector<float> m_scales;    // [n_samples][seq*hidden/group], Delta_m of every group
   std::vector<uint8_t> seen;
   uint32_t status;
+  int rounding = 0;              // of the messages only (0: interval number, 1: stochastic); the store's own
+  uint64_t seed = 0, epoch = 0;  // re-quantization always takes the interval number, so that both sides agree
 };
 
 int resolve_low(SideLow* S, const int32_t* ids, int y) {
@@ -581,6 +583,10 @@ void* aqo_low_create(int64_t n_samples, int seq, int hidden, int bits, int group
   return S;
 }
 void aqo_low_destroy(void* h) { delete (SideLow*)h; }
+void aqo_low_set_rounding(void* h, int rounding, uint64_t seed, uint64_t epoch) {
+  SideLow* S = (SideLow*)h;
+  S->rounding = rounding; S->seed = seed; S->epoch = epoch;
+}
 const uint8_t* aqo_low_m_codes(void* h) { return ((SideLow*)h)->m_codes.data(); }
 const float* aqo_low_m_scales(void* h) { return ((SideLow*)h)->m_scales.data(); }
 const uint8_t* aqo_low_seen(void* h) { return ((SideLow*)h)->seen.data(); }
@@ -614,7 +620,10 @@ void aqo_low_encode(void* h, const uint16_t* act, const int32_t* ids, int n_batc
           d[j] = t_to_float(a[base + j], S->dtype) - m_deq[j];
         }
         float delta;
-        quantize_group(d.data(), (int)G, S->bits, k.data(), &delta);
+        if (S->rounding == 1)
+          quantize_group_stochastic(d.data(), (int)G, S->bits, S->seed, S->epoch, (uint32_t)ids[y], base, k.data(), &delta);
+        else
+          quantize_group(d.data(), (int)G, S->bits, k.data(), &delta);
         SC[g] = delta;
         for (int j = 0; j < G; ++j) {
           put_code(P, base + j, S->bits, k[j]);

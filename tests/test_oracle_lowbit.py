@@ -175,3 +175,58 @@ def test_binary32_store(dtype):
         err = np.abs(a - snd.m_codes()[ids].view(np.float32)).reshape(2, -1, group).max(-1)
         assert (err <= D * 2.0 ** (-bits * visit) * (1 + 1e-4) + np.abs(a).reshape(2, -1, group).max(-1) * 2.0 ** -21).all()
     assert err.max() < 1e-3 * D.max()                      # far below what fp16 / bf16 storage could hold
+
+
+@pytest.mark.parametrize("m_bits", [8, 32])
+def test_stochastic_messages_over_the_low_precision_store(m_bits):
+    """Unbiased rounding applies to the message only: its codes are those of the separately
+    pinned bare stochastic quantizer on a - m_deq (stream = sample id, place = the group's first
+    element); the store is re-quantized with the interval number as always, so the receiver,
+    which never sees the rounding mode, ends with the same store."""
+    rng = np.random.default_rng(43)
+    N, seq, hidden, bits, group = 3, 2, 64, 3, 16
+    E = seq * hidden
+    snd = oracle.SideLow(N, seq, hidden, bits, group, FP16, m_bits)
+    rcv = oracle.SideLow(N, seq, hidden, bits, group, FP16, m_bits)
+    ids = np.array([2, 0], np.int32)
+
+    def stored(side, sample):
+        if m_bits == 32:
+            return side.m_codes()[sample].view(np.float32).copy()
+        k = oracle.get_codes(side.m_codes()[sample], E, m_bits)
+        steps = np.repeat(side.m_scales()[sample], group)
+        return np.array([oracle.reconstruct(int(kk), float(dd)) for kk, dd in zip(k, steps)], np.float32)
+
+    a0 = _rand_act(rng, (2, seq, hidden), FP16)
+    snd.set_rounding(True, seed=91, epoch=0)
+    p, s, first = snd.encode(a0, ids)
+    rcv.decode(p, s, ids, raw=a0)
+    assert first.all() and not p.any()
+    differs = False
+    for epoch in range(1, 4):
+        snd.set_rounding(True, seed=91, epoch=epoch)
+        act = _rand_act(rng, (2, seq, hidden), FP16)
+        before = [stored(snd, int(i)) for i in ids]
+        p, s, first = snd.encode(act, ids)
+        out, _ = rcv.decode(p, s, ids)
+        assert not first.any()
+        assert np.array_equal(snd.m_codes(), rcv.m_codes()) and np.array_equal(snd.m_scales(), rcv.m_scales())
+        assert snd.checksum() == rcv.checksum()
+        a = _f32(act.reshape(2, E), FP16)
+        for y in range(2):
+            d = a[y] - before[y]
+            m_new = np.empty(E, np.float32)
+            for g in range(E // group):
+                sl = slice(g * group, (g + 1) * group)
+                k, delta = oracle.quantize_group_stochastic(d[sl], bits, 91, epoch, int(ids[y]), first_elem=g * group)
+                assert np.array_equal(oracle.get_codes(p[y], E, bits)[sl], k) and s[y, g] == delta
+                differs |= not np.array_equal(k, oracle.quantize_group(d[sl], bits)[0])
+                m_new[sl] = before[y][sl] + np.array([oracle.reconstruct(int(kk), delta) for kk in k], np.float32)
+                if m_bits != 32:                              # the store's own quantizer: interval number
+                    km, dm = oracle.quantize_group(m_new[sl], m_bits)
+                    assert np.array_equal(oracle.get_codes(snd.m_codes()[ids[y]], E, m_bits)[sl], km)
+                    assert snd.m_scales()[ids[y], g] == dm
+            if m_bits == 32:
+                assert np.array_equal(stored(snd, int(ids[y])), m_new)
+            assert np.array_equal(out[y].reshape(-1), m_new.astype(np.float16).view(np.uint16))
+    assert differs                                            # the mode did change some codes
