@@ -164,9 +164,11 @@ int aq_prefetch(aq_handle* h, const int32_t* sample_ids_host, int n);
  *   m_deq = (km + 1/2) * Delta_m;  sender: Delta = Q_b(act - m_deq);  m_new = m_deq + Delta (binary32);
  *   store <- Q_mbits(m_new);  the receiver's `out` is T(m_new);
  *   first visit: m_new = act (resp. the raw message), out = the raw message.
- * aq_encode / aq_decode and the host-buffer forms work as for aq_create; AQ_ROUND_STOCHASTIC and
- * aq_state_checksum_noalloc answer AQ_EUNSUPPORTED on such a handle.  aq_state_checksum covers the
- * code bytes (as 32-bit words), then the steps, then the seen-set.
+ * aq_encode / aq_decode and the host-buffer forms work as for aq_create.  AQ_ROUND_STOCHASTIC
+ * applies to the message (Q_b) only: the store's own re-quantization always takes the interval
+ * number, so that the receiver, which never learns the rounding mode, ends with the same store.
+ * aq_state_checksum_noalloc answers AQ_EUNSUPPORTED on such a handle.  aq_state_checksum covers
+ * the code bytes (as 32-bit words), then the steps, then the seen-set.
  */
 aq_handle* aq_create_lowbit(int64_t n_samples, int seq, int hidden, int bits, int group, int m_bits);
 

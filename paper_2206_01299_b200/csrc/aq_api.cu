@@ -315,7 +315,6 @@ int aq_encode(aq_handle* h, const void* act, const int32_t* sample_ids, void* pa
   aq::EncodeArgs a{act, sample_ids, static_cast<uint8_t*>(packed), scales, h->first_flags, h->n_batch,
                    h->rounding == AQ_ROUND_STOCHASTIC, h->seed, h->epoch};
   if (h->st.m_bits) {
-    if (a.stochastic) return fail(h, AQ_EUNSUPPORTED, "aq_encode: stochastic rounding is not built for the low-precision and binary32 stores");
     AQ_CUDA(h, aq::launch_encode_lowbit(h->dtype, h->bits, h->st, a, h->stream));
     return AQ_OK;
   }

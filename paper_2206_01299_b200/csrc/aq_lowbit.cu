@@ -53,8 +53,8 @@ __device__ __forceinline__ void lowbit_put(const State& st, uint8_t* m_codes, fl
 
 // Delta visit of n rows starting at chunk c0 of one sample: all loads of the rows first, then
 // the arithmetic.  FULL: n == kRowsPerIter and every chunk is inside the sample.
-template <typename T, int BITS, int MBITS, bool SENDER, bool FULL>
-__device__ __forceinline__ void lowbit_rows(const State& st, const T* __restrict__ act, const uint8_t* __restrict__ wire_r,
+template <typename T, int BITS, int MBITS, bool SENDER, bool STOCH, bool FULL>
+__device__ __forceinline__ void lowbit_rows(const State& st, const EncodeArgs& ea, uint32_t stream_id, const T* __restrict__ act, const uint8_t* __restrict__ wire_r,
                                             const float* __restrict__ scale_r, uint8_t* __restrict__ wire_w,
                                             float* __restrict__ scale_w, T* __restrict__ out, uint8_t* m_codes,
                                             float* m_scales, int c0, int n, int lane, bool words_ok) {
@@ -104,7 +104,9 @@ __device__ __forceinline__ void lowbit_rows(const State& st, const T* __restrict
 #pragma unroll
         for (int j = 0; j < 8; ++j) d[j] = __fsub_rn(af[j], m_deq[j]);
         const float s = group_max_any(abs_max8(d), st.lanes_per_group);
-        quantize8<BITS, true, false>(d, s, make_uint4(0, 0, 0, 0), delta[i], codes, q);
+        uint4 noise = make_uint4(0, 0, 0, 0);                // the message's rounding; the store's stays deterministic
+        if constexpr (STOCH) noise = chunk_noise(ea.seed, ea.epoch, stream_id, (uint32_t)c);
+        quantize8<BITS, true, STOCH>(d, s, noise, delta[i], codes, q);
       } else {
         dequantize8<BITS>(kw[i], delta[i], q);
       }
@@ -123,7 +125,7 @@ __device__ __forceinline__ void lowbit_rows(const State& st, const T* __restrict
 
 // CTAs per multiprocessor, measured: the re-quantizing kernels are bound by instruction issue and
 // gain from every resident warp; the binary32 store is bound by memory and best at four.
-template <typename T, int BITS, int MBITS, bool SENDER>
+template <typename T, int BITS, int MBITS, bool SENDER, bool STOCH>
 __global__ void __launch_bounds__(kThreads, MBITS == 32 ? 4 : 6)
     lowbit_kernel(const State st, const EncodeArgs ea, const DecodeArgs da, const LaunchPlan plan) {
   const int tid = threadIdx.x;
@@ -153,11 +155,13 @@ __global__ void __launch_bounds__(kThreads, MBITS == 32 ? 4 : 6)
   if (mode == kModeDelta) {
     const int whole_end = min(r_end, st.chunks / kThreads);
     for (; r + kRowsPerIter <= whole_end; r += kRowsPerIter)
-      lowbit_rows<T, BITS, MBITS, SENDER, true>(st, in, wire_r, scale_r, wire_w, scale_w, out, m_codes, m_scales,
-                                                r * kThreads + tid, kRowsPerIter, lane, words_ok);
+      lowbit_rows<T, BITS, MBITS, SENDER, STOCH, true>(st, ea, (uint32_t)sample.id, in, wire_r, scale_r, wire_w, scale_w,
+                                                       out, m_codes, m_scales, r * kThreads + tid, kRowsPerIter,
+                                                       lane, words_ok);
     for (; r < r_end; r += kRowsPerIter)
-      lowbit_rows<T, BITS, MBITS, SENDER, false>(st, in, wire_r, scale_r, wire_w, scale_w, out, m_codes, m_scales,
-                                                 r * kThreads + tid, min(kRowsPerIter, r_end - r), lane, words_ok);
+      lowbit_rows<T, BITS, MBITS, SENDER, STOCH, false>(st, ea, (uint32_t)sample.id, in, wire_r, scale_r, wire_w, scale_w,
+                                                        out, m_codes, m_scales, r * kThreads + tid,
+                                                        min(kRowsPerIter, r_end - r), lane, words_ok);
     return;
   }
   // first visit: the activation (the raw message) is the update of an empty store, so this
@@ -200,12 +204,12 @@ cudaError_t launch_lowbit(K kernel, const State& st, const EncodeArgs& ea, const
   return launch_overlapped(kernel, dim3((unsigned)gx, (unsigned)n_batch), s, st, ea, da, plan);
 }
 
-#define AQ_DISPATCH_MBITS(T, B, SENDER)                                                             \
+#define AQ_DISPATCH_MBITS(T, B, SENDER, STOCH)                                                      \
   switch (st.m_bits) {                                                                              \
-    case 2: return launch_lowbit(lowbit_kernel<T, B, 2, SENDER>, st, ea, da, n_batch, s);           \
-    case 4: return launch_lowbit(lowbit_kernel<T, B, 4, SENDER>, st, ea, da, n_batch, s);           \
-    case 8: return launch_lowbit(lowbit_kernel<T, B, 8, SENDER>, st, ea, da, n_batch, s);           \
-    case 32: return launch_lowbit(lowbit_kernel<T, B, 32, SENDER>, st, ea, da, n_batch, s);         \
+    case 2: return launch_lowbit(lowbit_kernel<T, B, 2, SENDER, STOCH>, st, ea, da, n_batch, s);    \
+    case 4: return launch_lowbit(lowbit_kernel<T, B, 4, SENDER, STOCH>, st, ea, da, n_batch, s);    \
+    case 8: return launch_lowbit(lowbit_kernel<T, B, 8, SENDER, STOCH>, st, ea, da, n_batch, s);    \
+    case 32: return launch_lowbit(lowbit_kernel<T, B, 32, SENDER, STOCH>, st, ea, da, n_batch, s);  \
     default: return cudaErrorInvalidValue;                                                          \
   }
 
@@ -214,16 +218,22 @@ cudaError_t launch_lowbit(K kernel, const State& st, const EncodeArgs& ea, const
 cudaError_t launch_encode_lowbit(int dtype, int bits, const State& st, const EncodeArgs& ea, cudaStream_t s) {
   const DecodeArgs da{};
   const int n_batch = ea.n_batch;
-#define AQ_CALL(T, B) AQ_DISPATCH_MBITS(T, B, true)
-  AQ_DISPATCH(dtype, bits, AQ_CALL)
+  if (ea.stochastic) {
+#define AQ_CALL(T, B) AQ_DISPATCH_MBITS(T, B, true, true)
+    AQ_DISPATCH(dtype, bits, AQ_CALL)
 #undef AQ_CALL
+  } else {
+#define AQ_CALL(T, B) AQ_DISPATCH_MBITS(T, B, true, false)
+    AQ_DISPATCH(dtype, bits, AQ_CALL)
+#undef AQ_CALL
+  }
   return cudaErrorInvalidValue;
 }
 
 cudaError_t launch_decode_lowbit(int dtype, int bits, const State& st, const DecodeArgs& da, cudaStream_t s) {
   const EncodeArgs ea{};
   const int n_batch = da.n_batch;
-#define AQ_CALL(T, B) AQ_DISPATCH_MBITS(T, B, false)
+#define AQ_CALL(T, B) AQ_DISPATCH_MBITS(T, B, false, false)
   AQ_DISPATCH(dtype, bits, AQ_CALL)
 #undef AQ_CALL
   return cudaErrorInvalidValue;

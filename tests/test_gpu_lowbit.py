@@ -42,7 +42,7 @@ class LowSide:
         return codes, steps, seen
 
 
-def run_lowbit(cfg, m_bits, n_batch=None):
+def run_lowbit(cfg, m_bits, n_batch=None, stochastic_seed=None):
     nb = n_batch or cfg.n_batch
     gs, gr = LowSide(cfg, nb, m_bits), LowSide(cfg, nb, m_bits)
     od = DT[cfg.dtype][1]
@@ -51,7 +51,13 @@ def run_lowbit(cfg, m_bits, n_batch=None):
     scales = torch.empty((nb, cfg.groups), dtype=torch.float32, device="cuda")
     out = torch.empty((nb, cfg.seq, cfg.hidden), dtype=cfg.torch_dtype, device="cuda")
     try:
+        if stochastic_seed is not None:                      # only the sender rounds
+            aq.aq_configure(gs.h, aq.AQ_ROUNDING, aq.AQ_ROUND_STOCHASTIC)
+            aq.aq_configure(gs.h, aq.AQ_SEED, stochastic_seed)
         for epoch in range(cfg.epochs):
+            if stochastic_seed is not None:
+                aq.aq_configure(gs.h, aq.AQ_EPOCH, (epoch << 33) | 3)
+                os_.set_rounding(True, stochastic_seed, (epoch << 33) | 3)
             order = synth.epoch_order(cfg, epoch)
             for c in range(cfg.n_samples // nb):
                 ids = order[c * nb:(c + 1) * nb].contiguous()
@@ -94,6 +100,16 @@ def test_large_shapes_reduced_id_space(m_bits):
     run_lowbit(synth.shrink(synth.GPT2_XL, 8, seq=96, epochs=3), m_bits, n_batch=4)
     run_lowbit(synth.shrink(synth.DEBERTA_XXL, 16, seq=40), m_bits)
     run_lowbit(synth.shrink(synth.SWEEP_FWD, 4, seq=64), m_bits)
+
+
+@pytest.mark.parametrize("m_bits", [2, 4, 8, 32])
+def test_stochastic_messages_over_a_low_precision_store(m_bits):
+    """The unbiased rounding applies to the message; the store is re-quantized deterministically
+    and the receiver, which has no rounding setting, must end with the same store."""
+    run_lowbit(synth.TINY, m_bits, stochastic_seed=0x5EED0 + m_bits)
+    run_lowbit(synth.shrink(synth.GPT2_XL, 8, seq=96, epochs=3), m_bits, n_batch=4, stochastic_seed=(1 << 40) + m_bits)
+    cfg = synth.Boundary("low-stoch-ragged", 6, 3, 37, 136, "bf16", 5, 8, 3, "outlier", 0.3, seed=611)
+    run_lowbit(cfg, m_bits, stochastic_seed=7)
 
 
 @pytest.mark.parametrize("dtype", ["fp16", "bf16"])
@@ -139,10 +155,6 @@ def test_bad_ids_import_export_and_unsupported_calls():
         assert aq.aq_state_checksum(fresh.h) == aq.aq_state_checksum(gs.h)
         fresh.close()
         # what is not built for this store says so
-        aq.aq_configure(gs.h, aq.AQ_ROUNDING, aq.AQ_ROUND_STOCHASTIC)
-        with pytest.raises(aq.AqError) as e:
-            aq.aq_encode(gs.h, act, ids.cuda(), packed, scales)
-        assert e.value.code == aq.AQ_EUNSUPPORTED
         with pytest.raises(aq.AqError) as e:
             aq.aq_state_checksum_noalloc(gs.h)
         assert e.value.code == aq.AQ_EUNSUPPORTED
