@@ -59,6 +59,9 @@ def parse_args():
     ap.add_argument("--m-bits", type=int, default=0, choices=[0, 2, 4, 8, 32],
                     help="keep the previous messages in this many bits per element (0 = the activation type, 32 = binary32)")
     ap.add_argument("--hosted", action="store_true", help="keep m in page-locked host memory (aq_create_hosted)")
+    ap.add_argument("--stage-compute-ms", type=float, default=0.0,
+                    help="stand-in for the stage's own work: a kernel that holds the handles' stream for about this many "
+                         "ms after every step, to see what of the codec's time stays on the critical path")
     ap.add_argument("--prefetch", action="store_true",
                     help="with --hosted: fetch every call's previous messages ahead of it (aq_prefetch); the calls "
                          "then run on staged rows in HBM and write them back behind the caller")
@@ -345,18 +348,43 @@ def main():
                        + 2 * (n_grad * bbits // 8 + n_grad // bw.group * 4))           # backward wire
 
     host_ids = {}                                      # device id list -> its host copy (aq_prefetch reads ids on the host)
+    ahead = {"key": None}                              # the step whose rows were fetched at the end of the step before
 
-    def run_step(arena, ids_dev, s, raw=False):
+    def prefetch(ids_dev, lo):
+        key = ids_dev.data_ptr()
+        if key not in host_ids:                        # once per id list: a device-to-host copy in the timed
+            host_ids[key] = ids_dev.cpu()              # steps would queue behind the write-backs
+        ih = host_ids[key][lo:lo + nb]
+        aq.aq_prefetch(snd, ih)
+        aq.aq_prefetch(rcv, ih)
+
+    # stand-in for the stage's own work: a kernel that occupies the handles' stream for a fixed number of
+    # clock cycles and draws next to no power, so that its duration does not depend on what runs beside it
+    # (dense matrix products throttle under the power cap, by another amount in every mode compared)
+    stage_cycles, stage_ms = 0, 0.0
+    if args.stage_compute_ms > 0:
+        stage_cycles = int(args.stage_compute_ms * 1e-3 * 1.965e9)
+        with torch.cuda.stream(stream):
+            torch.cuda._sleep(stage_cycles)
+            c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            c0.record(stream)
+            for _ in range(4):
+                torch.cuda._sleep(stage_cycles)
+            c1.record(stream)
+        torch.cuda.synchronize()
+        stage_ms = c0.elapsed_time(c1) / 4
+
+    def run_step(arena, ids_dev, s, raw=False, nxt=None):
         """One macro-batch: MACRO micro-batches in launches of nb, each encoded then decoded (the pipeline
-        sweep: encode, wire, decode, then the gradient of the macro-batch quantized, wired and dequantized)."""
+        sweep: encode, wire, decode, then the gradient of the macro-batch quantized, wired and dequantized).
+        nxt = (ids_dev, s) of the step that follows: with --prefetch its rows are asked for as soon as this
+        step's calls are issued, so that they travel while the stage computes."""
         for l in range(launches_per_step):
             lo = s * MACRO + l * nb
             a, i = arena[lo:lo + nb], ids_dev[lo:lo + nb]
             p, sc, o = packed[l * nb:(l + 1) * nb], scales[l * nb:(l + 1) * nb], out[l * nb:(l + 1) * nb]
-            if args.prefetch:
-                ih = host_ids.setdefault(ids_dev.data_ptr(), ids_dev.cpu())[lo:lo + nb]
-                aq.aq_prefetch(snd, ih)
-                aq.aq_prefetch(rcv, ih)
+            if args.prefetch and ahead["key"] != (ids_dev.data_ptr(), lo):
+                prefetch(ids_dev, lo)
             aq.aq_encode(snd, a, i, p, sc)
             if raw:
                 aq.aq_configure(rcv, aq.AQ_RAW, a)
@@ -366,6 +394,12 @@ def main():
                 aq.aq_decode(rcv, rp, rs, i, o)
             else:
                 aq.aq_decode(rcv, p, sc, i, o)
+        ahead["key"] = None
+        if args.prefetch and nxt is not None and launches_per_step == 1:
+            prefetch(nxt[0], nxt[1] * MACRO)
+            ahead["key"] = (nxt[0].data_ptr(), nxt[1] * MACRO)
+        if stage_cycles:
+            torch.cuda._sleep(stage_cycles)
         if sweep:
             aq.aq_quant_grad(rcv, grads[s % 4], n_grad, bbits, g_tx[0], g_tx[1])
             g_rx[0].copy_(g_tx[0], non_blocking=True)    # the backward wire (same stream as the handles)
@@ -472,7 +506,7 @@ def main():
                 if graphs:
                     graphs[args.warmup + t].replay()
                 else:
-                    run_step(*step_source(args.warmup + t))
+                    run_step(*step_source(args.warmup + t), nxt=step_source(args.warmup + t + 1)[1:])
             t_end.record(stream)
             torch.cuda.synchronize()
             wall_ms = (time.perf_counter() - wall0) * 1e3
@@ -487,12 +521,12 @@ def main():
         # the calls' time once their rows have arrived: what stays on the critical path of a pipeline stage
         lat = []
         with torch.cuda.stream(stream):
+            if ahead["key"] is not None:                      # use up the rows asked for by the last timed step
+                run_step(*step_source(total_steps))
             for r in range(8):
-                arena, ids_dev, sidx = step_source(total_steps + r)
+                arena, ids_dev, sidx = step_source(total_steps + 1 + r)
                 lo = sidx * MACRO
-                ih = host_ids.setdefault(ids_dev.data_ptr(), ids_dev.cpu())[lo:lo + nb]
-                aq.aq_prefetch(snd, ih)
-                aq.aq_prefetch(rcv, ih)
+                prefetch(ids_dev, lo)
                 torch.cuda.synchronize()
                 a0, a1 = ev(), ev()
                 a0.record(stream)
@@ -571,6 +605,8 @@ def main():
     }
     if staged_call_us is not None:
         line["staged_encode_plus_decode_us"] = staged_call_us
+    if stage_cycles:
+        line["config"]["stage_compute_ms_per_step"] = stage_ms
     line.update(result_extra)
     print(json.dumps(line))
 
