@@ -163,3 +163,55 @@ def test_bad_ids_import_export_and_unsupported_calls():
     finally:
         gs.close()
         gr.close()
+
+
+def test_gpt2_boundary_full_id_space_with_an_8_bit_store():
+    """4096 ids (3.8 GB of codes and steps per side), 32 micro-batches of 1 x 1024 x 1600 fp16 per
+    launch: the launch shape that the benchmark times with --m-bits 8.  The oracle follows the
+    sampled ids only, one small store each."""
+    free, _ = torch.cuda.mem_get_info()
+    if free < 12 * 2 ** 30:
+        pytest.skip("needs 12 GiB of free device memory")
+    cfg, per_launch, m_bits = synth.GPT2_XL, 32, 8
+    gs, gr = LowSide(cfg, per_launch, m_bits), LowSide(cfg, per_launch, m_bits)
+    packed = torch.empty((per_launch, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
+    scales = torch.empty((per_launch, cfg.groups), dtype=torch.float32, device="cuda")
+    out = torch.empty((per_launch, cfg.seq, cfg.hidden), dtype=cfg.torch_dtype, device="cuda")
+    buf = np.empty(aq.aq_m_bytes_per_sample(gs.h), np.uint8)
+    tracked = {}
+    try:
+        order = synth.epoch_order(cfg, 0)
+        for epoch in range(3):
+            for step in (0, 63, cfg.n_samples // per_launch - 1):
+                ids = order[step * per_launch:(step + 1) * per_launch].contiguous()
+                act = synth.activation(cfg, ids, epoch, device="cuda")
+                aq.aq_encode(gs.h, act, ids.cuda(), packed, scales)
+                aq.aq_configure(gr.h, aq.AQ_RAW, act if epoch == 0 else None)
+                aq.aq_decode(gr.h, packed, scales, ids.cuda(), out)
+                torch.cuda.synchronize()
+                for y in (0, per_launch - 1):
+                    sid = int(ids[y])
+                    if sid not in tracked:
+                        tracked[sid] = tuple(oracle.SideLow(1, cfg.seq, cfg.hidden, cfg.bits, cfg.group, DT[cfg.dtype][1], m_bits)
+                                             for _ in range(2))
+                    o_s, o_r = tracked[sid]
+                    zero = np.zeros(1, np.int32)
+                    a_np = bits16(act[y:y + 1])
+                    p_o, s_o, f_o = o_s.encode(a_np, zero)
+                    out_o, _ = o_r.decode(p_o, s_o, zero, raw=a_np if epoch == 0 else None)
+                    assert f_o[0] == (epoch == 0)
+                    assert np.array_equal(packed[y].cpu().numpy(), p_o[0]), (epoch, step, y, "packed")
+                    assert np.array_equal(scales[y].cpu().numpy().view(np.uint32), s_o[0].view(np.uint32)), (epoch, step, y)
+                    assert np.array_equal(bits16(out[y]), out_o[0]), (epoch, step, y, "out")
+                    for g_side, o_side in ((gs, o_s), (gr, o_r)):
+                        assert aq.aq_export_sample(g_side.h, sid, buf) == 1
+                        assert np.array_equal(buf[:gs.code_bytes], o_side.m_codes()[0]), (epoch, step, y, "stored codes")
+                        assert np.array_equal(buf[gs.code_bytes:].view(np.uint32), o_side.m_scales()[0].view(np.uint32))
+        assert aq.aq_status(gs.h) == 0 and aq.aq_status(gr.h) == 0
+        assert aq.aq_state_checksum(gs.h) == aq.aq_state_checksum(gr.h)
+    finally:
+        gs.close()
+        gr.close()
+        for pair in tracked.values():
+            for side in pair:
+                side.close()

@@ -151,3 +151,58 @@ def test_deberta_boundary_full_id_space():
     _needs_gb(60)
     cfg = synth.DEBERTA_XXL
     _full_size_sampled(cfg, cfg.n_batch, steps=[0, 7, cfg.n_samples // cfg.n_batch - 1], samples_per_launch=3)
+
+
+def test_gpt2_boundary_full_id_space_with_stochastic_rounding():
+    """The benchmark's launch shape with the unbiased quantizer: the random stream of a sample is
+    keyed by its id, so the oracle keeps the four lowest ids under their own numbers and the
+    launches that hold them are run at full width."""
+    _needs_gb(34)
+    cfg, per_launch, seed, n_track = synth.GPT2_XL, 32, 0xA05D, 4
+    gs, gr = GpuSide(cfg, per_launch), GpuSide(cfg, per_launch)
+    od = DT[cfg.dtype][1]
+    o_s, o_r = (oracle.Side(n_track, cfg.seq, cfg.hidden, cfg.bits, cfg.group, od) for _ in range(2))
+    packed = torch.empty((per_launch, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
+    scales = torch.empty((per_launch, cfg.groups), dtype=torch.float32, device="cuda")
+    out = torch.empty((per_launch, cfg.seq, cfg.hidden), dtype=cfg.torch_dtype, device="cuda")
+    try:
+        aq.aq_configure(gs.h, aq.AQ_ROUNDING, aq.AQ_ROUND_STOCHASTIC)
+        aq.aq_configure(gs.h, aq.AQ_SEED, seed)
+        order = synth.epoch_order(cfg, 0)
+        where = {int(sid): int(pos) for pos, sid in enumerate(order.tolist()) if sid < n_track}
+        steps = sorted({pos // per_launch for pos in where.values()})
+        checked, differs, before = 0, False, {}
+        for epoch in range(3):
+            aq.aq_configure(gs.h, aq.AQ_EPOCH, epoch)
+            o_s.set_rounding(True, seed, epoch)
+            for step in steps:
+                ids = order[step * per_launch:(step + 1) * per_launch].contiguous()
+                act = synth.activation(cfg, ids, epoch, device="cuda")
+                aq.aq_encode(gs.h, act, ids.cuda(), packed, scales)
+                aq.aq_configure(gr.h, aq.AQ_RAW, act if epoch == 0 else None)
+                aq.aq_decode(gr.h, packed, scales, ids.cuda(), out)
+                torch.cuda.synchronize()
+                for sid, pos in where.items():
+                    if pos // per_launch != step:
+                        continue
+                    y = pos % per_launch
+                    one = np.array([sid], np.int32)
+                    a_np = bits16(act[y:y + 1])
+                    p_o, s_o, f_o = o_s.encode(a_np, one)
+                    out_o, _ = o_r.decode(p_o, s_o, one, raw=a_np if epoch == 0 else None)
+                    assert f_o[0] == (epoch == 0)
+                    assert np.array_equal(packed[y].cpu().numpy(), p_o[0]), (epoch, step, y, "packed")
+                    assert np.array_equal(scales[y].cpu().numpy().view(np.uint32), s_o[0].view(np.uint32)), (epoch, step, y)
+                    assert np.array_equal(bits16(out[y]), out_o[0]), (epoch, step, y, "out")
+                    assert np.array_equal(gs.m_row(sid)[0], o_s.m()[sid]) and np.array_equal(gr.m_row(sid)[0], o_r.m()[sid])
+                    checked += 1
+                    if epoch:                                  # the mode is on: some codes differ from the interval number's
+                        d = (act[y].float() - torch.from_numpy(before[sid].view(np.float16).astype(np.float32)).cuda()).cpu().numpy()
+                        k_det = oracle.quantize_group(d.reshape(-1)[:cfg.group], cfg.bits)[0]
+                        differs |= not np.array_equal(oracle.get_codes(p_o[0], cfg.elems, cfg.bits)[:cfg.group], k_det)
+                    before[sid] = o_s.m()[sid].copy()
+        assert checked == 3 * n_track and differs
+        assert aq.aq_status(gs.h) == 0 and aq.aq_status(gr.h) == 0
+        assert aq.aq_state_checksum(gs.h) == aq.aq_state_checksum(gr.h)
+    finally:
+        gs.close(), gr.close(), o_s.close(), o_r.close()
