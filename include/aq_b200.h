@@ -264,9 +264,13 @@ int64_t aq_m_bytes_per_sample(aq_handle* h);
  * Host-buffer forms: same operations, but every pointer is HOST memory (pinned memory
  * makes the copies asynchronous to the CPU; pageable works).  The call copies the inputs
  * to device staging buffers owned by the handle (allocated on first use, sized for the
- * current AQ_BATCH), runs the same kernel, copies the results back and returns after the
- * stream has finished.  raw_host may be NULL (then first visits at the receiver are
- * skipped and reported, as with AQ_RAW = 0).
+ * current AQ_BATCH), runs the same kernel, copies the results back and returns when they
+ * have arrived.  raw_host may be NULL (then first visits at the receiver are
+ * skipped and reported, as with AQ_RAW = 0).  From 8 samples per call on, and when every id
+ * is in range and appears once, the batch moves in four pieces: the copy in of one piece, the
+ * kernel of the one before and the copy out of the one before that run together (two more
+ * streams of the handle's own, ordered against the handle's stream by events); the results
+ * do not depend on it.
  */
 int aq_encode_host(aq_handle* h, const void* act_host, const int32_t* sample_ids_host,
                    void* packed_host, float* scales_host);

@@ -49,6 +49,11 @@ struct aq_handle {
   int32_t* d_ids = nullptr;
   uint8_t* d_packed = nullptr;
   float* d_scales = nullptr;
+  // the host-buffer calls move a batch in kSlices pieces: copies in on in_stream, kernels on the
+  // handle's stream, copies out on out_stream, so that neighbouring pieces overlap
+  static constexpr int kSlices = 4;
+  cudaStream_t in_stream = nullptr, out_stream = nullptr;
+  cudaEvent_t ev_begin = nullptr, ev_in[kSlices] = {}, ev_done[kSlices] = {};
   char err[256] = {0};
 };
 
@@ -112,6 +117,30 @@ int ensure_staging(aq_handle* h) {
   AQ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&h->d_scales), nb * (size_t)h->st.groups * sizeof(float)));
   h->staged_batch = (int)nb;
   return AQ_OK;
+}
+
+int ensure_slicing(aq_handle* h) {
+  if (h->in_stream) return AQ_OK;
+  AQ_CUDA(h, cudaStreamCreateWithFlags(&h->in_stream, cudaStreamNonBlocking));
+  AQ_CUDA(h, cudaStreamCreateWithFlags(&h->out_stream, cudaStreamNonBlocking));
+  AQ_CUDA(h, cudaEventCreateWithFlags(&h->ev_begin, cudaEventDisableTiming));
+  for (int i = 0; i < aq_handle::kSlices; ++i) {
+    AQ_CUDA(h, cudaEventCreateWithFlags(&h->ev_in[i], cudaEventDisableTiming));
+    AQ_CUDA(h, cudaEventCreateWithFlags(&h->ev_done[i], cudaEventDisableTiming));
+  }
+  return AQ_OK;
+}
+
+// A host-buffer call may run in slices when every id is in range and appears once (the kernels
+// look for repeats inside one launch only) and m is in device memory.
+bool sliceable(const aq_handle* h, const int32_t* ids_host) {
+  if (h->n_batch < 2 * aq_handle::kSlices || h->m_host) return false;
+  std::unordered_set<int32_t> taken;
+  for (int j = 0; j < h->n_batch; ++j) {
+    const int32_t id = ids_host[j];
+    if (id < 0 || (long long)id >= h->st.n_samples || !taken.insert(id).second) return false;
+  }
+  return true;
 }
 
 // Hosted store: rows that a staged call updated travel back to host memory on copy_stream.
@@ -243,6 +272,11 @@ void aq_destroy(aq_handle* h) {
   DeviceGuard g(h->device);
   cudaStreamSynchronize(h->stream);
   free_staging(h);
+  if (h->in_stream) {
+    cudaStreamDestroy(h->in_stream); cudaStreamDestroy(h->out_stream);
+    cudaEventDestroy(h->ev_begin);
+    for (int i = 0; i < aq_handle::kSlices; ++i) { cudaEventDestroy(h->ev_in[i]); cudaEventDestroy(h->ev_done[i]); }
+  }
   if (h->copy_stream) {
     cudaStreamSynchronize(h->copy_stream);
     cudaStreamDestroy(h->copy_stream);
@@ -305,6 +339,26 @@ int aq_configure(aq_handle* h, int key, int64_t value) {
   }
 }
 
+static int launch_encode_call(aq_handle* h, const aq::EncodeArgs& a) {
+  if (h->st.m_bits) {
+    AQ_CUDA(h, aq::launch_encode_lowbit(h->dtype, h->bits, h->st, a, h->stream));
+    return AQ_OK;
+  }
+  AQ_CUDA(h, settle(h));
+  AQ_CUDA(h, aq::launch_encode(h->dtype, h->bits, h->st, a, h->stream));
+  return AQ_OK;
+}
+
+static int launch_decode_call(aq_handle* h, const aq::DecodeArgs& a) {
+  if (h->st.m_bits) {
+    AQ_CUDA(h, aq::launch_decode_lowbit(h->dtype, h->bits, h->st, a, h->stream));
+    return AQ_OK;
+  }
+  AQ_CUDA(h, settle(h));
+  AQ_CUDA(h, aq::launch_decode(h->dtype, h->bits, h->st, a, h->stream));
+  return AQ_OK;
+}
+
 int aq_encode(aq_handle* h, const void* act, const int32_t* sample_ids, void* packed, float* scales) {
   if (!h) return fail(nullptr, AQ_EINVAL, "null handle");
   if (h->n_batch == 0) return AQ_OK;
@@ -314,15 +368,9 @@ int aq_encode(aq_handle* h, const void* act, const int32_t* sample_ids, void* pa
   DeviceGuard g(h->device);
   aq::EncodeArgs a{act, sample_ids, static_cast<uint8_t*>(packed), scales, h->first_flags, h->n_batch,
                    h->rounding == AQ_ROUND_STOCHASTIC, h->seed, h->epoch};
-  if (h->st.m_bits) {
-    AQ_CUDA(h, aq::launch_encode_lowbit(h->dtype, h->bits, h->st, a, h->stream));
-    return AQ_OK;
-  }
-  if (h->prefetch_pending)
+  if (h->prefetch_pending && !h->st.m_bits)
     return run_staged(h, [&](const aq::State& st) { return aq::launch_encode(h->dtype, h->bits, st, a, h->stream); });
-  AQ_CUDA(h, settle(h));
-  AQ_CUDA(h, aq::launch_encode(h->dtype, h->bits, h->st, a, h->stream));
-  return AQ_OK;
+  return launch_encode_call(h, a);
 }
 
 int aq_decode(aq_handle* h, const void* packed, const float* scales, const int32_t* sample_ids, void* out) {
@@ -333,15 +381,9 @@ int aq_decode(aq_handle* h, const void* packed, const float* scales, const int32
     return fail(h, AQ_EINVAL, "aq_decode: packed, scales and out must be 16-byte aligned");
   DeviceGuard g(h->device);
   aq::DecodeArgs a{static_cast<const uint8_t*>(packed), scales, h->raw, sample_ids, out, h->first_flags, h->n_batch};
-  if (h->st.m_bits) {
-    AQ_CUDA(h, aq::launch_decode_lowbit(h->dtype, h->bits, h->st, a, h->stream));
-    return AQ_OK;
-  }
-  if (h->prefetch_pending)
+  if (h->prefetch_pending && !h->st.m_bits)
     return run_staged(h, [&](const aq::State& st) { return aq::launch_decode(h->dtype, h->bits, st, a, h->stream); });
-  AQ_CUDA(h, settle(h));
-  AQ_CUDA(h, aq::launch_decode(h->dtype, h->bits, h->st, a, h->stream));
-  return AQ_OK;
+  return launch_decode_call(h, a);
 }
 
 static int check_grad_args(aq_handle* h, const void* a, const void* b, const void* c, int64_t n_elems, int bits) {
@@ -410,6 +452,13 @@ int64_t aq_m_bytes_per_sample(aq_handle* h) {
   return h->st.m_bytes + (h->st.m_scales ? h->st.groups * (int64_t)sizeof(float) : 0);
 }
 
+// slice i of kSlices over n samples: [lo, lo + cnt)
+static void slice_of(int n, int i, size_t* lo, size_t* cnt) {
+  const int base = n / aq_handle::kSlices, rest = n % aq_handle::kSlices;
+  *lo = (size_t)i * base + (size_t)(i < rest ? i : rest);
+  *cnt = (size_t)base + (i < rest ? 1 : 0);
+}
+
 int aq_encode_host(aq_handle* h, const void* act_host, const int32_t* sample_ids_host, void* packed_host,
                    float* scales_host) {
   if (!h) return fail(nullptr, AQ_EINVAL, "null handle");
@@ -419,13 +468,42 @@ int aq_encode_host(aq_handle* h, const void* act_host, const int32_t* sample_ids
   int rc = ensure_staging(h);
   if (rc != AQ_OK) return rc;
   const size_t nb = (size_t)h->n_batch;
-  AQ_CUDA(h, cudaMemcpyAsync(h->d_act, act_host, nb * (size_t)h->st.elems * 2, cudaMemcpyHostToDevice, h->stream));
-  AQ_CUDA(h, cudaMemcpyAsync(h->d_ids, sample_ids_host, nb * sizeof(int32_t), cudaMemcpyHostToDevice, h->stream));
-  rc = aq_encode(h, h->d_act, h->d_ids, h->d_packed, h->d_scales);
+  const size_t act_b = (size_t)h->st.elems * 2, packed_b = (size_t)h->st.packed_bytes, scales_b = (size_t)h->st.groups * sizeof(float);
+  if (!sliceable(h, sample_ids_host)) {
+    AQ_CUDA(h, cudaMemcpyAsync(h->d_act, act_host, nb * act_b, cudaMemcpyHostToDevice, h->stream));
+    AQ_CUDA(h, cudaMemcpyAsync(h->d_ids, sample_ids_host, nb * sizeof(int32_t), cudaMemcpyHostToDevice, h->stream));
+    rc = aq_encode(h, h->d_act, h->d_ids, h->d_packed, h->d_scales);
+    if (rc != AQ_OK) return rc;
+    AQ_CUDA(h, cudaMemcpyAsync(packed_host, h->d_packed, nb * packed_b, cudaMemcpyDeviceToHost, h->stream));
+    AQ_CUDA(h, cudaMemcpyAsync(scales_host, h->d_scales, nb * scales_b, cudaMemcpyDeviceToHost, h->stream));
+    AQ_CUDA(h, cudaStreamSynchronize(h->stream));
+    return AQ_OK;
+  }
+  rc = ensure_slicing(h);
   if (rc != AQ_OK) return rc;
-  AQ_CUDA(h, cudaMemcpyAsync(packed_host, h->d_packed, nb * (size_t)h->st.packed_bytes, cudaMemcpyDeviceToHost, h->stream));
-  AQ_CUDA(h, cudaMemcpyAsync(scales_host, h->d_scales, nb * (size_t)h->st.groups * sizeof(float), cudaMemcpyDeviceToHost, h->stream));
-  AQ_CUDA(h, cudaStreamSynchronize(h->stream));
+  AQ_CUDA(h, cudaEventRecord(h->ev_begin, h->stream));          // the staging block is free once earlier work is done
+  AQ_CUDA(h, cudaStreamWaitEvent(h->in_stream, h->ev_begin, 0));
+  AQ_CUDA(h, cudaMemcpyAsync(h->d_ids, sample_ids_host, nb * sizeof(int32_t), cudaMemcpyHostToDevice, h->in_stream));
+  for (int i = 0; i < aq_handle::kSlices; ++i) {
+    size_t lo, cnt;
+    slice_of(h->n_batch, i, &lo, &cnt);
+    char* d_act = static_cast<char*>(h->d_act) + lo * act_b;
+    AQ_CUDA(h, cudaMemcpyAsync(d_act, static_cast<const char*>(act_host) + lo * act_b, cnt * act_b, cudaMemcpyHostToDevice, h->in_stream));
+    AQ_CUDA(h, cudaEventRecord(h->ev_in[i], h->in_stream));
+    AQ_CUDA(h, cudaStreamWaitEvent(h->stream, h->ev_in[i], 0));
+    const aq::EncodeArgs a{d_act, h->d_ids + lo, h->d_packed + lo * packed_b, h->d_scales + lo * (size_t)h->st.groups,
+                           h->first_flags ? h->first_flags + lo : nullptr, (int)cnt,
+                           h->rounding == AQ_ROUND_STOCHASTIC, h->seed, h->epoch};
+    rc = launch_encode_call(h, a);
+    if (rc != AQ_OK) return rc;
+    AQ_CUDA(h, cudaEventRecord(h->ev_done[i], h->stream));
+    AQ_CUDA(h, cudaStreamWaitEvent(h->out_stream, h->ev_done[i], 0));
+    AQ_CUDA(h, cudaMemcpyAsync(static_cast<char*>(packed_host) + lo * packed_b, h->d_packed + lo * packed_b, cnt * packed_b,
+                               cudaMemcpyDeviceToHost, h->out_stream));
+    AQ_CUDA(h, cudaMemcpyAsync(reinterpret_cast<char*>(scales_host) + lo * scales_b, h->d_scales + lo * (size_t)h->st.groups,
+                               cnt * scales_b, cudaMemcpyDeviceToHost, h->out_stream));
+  }
+  AQ_CUDA(h, cudaStreamSynchronize(h->out_stream));
   return AQ_OK;
 }
 
@@ -438,20 +516,49 @@ int aq_decode_host(aq_handle* h, const void* packed_host, const float* scales_ho
   int rc = ensure_staging(h);
   if (rc != AQ_OK) return rc;
   const size_t nb = (size_t)h->n_batch;
-  const size_t act_bytes = nb * (size_t)h->st.elems * 2;
-  AQ_CUDA(h, cudaMemcpyAsync(h->d_packed, packed_host, nb * (size_t)h->st.packed_bytes, cudaMemcpyHostToDevice, h->stream));
-  AQ_CUDA(h, cudaMemcpyAsync(h->d_scales, scales_host, nb * (size_t)h->st.groups * sizeof(float), cudaMemcpyHostToDevice, h->stream));
-  AQ_CUDA(h, cudaMemcpyAsync(h->d_ids, sample_ids_host, nb * sizeof(int32_t), cudaMemcpyHostToDevice, h->stream));
+  const size_t act_b = (size_t)h->st.elems * 2, packed_b = (size_t)h->st.packed_bytes, scales_b = (size_t)h->st.groups * sizeof(float);
   // the staging block holds the raw message on the way in and the activation on the way out
   // (every element is read before the same thread overwrites it)
-  if (raw_host) AQ_CUDA(h, cudaMemcpyAsync(h->d_act, raw_host, act_bytes, cudaMemcpyHostToDevice, h->stream));
-  const void* saved_raw = h->raw;
-  h->raw = raw_host ? h->d_act : nullptr;
-  rc = aq_decode(h, h->d_packed, h->d_scales, h->d_ids, h->d_act);
-  h->raw = saved_raw;
+  if (!sliceable(h, sample_ids_host)) {
+    AQ_CUDA(h, cudaMemcpyAsync(h->d_packed, packed_host, nb * packed_b, cudaMemcpyHostToDevice, h->stream));
+    AQ_CUDA(h, cudaMemcpyAsync(h->d_scales, scales_host, nb * scales_b, cudaMemcpyHostToDevice, h->stream));
+    AQ_CUDA(h, cudaMemcpyAsync(h->d_ids, sample_ids_host, nb * sizeof(int32_t), cudaMemcpyHostToDevice, h->stream));
+    if (raw_host) AQ_CUDA(h, cudaMemcpyAsync(h->d_act, raw_host, nb * act_b, cudaMemcpyHostToDevice, h->stream));
+    const void* saved_raw = h->raw;
+    h->raw = raw_host ? h->d_act : nullptr;
+    rc = aq_decode(h, h->d_packed, h->d_scales, h->d_ids, h->d_act);
+    h->raw = saved_raw;
+    if (rc != AQ_OK) return rc;
+    AQ_CUDA(h, cudaMemcpyAsync(out_host, h->d_act, nb * act_b, cudaMemcpyDeviceToHost, h->stream));
+    AQ_CUDA(h, cudaStreamSynchronize(h->stream));
+    return AQ_OK;
+  }
+  rc = ensure_slicing(h);
   if (rc != AQ_OK) return rc;
-  AQ_CUDA(h, cudaMemcpyAsync(out_host, h->d_act, act_bytes, cudaMemcpyDeviceToHost, h->stream));
-  AQ_CUDA(h, cudaStreamSynchronize(h->stream));
+  AQ_CUDA(h, cudaEventRecord(h->ev_begin, h->stream));
+  AQ_CUDA(h, cudaStreamWaitEvent(h->in_stream, h->ev_begin, 0));
+  AQ_CUDA(h, cudaMemcpyAsync(h->d_ids, sample_ids_host, nb * sizeof(int32_t), cudaMemcpyHostToDevice, h->in_stream));
+  for (int i = 0; i < aq_handle::kSlices; ++i) {
+    size_t lo, cnt;
+    slice_of(h->n_batch, i, &lo, &cnt);
+    char* d_act = static_cast<char*>(h->d_act) + lo * act_b;
+    AQ_CUDA(h, cudaMemcpyAsync(h->d_packed + lo * packed_b, static_cast<const char*>(packed_host) + lo * packed_b, cnt * packed_b,
+                               cudaMemcpyHostToDevice, h->in_stream));
+    AQ_CUDA(h, cudaMemcpyAsync(h->d_scales + lo * (size_t)h->st.groups, reinterpret_cast<const char*>(scales_host) + lo * scales_b,
+                               cnt * scales_b, cudaMemcpyHostToDevice, h->in_stream));
+    if (raw_host)
+      AQ_CUDA(h, cudaMemcpyAsync(d_act, static_cast<const char*>(raw_host) + lo * act_b, cnt * act_b, cudaMemcpyHostToDevice, h->in_stream));
+    AQ_CUDA(h, cudaEventRecord(h->ev_in[i], h->in_stream));
+    AQ_CUDA(h, cudaStreamWaitEvent(h->stream, h->ev_in[i], 0));
+    const aq::DecodeArgs a{h->d_packed + lo * packed_b, h->d_scales + lo * (size_t)h->st.groups, raw_host ? d_act : nullptr,
+                           h->d_ids + lo, d_act, h->first_flags ? h->first_flags + lo : nullptr, (int)cnt};
+    rc = launch_decode_call(h, a);
+    if (rc != AQ_OK) return rc;
+    AQ_CUDA(h, cudaEventRecord(h->ev_done[i], h->stream));
+    AQ_CUDA(h, cudaStreamWaitEvent(h->out_stream, h->ev_done[i], 0));
+    AQ_CUDA(h, cudaMemcpyAsync(static_cast<char*>(out_host) + lo * act_b, d_act, cnt * act_b, cudaMemcpyDeviceToHost, h->out_stream));
+  }
+  AQ_CUDA(h, cudaStreamSynchronize(h->out_stream));
   return AQ_OK;
 }
 

@@ -257,6 +257,46 @@ def test_non_default_stream_and_host_buffer_forms():
         gr.close()
 
 
+@pytest.mark.parametrize("n_batch", [8, 11, 32])
+def test_host_buffer_forms_in_slices(n_batch):
+    """From 8 samples per call on, the host-buffer calls move the batch in four pieces whose copies
+    and kernels overlap (ragged pieces at 11); a call with a repeated or a bad id is not cut up,
+    so that the repeat is still found.  Every output, the first-visit flags and the state must be
+    those of the oracle either way."""
+    cfg = synth.Boundary("host-sliced", 64, n_batch, 5, 192, "fp16", 3, 64, 3, "normal", 0.05, seed=33)
+    gs, gr = GpuSide(cfg, n_batch), GpuSide(cfg, n_batch)
+    os_, or_ = (oracle.Side(64, 5, 192, 3, 64, oracle.FP16) for _ in range(2))
+    aq.aq_configure(gs.h, aq.AQ_ROUNDING, aq.AQ_ROUND_STOCHASTIC)
+    aq.aq_configure(gs.h, aq.AQ_SEED, 99)
+    try:
+        packed = torch.empty((n_batch, cfg.packed_bytes), dtype=torch.uint8).pin_memory()
+        scales = torch.empty((n_batch, cfg.groups), dtype=torch.float32).pin_memory()
+        out = torch.empty((n_batch, 5, 192), dtype=torch.float16).pin_memory()
+        for call in range(6):
+            aq.aq_configure(gs.h, aq.AQ_EPOCH, call)
+            os_.set_rounding(True, 99, call)
+            ids = synth.epoch_order(cfg, call)[:n_batch].clone()          # overlapping draws: first and later visits mixed
+            if call == 3:
+                ids[n_batch - 1] = ids[1]                                 # a repeat across two pieces
+            if call == 4:
+                ids[2] = 64                                               # out of range
+            act = synth.activation(cfg, torch.arange(n_batch), call).pin_memory()
+            packed.fill_(0xCD), scales.fill_(-1.0), out.fill_(7.0)
+            aq.aq_encode_host(gs.h, act, ids, packed, scales)
+            aq.aq_decode_host(gr.h, packed, scales, act, ids, out)
+            p_o, s_o, f_o = os_.encode(bits16(act), ids.numpy())
+            out_o, fr_o = or_.decode(p_o, s_o, ids.numpy(), raw=bits16(act))
+            assert np.array_equal(packed.numpy(), p_o) and np.array_equal(scales.numpy(), s_o), call
+            assert np.array_equal(bits16(out), out_o), call
+            assert np.array_equal(gs.first.cpu().numpy()[:n_batch], f_o), call
+            assert np.array_equal(gr.first.cpu().numpy()[:n_batch], fr_o), call
+            assert aq.aq_status(gs.h) == os_.status() and aq.aq_status(gr.h) == or_.status()
+        assert aq.aq_state_checksum(gs.h) == aq.aq_state_checksum(gr.h) == os_.checksum() == or_.checksum()
+        assert np.array_equal(gs.m_all(), os_.m()) and np.array_equal(gr.m_all(), or_.m())
+    finally:
+        gs.close(), gr.close(), os_.close(), or_.close()
+
+
 def test_import_export_round_trip():
     cfg = synth.Boundary("ckpt", 3, 1, 4, 64, "fp16", 4, 64, 1, "normal", 0.1, seed=8)
     a, b = GpuSide(cfg, 1), GpuSide(cfg, 1)
