@@ -139,7 +139,8 @@ aq_handle* aq_create_hosted(int64_t n_samples, int seq, int hidden, int bits, in
  * critical path).  sample_ids_host int32[n] (host; copied before the call returns), n must equal
  * AQ_BATCH now and at that call.  The call returns at once; on a copy stream of the handle's
  * own, behind everything issued so far on the handle's stream, each sample's row of m is copied
- * into a staging block in device memory (n rows, allocated at the first use and when n grows).
+ * into a staging block in device memory (n rows, allocated at the first use and when n grows):
+ * by one copy per row, or by one kernel when there are more than 64 rows or rows under 64 KB.
  * The next aq_encode / aq_decode (aq_encode_host / aq_decode_host too) then
  *   - waits on the device, not on the host, until the rows have arrived,
  *   - runs the same kernel on the staged rows at device-memory speed, with the same results as

@@ -33,6 +33,8 @@ struct aq_handle {
   cudaEvent_t ev_written = nullptr;          // copy_stream: its rows are back in host memory
   void* slots = nullptr;                     // T[slots_batch][elems]
   int32_t* d_slot_ids = nullptr;             // [slots_batch] ids as given to aq_prefetch
+  int32_t* d_copy_ids = nullptr;             // [slots_batch] the same with -1 where no row is to be moved
+  bool rows_by_kernel = false;               // how the pending prefetch's rows travel (see aq_prefetch)
   int slots_batch = 0;
   std::vector<int32_t> staged_ids;           // per slot: the sample whose row it holds, -1 = nothing to copy
   // the ids travel to d_slot_ids from page-locked blocks used in turn (a pageable source would
@@ -164,11 +166,15 @@ int run_staged(aq_handle* h, Launch launch) {
   AQ_CUDA(h, cudaEventRecord(h->ev_computed, h->stream));
   AQ_CUDA(h, cudaStreamWaitEvent(h->copy_stream, h->ev_computed, 0));
   const size_t bytes = (size_t)h->st.m_bytes;
-  for (size_t j = 0; j < h->staged_ids.size(); ++j) {
-    const int32_t id = h->staged_ids[j];
-    if (id < 0) continue;
-    AQ_CUDA(h, cudaMemcpyAsync(static_cast<char*>(h->m_host) + (size_t)id * bytes,
-                               static_cast<const char*>(h->slots) + j * bytes, bytes, cudaMemcpyDeviceToHost, h->copy_stream));
+  if (h->rows_by_kernel) {
+    AQ_CUDA(h, aq::launch_copy_rows(h->slots, h->st.m, h->d_copy_ids, h->n_batch, (long long)bytes, false, h->copy_stream));
+  } else {
+    for (size_t j = 0; j < h->staged_ids.size(); ++j) {
+      const int32_t id = h->staged_ids[j];
+      if (id < 0) continue;
+      AQ_CUDA(h, cudaMemcpyAsync(static_cast<char*>(h->m_host) + (size_t)id * bytes,
+                                 static_cast<const char*>(h->slots) + j * bytes, bytes, cudaMemcpyDeviceToHost, h->copy_stream));
+    }
   }
   AQ_CUDA(h, cudaEventRecord(h->ev_written, h->copy_stream));
   h->writeback_issued = true;
@@ -242,7 +248,7 @@ static aq_handle* create_handle(int64_t n_samples, int seq, int hidden, int bits
     for (cudaEvent_t* ev : {&h->ev_settled, &h->ev_staged, &h->ev_computed, &h->ev_written})
       if (e == cudaSuccess) e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming);
     for (int i = 0; i < aq_handle::kIdRing; ++i) {
-      if (e == cudaSuccess) e = cudaHostAlloc(reinterpret_cast<void**>(&h->ids_pinned[i]), aq::kMaxBatch * sizeof(int32_t), cudaHostAllocPortable);
+      if (e == cudaSuccess) e = cudaHostAlloc(reinterpret_cast<void**>(&h->ids_pinned[i]), 2 * aq::kMaxBatch * sizeof(int32_t), cudaHostAllocPortable);
       if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_ids_sent[i], cudaEventDisableTiming);
     }
   }
@@ -282,7 +288,7 @@ void aq_destroy(aq_handle* h) {
     cudaStreamDestroy(h->copy_stream);
     cudaEventDestroy(h->ev_settled); cudaEventDestroy(h->ev_staged);
     cudaEventDestroy(h->ev_computed); cudaEventDestroy(h->ev_written);
-    cudaFree(h->slots); cudaFree(h->d_slot_ids);
+    cudaFree(h->slots); cudaFree(h->d_slot_ids); cudaFree(h->d_copy_ids);
     for (int i = 0; i < aq_handle::kIdRing; ++i) {
       cudaFreeHost(h->ids_pinned[i]);
       cudaEventDestroy(h->ev_ids_sent[i]);
@@ -573,10 +579,11 @@ int aq_prefetch(aq_handle* h, const int32_t* sample_ids_host, int n) {
   if (h->slots_batch < n) {
     AQ_CUDA(h, cudaStreamSynchronize(h->copy_stream));
     AQ_CUDA(h, cudaStreamSynchronize(h->stream));
-    cudaFree(h->slots); cudaFree(h->d_slot_ids);
-    h->slots = nullptr; h->d_slot_ids = nullptr; h->slots_batch = 0;
+    cudaFree(h->slots); cudaFree(h->d_slot_ids); cudaFree(h->d_copy_ids);
+    h->slots = nullptr; h->d_slot_ids = nullptr; h->d_copy_ids = nullptr; h->slots_batch = 0;
     AQ_CUDA(h, cudaMalloc(&h->slots, (size_t)n * bytes));
     AQ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&h->d_slot_ids), (size_t)n * sizeof(int32_t)));
+    AQ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&h->d_copy_ids), (size_t)n * sizeof(int32_t)));
     h->slots_batch = n;
   }
   // rows to move: every id once (the kernels skip an id's later occurrences and ids out of range)
@@ -591,14 +598,25 @@ int aq_prefetch(aq_handle* h, const int32_t* sample_ids_host, int n) {
   AQ_CUDA(h, cudaStreamWaitEvent(h->copy_stream, h->ev_settled, 0));
   const int ring = (int)(h->prefetches++ % aq_handle::kIdRing);
   AQ_CUDA(h, cudaEventSynchronize(h->ev_ids_sent[ring]));      // long done, unless kIdRing prefetches are queued
+  int32_t* copy_ids_pinned = h->ids_pinned[ring] + aq::kMaxBatch;
   memcpy(h->ids_pinned[ring], sample_ids_host, (size_t)n * sizeof(int32_t));
+  memcpy(copy_ids_pinned, h->staged_ids.data(), (size_t)n * sizeof(int32_t));
   AQ_CUDA(h, cudaMemcpyAsync(h->d_slot_ids, h->ids_pinned[ring], (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice, h->copy_stream));
+  AQ_CUDA(h, cudaMemcpyAsync(h->d_copy_ids, copy_ids_pinned, (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice, h->copy_stream));
   AQ_CUDA(h, cudaEventRecord(h->ev_ids_sent[ring], h->copy_stream));
-  for (int j = 0; j < n; ++j) {
-    const int32_t id = h->staged_ids[j];
-    if (id < 0) continue;
-    AQ_CUDA(h, cudaMemcpyAsync(static_cast<char*>(h->slots) + (size_t)j * bytes,
-                               static_cast<const char*>(h->m_host) + (size_t)id * bytes, bytes, cudaMemcpyHostToDevice, h->copy_stream));
+  // a few large rows: one copy per row through the copy engines, the faster way over the host
+  // link; many rows or small ones: one kernel that reads the mapped host block, since a copy
+  // call costs microseconds of host time each
+  h->rows_by_kernel = n > 64 || bytes < (64u << 10);
+  if (h->rows_by_kernel) {
+    AQ_CUDA(h, aq::launch_copy_rows(h->st.m, h->slots, h->d_copy_ids, n, (long long)bytes, true, h->copy_stream));
+  } else {
+    for (int j = 0; j < n; ++j) {
+      const int32_t id = h->staged_ids[j];
+      if (id < 0) continue;
+      AQ_CUDA(h, cudaMemcpyAsync(static_cast<char*>(h->slots) + (size_t)j * bytes,
+                                 static_cast<const char*>(h->m_host) + (size_t)id * bytes, bytes, cudaMemcpyHostToDevice, h->copy_stream));
+    }
   }
   AQ_CUDA(h, cudaEventRecord(h->ev_staged, h->copy_stream));
   h->prefetch_pending = true;

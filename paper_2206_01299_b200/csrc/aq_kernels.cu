@@ -280,6 +280,32 @@ __global__ void __launch_bounds__(kThreads) dequant_grad_kernel(const uint8_t* _
   }
 }
 
+// ------------------------------------------------------------------ rows between a store and a staging block
+
+constexpr int kCopyPiecesPerThread = 4;
+
+__global__ void __launch_bounds__(kThreads) copy_rows_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst,
+                                                             const int32_t* __restrict__ ids, long long row_pieces,
+                                                             bool gather) {
+  const int y = blockIdx.y;
+  const long long id = ids[y];
+  if (id < 0) return;
+  const uint4* from = src + (gather ? id : (long long)y) * row_pieces;
+  uint4* to = dst + (gather ? (long long)y : id) * row_pieces;
+  const long long p0 = (long long)blockIdx.x * (kThreads * kCopyPiecesPerThread) + threadIdx.x;
+  uint4 v[kCopyPiecesPerThread];
+#pragma unroll
+  for (int i = 0; i < kCopyPiecesPerThread; ++i) {
+    const long long p = p0 + i * kThreads;
+    if (p < row_pieces) v[i] = from[p];
+  }
+#pragma unroll
+  for (int i = 0; i < kCopyPiecesPerThread; ++i) {
+    const long long p = p0 + i * kThreads;
+    if (p < row_pieces) to[p] = v[i];
+  }
+}
+
 // ------------------------------------------------------------------ state digest
 
 __device__ __forceinline__ unsigned long long mix64(unsigned long long index, unsigned long long word) {
@@ -420,6 +446,16 @@ cudaError_t launch_dequant_grad(int dtype, int bits, int lanes_per_group, const 
   return launch_overlapped(dequant_grad_kernel<T, B>, dim3(grid), s, packed, scales, chunks, lanes_per_group, reinterpret_cast<T*>(out))
   AQ_DISPATCH(dtype, bits, AQ_CALL)
 #undef AQ_CALL
+  return cudaGetLastError();
+}
+
+cudaError_t launch_copy_rows(const void* src, void* dst, const int32_t* ids, int n, long long row_bytes, bool gather,
+                             cudaStream_t s) {
+  if (n <= 0 || row_bytes <= 0) return cudaSuccess;
+  const long long pieces = row_bytes / 16;
+  const long long per_cta = (long long)kThreads * kCopyPiecesPerThread;
+  const dim3 grid((unsigned)((pieces + per_cta - 1) / per_cta), (unsigned)n);
+  copy_rows_kernel<<<grid, kThreads, 0, s>>>(static_cast<const uint4*>(src), static_cast<uint4*>(dst), ids, pieces, gather);
   return cudaGetLastError();
 }
 

@@ -37,6 +37,16 @@ def test_same_samples_in_consecutive_prefetched_calls():
     run_boundary(cfg, hosted=True, prefetch=lambda k: True)
 
 
+def test_prefetch_of_many_rows_goes_through_one_kernel():
+    """More than 64 rows, or rows below 64 KB, are gathered into the staging block and scattered
+    back by one kernel over the mapped host block instead of one copy per row: the largest batch
+    of the smallest samples, and a hundred rows of 96 KB."""
+    cfg = synth.Boundary("staged-wide", 4096, 4096, 1, 64, "fp16", 4, 64, 2, "normal", 0.1, seed=517)
+    run_boundary(cfg, hosted=True, prefetch=lambda k: True, check_all_m=False)
+    cfg = synth.Boundary("staged-hundred", 200, 100, 32, 1536, "bf16", 2, 128, 3, "student_t3", 0.02, seed=518)
+    run_boundary(cfg, hosted=True, prefetch=lambda k: k != 2, check_all_m=False)
+
+
 def test_prefetch_of_bad_and_repeated_ids():
     cfg = synth.Boundary("staged-ids", 8, 6, 4, 64, "fp16", 4, 64, 3, "normal", 0.1, seed=514)
     gs, gr = GpuSide(cfg, 6, hosted=True), GpuSide(cfg, 6, hosted=True)
