@@ -287,9 +287,14 @@ def main():
 
     if args.prefetch and not args.hosted:
         raise SystemExit("--prefetch needs --hosted")
+    if args.hosted and args.m_bits == 32:
+        raise SystemExit("the binary32 store is not offered in host memory")
+    if args.prefetch and args.m_bits:
+        raise SystemExit("--prefetch is built for the 16-bit store")
     handles = []
     for _ in range(2):
-        h = (aq.aq_create_fp32(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group) if args.m_bits == 32
+        h = (aq.aq_create_hosted_lowbit(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, args.m_bits) if args.m_bits in (2, 4, 8) and args.hosted
+             else aq.aq_create_fp32(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group) if args.m_bits == 32
              else aq.aq_create_lowbit(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, args.m_bits) if args.m_bits
              else aq.aq_create_hosted(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group) if args.hosted
              else aq.aq_create(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group))

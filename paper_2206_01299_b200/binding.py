@@ -24,6 +24,7 @@ SIGNATURES = {
     "aq_create_hosted": (C.c_void_p, [C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int]),
     "aq_create_fp32": (C.c_void_p, [C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int]),
     "aq_create_lowbit": (C.c_void_p, [C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int]),
+    "aq_create_hosted_lowbit": (C.c_void_p, [C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int]),
     "aq_destroy": (None, [C.c_void_p]),
     "aq_configure": (C.c_int, [C.c_void_p, C.c_int, C.c_int64]),
     "aq_encode": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -113,6 +114,13 @@ def aq_create_fp32(n_samples, seq, hidden, bits, group):
 
 def aq_create_lowbit(n_samples, seq, hidden, bits, group, m_bits):
     h = lib().aq_create_lowbit(n_samples, seq, hidden, bits, group, m_bits)
+    if not h:
+        raise AqError(AQ_EINVAL, aq_last_error(None))
+    return h
+
+
+def aq_create_hosted_lowbit(n_samples, seq, hidden, bits, group, m_bits):
+    h = lib().aq_create_hosted_lowbit(n_samples, seq, hidden, bits, group, m_bits)
     if not h:
         raise AqError(AQ_EINVAL, aq_last_error(None))
     return h

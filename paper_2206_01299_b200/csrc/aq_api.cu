@@ -24,6 +24,7 @@ struct aq_handle {
   uint8_t* first_flags = nullptr;
   unsigned long long* sum_dev = nullptr;     // scratch of aq_state_checksum
   void* m_host = nullptr;                    // hosted store: the pinned host block that st.m maps
+  float* m_scales_host = nullptr;            // ... and the one that st.m_scales maps (low-precision hosted store)
   // hosted store, staged visits: aq_prefetch copies the next call's m(xi) into `slots` on
   // copy_stream, the call works there and copies the rows back on copy_stream afterwards
   cudaStream_t copy_stream = nullptr;
@@ -196,6 +197,15 @@ aq_handle* aq_create_hosted(int64_t n_samples, int seq, int hidden, int bits, in
   return create_handle(n_samples, seq, hidden, bits, group, 0, true);
 }
 
+aq_handle* aq_create_hosted_lowbit(int64_t n_samples, int seq, int hidden, int bits, int group, int m_bits) {
+  if (m_bits != 2 && m_bits != 4 && m_bits != 8) {
+    g_create_err[0] = 0;
+    fail(nullptr, AQ_EINVAL, "m_bits must be 2, 4 or 8 (got %d)", m_bits);
+    return nullptr;
+  }
+  return create_handle(n_samples, seq, hidden, bits, group, m_bits, true);
+}
+
 aq_handle* aq_create_fp32(int64_t n_samples, int seq, int hidden, int bits, int group) {
   return create_handle(n_samples, seq, hidden, bits, group, 32);
 }
@@ -256,10 +266,15 @@ static aq_handle* create_handle(int64_t n_samples, int seq, int hidden, int bits
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&st.arrivals), sizeof(unsigned long long));
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&st.status), sizeof(uint32_t));
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&h->sum_dev), sizeof(unsigned long long));
-  if (e == cudaSuccess && m_steps) e = cudaMalloc(reinterpret_cast<void**>(&st.m_scales), m_scale_bytes);
+  if (e == cudaSuccess && m_steps && !hosted) e = cudaMalloc(reinterpret_cast<void**>(&st.m_scales), m_scale_bytes);
+  if (e == cudaSuccess && m_steps && hosted) {
+    e = cudaHostAlloc(reinterpret_cast<void**>(&h->m_scales_host), m_scale_bytes, cudaHostAllocMapped | cudaHostAllocPortable);
+    if (e == cudaSuccess) e = cudaHostGetDevicePointer(reinterpret_cast<void**>(&st.m_scales), h->m_scales_host, 0);
+  }
   if (e == cudaSuccess && !hosted) e = cudaMemset(st.m, 0, m_bytes);           // "initialized to 0"
   if (e == cudaSuccess && hosted) memset(h->m_host, 0, m_bytes);
-  if (e == cudaSuccess && m_steps) e = cudaMemset(st.m_scales, 0, m_scale_bytes);
+  if (e == cudaSuccess && m_steps && !hosted) e = cudaMemset(st.m_scales, 0, m_scale_bytes);
+  if (e == cudaSuccess && m_steps && hosted) memset(h->m_scales_host, 0, m_scale_bytes);
   if (e == cudaSuccess) e = cudaMemset(st.seen, 0, seen_bytes);
   if (e == cudaSuccess) e = cudaMemset(st.status, 0, sizeof(uint32_t));
   if (e == cudaSuccess) e = cudaMemset(st.arrivals, 0, sizeof(unsigned long long));
@@ -296,7 +311,8 @@ void aq_destroy(aq_handle* h) {
   }
   if (h->m_host) cudaFreeHost(h->m_host);
   else cudaFree(h->st.m);
-  cudaFree(h->st.m_scales);
+  if (h->m_scales_host) cudaFreeHost(h->m_scales_host);
+  else cudaFree(h->st.m_scales);
   cudaFree(h->st.seen);
   cudaFree(h->st.arrivals);
   cudaFree(h->st.status);
@@ -571,6 +587,7 @@ int aq_decode_host(aq_handle* h, const void* packed_host, const float* scales_ho
 int aq_prefetch(aq_handle* h, const int32_t* sample_ids_host, int n) {
   if (!h) return fail(nullptr, AQ_EINVAL, "null handle");
   if (!h->m_host) return fail(h, AQ_EUNSUPPORTED, "aq_prefetch: the handle keeps m in device memory (see aq_create_hosted)");
+  if (h->st.m_bits) return fail(h, AQ_EUNSUPPORTED, "aq_prefetch: staged visits are built for the 16-bit store only");
   if (n != h->n_batch) return fail(h, AQ_EINVAL, "aq_prefetch: n must equal AQ_BATCH (%d), got %d", h->n_batch, n);
   if (n == 0) return AQ_OK;
   if (!sample_ids_host) return fail(h, AQ_EINVAL, "aq_prefetch: null pointer");

@@ -13,9 +13,10 @@ pytestmark = pytest.mark.gpu
 
 
 class LowSide:
-    def __init__(self, cfg, n_batch, m_bits):
+    def __init__(self, cfg, n_batch, m_bits, hosted=False):
         self.cfg, self.m_bits = cfg, m_bits
-        self.h = (aq.aq_create_fp32(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group) if m_bits == 32
+        self.h = (aq.aq_create_hosted_lowbit(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, m_bits) if hosted
+                  else aq.aq_create_fp32(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group) if m_bits == 32
                   else aq.aq_create_lowbit(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, m_bits))
         aq.aq_configure(self.h, aq.AQ_DTYPE, DT[cfg.dtype][0])
         aq.aq_configure(self.h, aq.AQ_BATCH, n_batch)
@@ -42,9 +43,9 @@ class LowSide:
         return codes, steps, seen
 
 
-def run_lowbit(cfg, m_bits, n_batch=None, stochastic_seed=None):
+def run_lowbit(cfg, m_bits, n_batch=None, stochastic_seed=None, hosted=False):
     nb = n_batch or cfg.n_batch
-    gs, gr = LowSide(cfg, nb, m_bits), LowSide(cfg, nb, m_bits)
+    gs, gr = LowSide(cfg, nb, m_bits, hosted), LowSide(cfg, nb, m_bits, hosted)
     od = DT[cfg.dtype][1]
     os_, or_ = (oracle.SideLow(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, od, m_bits) for _ in range(2))
     packed = torch.empty((nb, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
@@ -100,6 +101,24 @@ def test_large_shapes_reduced_id_space(m_bits):
     run_lowbit(synth.shrink(synth.GPT2_XL, 8, seq=96, epochs=3), m_bits, n_batch=4)
     run_lowbit(synth.shrink(synth.DEBERTA_XXL, 16, seq=40), m_bits)
     run_lowbit(synth.shrink(synth.SWEEP_FWD, 4, seq=64), m_bits)
+
+
+@pytest.mark.parametrize("m_bits", [2, 4, 8])
+def test_low_precision_store_in_host_memory(m_bits):
+    """Codes and steps in page-locked host memory: the same kernels on mapped pointers, the same
+    results, checkpoint reads and digest included; no staged visits for this store."""
+    run_lowbit(synth.TINY, m_bits, hosted=True)
+    run_lowbit(synth.shrink(synth.GPT2_XL, 8, seq=96, epochs=3), m_bits, n_batch=4, hosted=True, stochastic_seed=21)
+    h = aq.aq_create_hosted_lowbit(4, 2, 64, 4, 64, m_bits)
+    try:
+        with pytest.raises(aq.AqError) as e:
+            aq.aq_prefetch(h, torch.zeros(1, dtype=torch.int32))
+        assert e.value.code == aq.AQ_EUNSUPPORTED
+    finally:
+        aq.aq_destroy(h)
+    for not_offered in (16, 32):
+        with pytest.raises(aq.AqError):
+            aq.aq_create_hosted_lowbit(4, 2, 64, 4, 64, not_offered)
 
 
 @pytest.mark.parametrize("m_bits", [2, 4, 8, 32])
