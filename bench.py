@@ -289,8 +289,6 @@ def main():
         raise SystemExit("--prefetch needs --hosted")
     if args.hosted and args.m_bits == 32:
         raise SystemExit("the binary32 store is not offered in host memory")
-    if args.prefetch and args.m_bits:
-        raise SystemExit("--prefetch is built for the 16-bit store")
     handles = []
     for _ in range(2):
         h = (aq.aq_create_hosted_lowbit(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, args.m_bits) if args.m_bits in (2, 4, 8) and args.hosted

@@ -185,7 +185,7 @@ aq_handle* aq_create_fp32(int64_t n_samples, int seq, int hidden, int bits, int 
  * Both at once: the store of aq_create_lowbit (m_bits 2, 4 or 8) kept in page-locked host
  * memory as for aq_create_hosted -- codes and steps alike.  An 8-bit store moves 1.06 instead of
  * 2 bytes per element over the host link in each direction.  The calls work on the host block
- * in place; aq_prefetch answers AQ_EUNSUPPORTED.  (Not offered for the binary32 store: its
+ * in place, or after aq_prefetch on staged rows (codes and steps).  (Not offered for the binary32 store: its
  * kernels read two 16-byte pieces 32 bytes apart per thread, which device memory serves at full
  * speed and the host link at a fifth of it.)
  */

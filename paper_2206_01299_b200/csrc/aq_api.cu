@@ -32,7 +32,8 @@ struct aq_handle {
   cudaEvent_t ev_staged = nullptr;           // copy_stream: the prefetched rows are in HBM
   cudaEvent_t ev_computed = nullptr;         // the handle's stream: the call that used them is done
   cudaEvent_t ev_written = nullptr;          // copy_stream: its rows are back in host memory
-  void* slots = nullptr;                     // T[slots_batch][elems]
+  void* slots = nullptr;                     // [slots_batch] rows of m (16-bit values, or the codes of a low-precision store)
+  float* slot_scales = nullptr;              // [slots_batch][groups] steps of those rows (low-precision store)
   int32_t* d_slot_ids = nullptr;             // [slots_batch] ids as given to aq_prefetch
   int32_t* d_copy_ids = nullptr;             // [slots_batch] the same with -1 where no row is to be moved
   bool rows_by_kernel = false;               // how the pending prefetch's rows travel (see aq_prefetch)
@@ -153,6 +154,35 @@ cudaError_t settle(aq_handle* h) {
   return cudaStreamWaitEvent(h->stream, h->ev_written, 0);
 }
 
+// The rows of the pending prefetch between the host blocks and the staging blocks, on
+// copy_stream: in = host to staging.  A low-precision store has two blocks, codes and steps.
+int move_rows(aq_handle* h, bool in) {
+  const int n = (int)h->staged_ids.size();
+  const size_t bytes = (size_t)h->st.m_bytes, step_bytes = (size_t)h->st.groups * sizeof(float);
+  const cudaMemcpyKind kind = in ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToHost;
+  if (h->rows_by_kernel) {
+    AQ_CUDA(h, aq::launch_copy_rows(in ? h->st.m : h->slots, in ? h->slots : h->st.m, h->d_copy_ids, n, (long long)bytes, in,
+                                    h->copy_stream));
+    if (h->m_scales_host)
+      AQ_CUDA(h, aq::launch_copy_rows(in ? h->st.m_scales : h->slot_scales, in ? h->slot_scales : h->st.m_scales, h->d_copy_ids,
+                                      n, (long long)step_bytes, in, h->copy_stream));
+    return AQ_OK;
+  }
+  for (int j = 0; j < n; ++j) {
+    const int32_t id = h->staged_ids[j];
+    if (id < 0) continue;
+    char* host_row = static_cast<char*>(h->m_host) + (size_t)id * bytes;
+    char* slot_row = static_cast<char*>(h->slots) + (size_t)j * bytes;
+    AQ_CUDA(h, cudaMemcpyAsync(in ? slot_row : host_row, in ? host_row : slot_row, bytes, kind, h->copy_stream));
+    if (h->m_scales_host) {
+      float* host_steps = h->m_scales_host + (size_t)id * (size_t)h->st.groups;
+      float* slot_steps = h->slot_scales + (size_t)j * (size_t)h->st.groups;
+      AQ_CUDA(h, cudaMemcpyAsync(in ? slot_steps : host_steps, in ? host_steps : slot_steps, step_bytes, kind, h->copy_stream));
+    }
+  }
+  return AQ_OK;
+}
+
 // A staged call: `launch` runs on the prefetched rows in HBM, then the rows go home.
 template <typename Launch>
 int run_staged(aq_handle* h, Launch launch) {
@@ -161,22 +191,14 @@ int run_staged(aq_handle* h, Launch launch) {
     return fail(h, AQ_EINVAL, "the pending aq_prefetch was for %d samples, AQ_BATCH is %d", (int)h->staged_ids.size(), h->n_batch);
   aq::State st = h->st;
   st.m = h->slots;
+  if (h->m_scales_host) st.m_scales = h->slot_scales;
   st.slot_ids = h->d_slot_ids;
   AQ_CUDA(h, cudaStreamWaitEvent(h->stream, h->ev_staged, 0));
   AQ_CUDA(h, launch(st));
   AQ_CUDA(h, cudaEventRecord(h->ev_computed, h->stream));
   AQ_CUDA(h, cudaStreamWaitEvent(h->copy_stream, h->ev_computed, 0));
-  const size_t bytes = (size_t)h->st.m_bytes;
-  if (h->rows_by_kernel) {
-    AQ_CUDA(h, aq::launch_copy_rows(h->slots, h->st.m, h->d_copy_ids, h->n_batch, (long long)bytes, false, h->copy_stream));
-  } else {
-    for (size_t j = 0; j < h->staged_ids.size(); ++j) {
-      const int32_t id = h->staged_ids[j];
-      if (id < 0) continue;
-      AQ_CUDA(h, cudaMemcpyAsync(static_cast<char*>(h->m_host) + (size_t)id * bytes,
-                                 static_cast<const char*>(h->slots) + j * bytes, bytes, cudaMemcpyDeviceToHost, h->copy_stream));
-    }
-  }
+  const int rc = move_rows(h, false);
+  if (rc != AQ_OK) return rc;
   AQ_CUDA(h, cudaEventRecord(h->ev_written, h->copy_stream));
   h->writeback_issued = true;
   return AQ_OK;
@@ -303,7 +325,7 @@ void aq_destroy(aq_handle* h) {
     cudaStreamDestroy(h->copy_stream);
     cudaEventDestroy(h->ev_settled); cudaEventDestroy(h->ev_staged);
     cudaEventDestroy(h->ev_computed); cudaEventDestroy(h->ev_written);
-    cudaFree(h->slots); cudaFree(h->d_slot_ids); cudaFree(h->d_copy_ids);
+    cudaFree(h->slots); cudaFree(h->slot_scales); cudaFree(h->d_slot_ids); cudaFree(h->d_copy_ids);
     for (int i = 0; i < aq_handle::kIdRing; ++i) {
       cudaFreeHost(h->ids_pinned[i]);
       cudaEventDestroy(h->ev_ids_sent[i]);
@@ -362,21 +384,21 @@ int aq_configure(aq_handle* h, int key, int64_t value) {
 }
 
 static int launch_encode_call(aq_handle* h, const aq::EncodeArgs& a) {
+  AQ_CUDA(h, settle(h));
   if (h->st.m_bits) {
     AQ_CUDA(h, aq::launch_encode_lowbit(h->dtype, h->bits, h->st, a, h->stream));
     return AQ_OK;
   }
-  AQ_CUDA(h, settle(h));
   AQ_CUDA(h, aq::launch_encode(h->dtype, h->bits, h->st, a, h->stream));
   return AQ_OK;
 }
 
 static int launch_decode_call(aq_handle* h, const aq::DecodeArgs& a) {
+  AQ_CUDA(h, settle(h));
   if (h->st.m_bits) {
     AQ_CUDA(h, aq::launch_decode_lowbit(h->dtype, h->bits, h->st, a, h->stream));
     return AQ_OK;
   }
-  AQ_CUDA(h, settle(h));
   AQ_CUDA(h, aq::launch_decode(h->dtype, h->bits, h->st, a, h->stream));
   return AQ_OK;
 }
@@ -390,8 +412,11 @@ int aq_encode(aq_handle* h, const void* act, const int32_t* sample_ids, void* pa
   DeviceGuard g(h->device);
   aq::EncodeArgs a{act, sample_ids, static_cast<uint8_t*>(packed), scales, h->first_flags, h->n_batch,
                    h->rounding == AQ_ROUND_STOCHASTIC, h->seed, h->epoch};
-  if (h->prefetch_pending && !h->st.m_bits)
-    return run_staged(h, [&](const aq::State& st) { return aq::launch_encode(h->dtype, h->bits, st, a, h->stream); });
+  if (h->prefetch_pending)
+    return run_staged(h, [&](const aq::State& st) {
+      return h->st.m_bits ? aq::launch_encode_lowbit(h->dtype, h->bits, st, a, h->stream)
+                          : aq::launch_encode(h->dtype, h->bits, st, a, h->stream);
+    });
   return launch_encode_call(h, a);
 }
 
@@ -403,8 +428,11 @@ int aq_decode(aq_handle* h, const void* packed, const float* scales, const int32
     return fail(h, AQ_EINVAL, "aq_decode: packed, scales and out must be 16-byte aligned");
   DeviceGuard g(h->device);
   aq::DecodeArgs a{static_cast<const uint8_t*>(packed), scales, h->raw, sample_ids, out, h->first_flags, h->n_batch};
-  if (h->prefetch_pending && !h->st.m_bits)
-    return run_staged(h, [&](const aq::State& st) { return aq::launch_decode(h->dtype, h->bits, st, a, h->stream); });
+  if (h->prefetch_pending)
+    return run_staged(h, [&](const aq::State& st) {
+      return h->st.m_bits ? aq::launch_decode_lowbit(h->dtype, h->bits, st, a, h->stream)
+                          : aq::launch_decode(h->dtype, h->bits, st, a, h->stream);
+    });
   return launch_decode_call(h, a);
 }
 
@@ -587,7 +615,6 @@ int aq_decode_host(aq_handle* h, const void* packed_host, const float* scales_ho
 int aq_prefetch(aq_handle* h, const int32_t* sample_ids_host, int n) {
   if (!h) return fail(nullptr, AQ_EINVAL, "null handle");
   if (!h->m_host) return fail(h, AQ_EUNSUPPORTED, "aq_prefetch: the handle keeps m in device memory (see aq_create_hosted)");
-  if (h->st.m_bits) return fail(h, AQ_EUNSUPPORTED, "aq_prefetch: staged visits are built for the 16-bit store only");
   if (n != h->n_batch) return fail(h, AQ_EINVAL, "aq_prefetch: n must equal AQ_BATCH (%d), got %d", h->n_batch, n);
   if (n == 0) return AQ_OK;
   if (!sample_ids_host) return fail(h, AQ_EINVAL, "aq_prefetch: null pointer");
@@ -596,9 +623,11 @@ int aq_prefetch(aq_handle* h, const int32_t* sample_ids_host, int n) {
   if (h->slots_batch < n) {
     AQ_CUDA(h, cudaStreamSynchronize(h->copy_stream));
     AQ_CUDA(h, cudaStreamSynchronize(h->stream));
-    cudaFree(h->slots); cudaFree(h->d_slot_ids); cudaFree(h->d_copy_ids);
-    h->slots = nullptr; h->d_slot_ids = nullptr; h->d_copy_ids = nullptr; h->slots_batch = 0;
+    cudaFree(h->slots); cudaFree(h->slot_scales); cudaFree(h->d_slot_ids); cudaFree(h->d_copy_ids);
+    h->slots = nullptr; h->slot_scales = nullptr; h->d_slot_ids = nullptr; h->d_copy_ids = nullptr; h->slots_batch = 0;
     AQ_CUDA(h, cudaMalloc(&h->slots, (size_t)n * bytes));
+    if (h->m_scales_host)
+      AQ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&h->slot_scales), (size_t)n * (size_t)h->st.groups * sizeof(float)));
     AQ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&h->d_slot_ids), (size_t)n * sizeof(int32_t)));
     AQ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&h->d_copy_ids), (size_t)n * sizeof(int32_t)));
     h->slots_batch = n;
@@ -625,16 +654,8 @@ int aq_prefetch(aq_handle* h, const int32_t* sample_ids_host, int n) {
   // link; many rows or small ones: one kernel that reads the mapped host block, since a copy
   // call costs microseconds of host time each
   h->rows_by_kernel = n > 64 || bytes < (64u << 10);
-  if (h->rows_by_kernel) {
-    AQ_CUDA(h, aq::launch_copy_rows(h->st.m, h->slots, h->d_copy_ids, n, (long long)bytes, true, h->copy_stream));
-  } else {
-    for (int j = 0; j < n; ++j) {
-      const int32_t id = h->staged_ids[j];
-      if (id < 0) continue;
-      AQ_CUDA(h, cudaMemcpyAsync(static_cast<char*>(h->slots) + (size_t)j * bytes,
-                                 static_cast<const char*>(h->m_host) + (size_t)id * bytes, bytes, cudaMemcpyHostToDevice, h->copy_stream));
-    }
-  }
+  const int rc = move_rows(h, true);
+  if (rc != AQ_OK) return rc;
   AQ_CUDA(h, cudaEventRecord(h->ev_staged, h->copy_stream));
   h->prefetch_pending = true;
   return AQ_OK;

@@ -73,7 +73,7 @@ cudaError_t launch_quant_grad(int dtype, int bits, int lanes_per_group, const vo
                               unsigned long long seed, unsigned long long epoch, cudaStream_t s);
 cudaError_t launch_dequant_grad(int dtype, int bits, int lanes_per_group, const uint8_t* packed,
                                 const float* scales, long long n_elems, void* out, cudaStream_t s);
-// Rows of `row_bytes` bytes (a multiple of 16) moved by one kernel: gather: dst row y <- src row
+// Rows of `row_bytes` bytes moved by one kernel (in 16-, 4- or 1-byte pieces, as the size and the bases allow): gather: dst row y <- src row
 // ids[y]; scatter: dst row ids[y] <- src row y; entries with ids[y] < 0 are left out.
 cudaError_t launch_copy_rows(const void* src, void* dst, const int32_t* ids, int n, long long row_bytes, bool gather,
                              cudaStream_t s);

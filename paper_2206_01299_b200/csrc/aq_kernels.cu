@@ -284,16 +284,17 @@ __global__ void __launch_bounds__(kThreads) dequant_grad_kernel(const uint8_t* _
 
 constexpr int kCopyPiecesPerThread = 4;
 
-__global__ void __launch_bounds__(kThreads) copy_rows_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst,
+template <typename Piece>
+__global__ void __launch_bounds__(kThreads) copy_rows_kernel(const Piece* __restrict__ src, Piece* __restrict__ dst,
                                                              const int32_t* __restrict__ ids, long long row_pieces,
                                                              bool gather) {
   const int y = blockIdx.y;
   const long long id = ids[y];
   if (id < 0) return;
-  const uint4* from = src + (gather ? id : (long long)y) * row_pieces;
-  uint4* to = dst + (gather ? (long long)y : id) * row_pieces;
+  const Piece* from = src + (gather ? id : (long long)y) * row_pieces;
+  Piece* to = dst + (gather ? (long long)y : id) * row_pieces;
   const long long p0 = (long long)blockIdx.x * (kThreads * kCopyPiecesPerThread) + threadIdx.x;
-  uint4 v[kCopyPiecesPerThread];
+  Piece v[kCopyPiecesPerThread];
 #pragma unroll
   for (int i = 0; i < kCopyPiecesPerThread; ++i) {
     const long long p = p0 + i * kThreads;
@@ -452,10 +453,20 @@ cudaError_t launch_dequant_grad(int dtype, int bits, int lanes_per_group, const 
 cudaError_t launch_copy_rows(const void* src, void* dst, const int32_t* ids, int n, long long row_bytes, bool gather,
                              cudaStream_t s) {
   if (n <= 0 || row_bytes <= 0) return cudaSuccess;
-  const long long pieces = row_bytes / 16;
   const long long per_cta = (long long)kThreads * kCopyPiecesPerThread;
+  // the widest piece that divides a row and that both blocks are aligned for
+  const uintptr_t where = reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst) | (uintptr_t)row_bytes;
+  const int piece = (where & 15u) == 0 ? 16 : (where & 3u) == 0 ? 4 : 1;
+  const long long pieces = row_bytes / piece;
   const dim3 grid((unsigned)((pieces + per_cta - 1) / per_cta), (unsigned)n);
-  copy_rows_kernel<<<grid, kThreads, 0, s>>>(static_cast<const uint4*>(src), static_cast<uint4*>(dst), ids, pieces, gather);
+  if (piece == 16)
+    copy_rows_kernel<uint4><<<grid, kThreads, 0, s>>>(static_cast<const uint4*>(src), static_cast<uint4*>(dst), ids, pieces, gather);
+  else if (piece == 4)
+    copy_rows_kernel<uint32_t><<<grid, kThreads, 0, s>>>(static_cast<const uint32_t*>(src), static_cast<uint32_t*>(dst), ids, pieces,
+                                                         gather);
+  else
+    copy_rows_kernel<uint8_t><<<grid, kThreads, 0, s>>>(static_cast<const uint8_t*>(src), static_cast<uint8_t*>(dst), ids, pieces,
+                                                        gather);
   return cudaGetLastError();
 }
 

@@ -146,7 +146,7 @@ __global__ void __launch_bounds__(kThreads, MBITS == 32 ? 4 : 6)
   T* out = SENDER ? nullptr : reinterpret_cast<T*>(da.out) + row * elems;
   const bool words_ok = (st.packed_bytes & 3) == 0;
   const bool touch = mode != kModeSkip;
-  const unsigned long long sid = touch ? (unsigned long long)(unsigned)sample.id : 0ull;
+  const unsigned long long sid = touch ? (unsigned long long)sample.row : 0ull;     // the sample's row of the store
   uint8_t* m_codes = static_cast<uint8_t*>(st.m) + sid * (unsigned long long)st.m_bytes;
   float* m_scales = (MBITS == 32) ? nullptr : st.m_scales + sid * (unsigned)st.groups;
 

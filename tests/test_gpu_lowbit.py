@@ -43,7 +43,7 @@ class LowSide:
         return codes, steps, seen
 
 
-def run_lowbit(cfg, m_bits, n_batch=None, stochastic_seed=None, hosted=False):
+def run_lowbit(cfg, m_bits, n_batch=None, stochastic_seed=None, hosted=False, prefetch=None):
     nb = n_batch or cfg.n_batch
     gs, gr = LowSide(cfg, nb, m_bits, hosted), LowSide(cfg, nb, m_bits, hosted)
     od = DT[cfg.dtype][1]
@@ -51,6 +51,7 @@ def run_lowbit(cfg, m_bits, n_batch=None, stochastic_seed=None, hosted=False):
     packed = torch.empty((nb, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
     scales = torch.empty((nb, cfg.groups), dtype=torch.float32, device="cuda")
     out = torch.empty((nb, cfg.seq, cfg.hidden), dtype=cfg.torch_dtype, device="cuda")
+    calls = 0
     try:
         if stochastic_seed is not None:                      # only the sender rounds
             aq.aq_configure(gs.h, aq.AQ_ROUNDING, aq.AQ_ROUND_STOCHASTIC)
@@ -66,6 +67,10 @@ def run_lowbit(cfg, m_bits, n_batch=None, stochastic_seed=None, hosted=False):
                 packed.fill_(0xAB)
                 scales.fill_(-7.0)
                 out.fill_(3.0)
+                if prefetch and prefetch(calls):                 # hosted store: rows fetched ahead of the call
+                    aq.aq_prefetch(gs.h, ids)
+                    aq.aq_prefetch(gr.h, ids)
+                calls += 1
                 aq.aq_encode(gs.h, act, ids.cuda(), packed, scales)
                 aq.aq_configure(gr.h, aq.AQ_RAW, act)
                 aq.aq_decode(gr.h, packed, scales, ids.cuda(), out)
@@ -106,16 +111,18 @@ def test_large_shapes_reduced_id_space(m_bits):
 @pytest.mark.parametrize("m_bits", [2, 4, 8])
 def test_low_precision_store_in_host_memory(m_bits):
     """Codes and steps in page-locked host memory: the same kernels on mapped pointers, the same
-    results, checkpoint reads and digest included; no staged visits for this store."""
+    results, checkpoint reads and digest included; visited in place, fetched ahead of the call
+    (codes and steps both staged and written back; rows by copies and rows by the kernel), and
+    the two mixed."""
     run_lowbit(synth.TINY, m_bits, hosted=True)
     run_lowbit(synth.shrink(synth.GPT2_XL, 8, seq=96, epochs=3), m_bits, n_batch=4, hosted=True, stochastic_seed=21)
-    h = aq.aq_create_hosted_lowbit(4, 2, 64, 4, 64, m_bits)
-    try:
-        with pytest.raises(aq.AqError) as e:
-            aq.aq_prefetch(h, torch.zeros(1, dtype=torch.int32))
-        assert e.value.code == aq.AQ_EUNSUPPORTED
-    finally:
-        aq.aq_destroy(h)
+    run_lowbit(synth.TINY, m_bits, hosted=True, prefetch=lambda k: True)
+    run_lowbit(synth.shrink(synth.GPT2_XL, 8, seq=96, epochs=3), m_bits, n_batch=4, hosted=True, stochastic_seed=22,
+               prefetch=lambda k: k % 3 != 1)
+    ragged = synth.Boundary("low-staged-ragged", 6, 3, 37, 136, "bf16", 5, 8, 3, "outlier", 0.3, seed=612)
+    run_lowbit(ragged, m_bits, hosted=True, prefetch=lambda k: True)
+    wide = synth.Boundary("low-staged-wide", 256, 128, 1, 64, "fp16", 4, 64, 2, "normal", 0.1, seed=613)
+    run_lowbit(wide, m_bits, hosted=True, prefetch=lambda k: True)
     for not_offered in (16, 32):
         with pytest.raises(aq.AqError):
             aq.aq_create_hosted_lowbit(4, 2, 64, 4, 64, not_offered)
