@@ -14,7 +14,7 @@ namespace aq {
 namespace {
 
 constexpr unsigned kFullMask = 0xffffffffu;
-constexpr int kChunksPerThread = 2;                      // grad kernels: chunks per thread
+constexpr int kChunksPerThread = 3;                      // grad kernels: chunks per thread (measured: 2, 3, 4)
 constexpr int kChunksPerCta = kThreads * kChunksPerThread;
 
 enum { kModeDelta = 0, kModeFirst = 1, kModeSkip = 2 };
