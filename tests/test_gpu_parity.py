@@ -297,6 +297,56 @@ def test_host_buffer_forms_in_slices(n_batch):
         gs.close(), gr.close(), os_.close(), or_.close()
 
 
+def test_two_boundaries_run_side_by_side_on_two_streams():
+    """A stage has a boundary on either side: two pairs of handles, each pair on a stream of its
+    own, fed without any synchronisation in between.  Handles share no state, so each pair must
+    give exactly what it gives alone."""
+    cfgs = [synth.Boundary("left", 12, 4, 24, 256, "fp16", 4, 64, 3, "normal", 0.05, seed=41),
+            synth.Boundary("right", 10, 5, 17, 384, "bf16", 2, 128, 3, "student_t3", 0.02, seed=42, stream=1)]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    sides = [(GpuSide(c, c.n_batch, st), GpuSide(c, c.n_batch, st)) for c, st in zip(cfgs, streams)]
+    oracles = [tuple(oracle.Side(c.n_samples, c.seq, c.hidden, c.bits, c.group, DT[c.dtype][1]) for _ in range(2)) for c in cfgs]
+    kept = [[], []]
+    try:
+        n_calls = [c.epochs * (c.n_samples // c.n_batch) for c in cfgs]
+        for call in range(max(n_calls)):
+            for b, c in enumerate(cfgs):
+                if call >= n_calls[b]:
+                    continue
+                per_epoch = c.n_samples // c.n_batch
+                epoch, k = divmod(call, per_epoch)
+                ids = synth.epoch_order(c, epoch)[k * c.n_batch:(k + 1) * c.n_batch].contiguous()
+                act = synth.activation(c, ids, epoch, device="cuda")
+                ids_d = ids.cuda()
+                packed = torch.empty((c.n_batch, c.packed_bytes), dtype=torch.uint8, device="cuda")
+                scales = torch.empty((c.n_batch, c.groups), dtype=torch.float32, device="cuda")
+                out = torch.empty_like(act)
+                torch.cuda.current_stream().synchronize()                 # the inputs are ready; the codec calls are not waited for
+                gs, gr = sides[b]
+                aq.aq_encode(gs.h, act, ids_d, packed, scales)
+                aq.aq_configure(gr.h, aq.AQ_RAW, act)
+                aq.aq_decode(gr.h, packed, scales, ids_d, out)
+                kept[b].append((ids, act, ids_d, packed, scales, out))
+        torch.cuda.synchronize()
+        for b, c in enumerate(cfgs):
+            o_s, o_r = oracles[b]
+            for ids, act, _, packed, scales, out in kept[b]:
+                p_o, s_o, _ = o_s.encode(bits16(act), ids.numpy())
+                out_o, _ = o_r.decode(p_o, s_o, ids.numpy(), raw=bits16(act))
+                assert np.array_equal(packed.cpu().numpy(), p_o) and np.array_equal(scales.cpu().numpy(), s_o), c.name
+                assert np.array_equal(bits16(out), out_o), c.name
+            gs, gr = sides[b]
+            assert aq.aq_state_checksum(gs.h) == aq.aq_state_checksum(gr.h) == o_s.checksum() == o_r.checksum()
+            assert np.array_equal(gs.m_all(), o_s.m()) and np.array_equal(gr.m_all(), o_r.m())
+    finally:
+        for pair in sides:
+            for g in pair:
+                g.close()
+        for pair in oracles:
+            for o in pair:
+                o.close()
+
+
 def test_import_export_round_trip():
     cfg = synth.Boundary("ckpt", 3, 1, 4, 64, "fp16", 4, 64, 1, "normal", 0.1, seed=8)
     a, b = GpuSide(cfg, 1), GpuSide(cfg, 1)
