@@ -40,7 +40,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one delta-visit launch of 32 GPT2-shaped sequences
 # (52,428,800 elements), from the ncu capture summarised in profiles/encode_decode_gpt2_boundary_ncu.md;
 # scaled by the elements of a launch.  Set to None when the kernels change after the capture.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = {"encode": 290332160 / 52428800, "decode": 286967040 / 52428800}
+NCU_TRAFFIC_BYTES_PER_ELEMENT = {"encode": 291368192 / 52428800, "decode": 287016960 / 52428800}
 NCU_TRAFFIC_WORKLOAD = "gpt2"
 
 
@@ -59,6 +59,7 @@ def parse_args():
     ap.add_argument("--m-bits", type=int, default=0, choices=[0, 2, 4, 8, 32],
                     help="keep the previous messages in this many bits per element (0 = the activation type, 32 = binary32)")
     ap.add_argument("--hosted", action="store_true", help="keep m in page-locked host memory (aq_create_hosted)")
+    ap.add_argument("--no-l2-prefetch", action="store_true", help="AQ_L2_PREFETCH = 0: plain loads only")
     ap.add_argument("--stage-compute-ms", type=float, default=0.0,
                     help="stand-in for the stage's own work: a kernel that holds the handles' stream for about this many "
                          "ms after every step, to see what of the codec's time stays on the critical path")
@@ -301,6 +302,8 @@ def main():
         aq.aq_configure(h, aq.AQ_STREAM, stream.cuda_stream)
         if args.rows_per_cta:
             aq.aq_configure(h, aq.AQ_ROWS_PER_CTA, args.rows_per_cta)
+        if args.no_l2_prefetch:
+            aq.aq_configure(h, aq.AQ_L2_PREFETCH, 0)
         if args.rounding == "stochastic":
             aq.aq_configure(h, aq.AQ_ROUNDING, aq.AQ_ROUND_STOCHASTIC)
             aq.aq_configure(h, aq.AQ_SEED, 20220601)
@@ -587,7 +590,7 @@ def main():
         "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": label, "hidden": cfg.hidden, "seq": cfg.seq,
-                   "micro_batch": cfg.n_batch, "sequences_per_step": MACRO, "sequences_per_launch": nb, "cuda_graph": bool(args.graph), "rounding": args.rounding, "m_bits": args.m_bits or 16,
+                   "micro_batch": cfg.n_batch, "sequences_per_step": MACRO, "sequences_per_launch": nb, "cuda_graph": bool(args.graph), "l2_prefetch": not args.no_l2_prefetch and not args.hosted, "rounding": args.rounding, "m_bits": args.m_bits or 16,
                    "m_in": ("host memory (page-locked), staged through HBM by aq_prefetch, written back on a copy stream; step time by the host clock" if args.prefetch
                             else "host memory (page-locked, mapped)" if args.hosted else "HBM"),
                    "act_dtype": cfg.dtype, "bits": cfg.bits, "group": cfg.group, "n_samples_per_side": cfg.n_samples,

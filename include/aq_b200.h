@@ -85,8 +85,13 @@ enum {
   AQ_EPOCH = 9,          /* 64-bit counter that the caller sets before a call: two calls that should draw
                             independent random numbers need different values (for activations the epoch
                             or step number; for gradients any number unique to the call); default 0 */
-  AQ_ROWS_PER_CTA = 6    /* tuning: rows (256 chunks = 2048 elements each) that one CTA of aq_encode /
+  AQ_ROWS_PER_CTA = 6,   /* tuning: rows (256 chunks = 2048 elements each) that one CTA of aq_encode /
                             aq_decode walks; 0 (default) = chosen from the size of the call (2..4) */
+  AQ_L2_PREFETCH = 10    /* tuning: 1 (default for stores in device memory) = every CTA of aq_encode /
+                            aq_decode asks for its rows of act and m to be brought into L2 before it
+                            loads them (one bulk-prefetch instruction, results unchanged); act must then
+                            be in device memory.  0 = plain loads only (default for hosted stores, whose
+                            staged calls use the value set here) */
 };
 enum { AQ_FP16 = 0, AQ_BF16 = 1 };
 /*

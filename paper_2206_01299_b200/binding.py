@@ -13,6 +13,7 @@ LIB_PATH = os.path.join(HERE, "libaq_b200.so")
 
 AQ_OK, AQ_EINVAL, AQ_ENOMEM, AQ_ECUDA, AQ_EUNSUPPORTED = 0, -1, -2, -3, -4
 AQ_DTYPE, AQ_BATCH, AQ_STREAM, AQ_RAW, AQ_FIRST_FLAGS, AQ_ROWS_PER_CTA = 1, 2, 3, 4, 5, 6
+AQ_L2_PREFETCH = 10
 AQ_ROUNDING, AQ_SEED, AQ_EPOCH = 7, 8, 9
 AQ_FP16, AQ_BF16 = 0, 1
 AQ_ROUND_INTERVAL, AQ_ROUND_STOCHASTIC = 0, 1

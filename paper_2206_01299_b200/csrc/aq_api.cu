@@ -16,6 +16,7 @@ struct aq_handle {
   int seq = 0, hidden = 0, bits = 0, group = 0;
   int dtype = AQ_FP16;
   int n_batch = 1;
+  int l2_prefetch = 1;                       // AQ_L2_PREFETCH as set; st.l2_prefetch is what in-place calls get
   int rounding = AQ_ROUND_INTERVAL;
   unsigned long long seed = 0, epoch = 0;
   int device = 0;
@@ -193,6 +194,7 @@ int run_staged(aq_handle* h, Launch launch) {
   st.m = h->slots;
   if (h->m_scales_host) st.m_scales = h->slot_scales;
   st.slot_ids = h->d_slot_ids;
+  st.l2_prefetch = h->l2_prefetch;                    // the staged rows are in device memory
   AQ_CUDA(h, cudaStreamWaitEvent(h->stream, h->ev_staged, 0));
   AQ_CUDA(h, launch(st));
   AQ_CUDA(h, cudaEventRecord(h->ev_computed, h->stream));
@@ -263,6 +265,7 @@ static aq_handle* create_handle(int64_t n_samples, int seq, int hidden, int bits
   st.groups = st.elems / group;
   st.lanes_per_group = lanes;
   st.lg_shift = __builtin_ctz((unsigned)lanes);
+  st.l2_prefetch = hosted ? 0 : h->l2_prefetch;     // rows in mapped host memory are not brought into L2
   cudaError_t e = cudaGetDevice(&h->device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&st.sms, cudaDevAttrMultiProcessorCount, h->device);
   st.m_bits = m_bits;
@@ -373,6 +376,11 @@ int aq_configure(aq_handle* h, int key, int64_t value) {
       return AQ_OK;
     case AQ_EPOCH:
       h->epoch = (unsigned long long)value;
+      return AQ_OK;
+    case AQ_L2_PREFETCH:
+      if (value != 0 && value != 1) return fail(h, AQ_EINVAL, "AQ_L2_PREFETCH must be 0 or 1");
+      h->l2_prefetch = (int)value;
+      h->st.l2_prefetch = h->m_host ? 0 : (int)value;      // rows in mapped host memory are not brought into L2
       return AQ_OK;
     case AQ_ROWS_PER_CTA:
       if (value < 0 || value > (1 << 20)) return fail(h, AQ_EINVAL, "AQ_ROWS_PER_CTA must be in 0..2^20");

@@ -342,6 +342,13 @@ __device__ __forceinline__ unsigned long long take_call_number(const State& st, 
 // multiprocessors while this grid is draining, and do not read anything before the previous
 // kernel of the stream has completed and its writes are visible.  (Both are hardware-managed
 // and no-ops for neighbours launched the ordinary way.)
+// Asks for `bytes` (a multiple of 16) from the 16-byte aligned address p to be brought into L2:
+// one instruction, nothing to wait for, no shared memory.  A CTA's first thread of its second
+// warp does this for the rows the CTA is about to walk while the first warp looks the sample up.
+__device__ __forceinline__ void prefetch_l2(const void* p, unsigned bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
+
 __device__ __forceinline__ void overlap_with_neighbours() {
   asm volatile("griddepcontrol.launch_dependents;");
   asm volatile("griddepcontrol.wait;" ::: "memory");

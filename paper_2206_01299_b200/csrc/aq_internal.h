@@ -39,6 +39,7 @@ struct State {
   int lg_shift;                   // log2(lanes_per_group)
   int sms;                        // multiprocessors of the handle's device
   int rows_per_cta;               // 0 = chosen by the launch layer (default); > 0 = fixed rows per CTA
+  int l2_prefetch;                // 1: encode / decode ask for a CTA's rows to be brought into L2 ahead of its loads
   const int32_t* slot_ids;        // null: row xi of m belongs to sample xi.  Else m is a staging block of the
                                   // running call: row y holds m of sample slot_ids[y] (hosted store, prefetched)
 };

@@ -95,11 +95,16 @@ __global__ void __launch_bounds__(kThreads, STOCH ? 4 : encode_ctas_per_sm<T, BI
   const int lane = tid & 31;
   const int y = blockIdx.y;                                       // sample of the call
   overlap_with_neighbours();
-  const Sample sample = open_sample(st, plan, a.ids, y, false, false, a.first_flags);
-  const int mode = sample.mode;
   // sizes per sample fit 32 bits (checked at create): 32 x 32 -> 64-bit products
   const unsigned elems = (unsigned)st.elems;
   const T* act = reinterpret_cast<const T*>(a.act) + (unsigned long long)(unsigned)y * elems;
+  // the CTA's chunks [pf_lo, pf_hi): its activation rows are asked for before the sample is known
+  const int pf_lo = blockIdx.x * plan.rows_per_cta * kThreads;
+  const int pf_hi = min(st.chunks, (int)(blockIdx.x + 1) * plan.rows_per_cta * kThreads);
+  const bool pf = st.l2_prefetch && tid == 32;
+  if (pf && pf_hi > pf_lo) prefetch_l2(act + (size_t)pf_lo * kChunk, (unsigned)(pf_hi - pf_lo) * 16u);
+  const Sample sample = open_sample(st, plan, a.ids, y, false, false, a.first_flags);
+  const int mode = sample.mode;
   uint8_t* stream = a.packed + (unsigned long long)(unsigned)y * (unsigned)st.packed_bytes;
   float* scales = a.scales + (unsigned long long)(unsigned)y * (unsigned)st.groups;
   const bool words_ok = (st.packed_bytes & 3) == 0;
@@ -108,6 +113,10 @@ __global__ void __launch_bounds__(kThreads, STOCH ? 4 : encode_ctas_per_sm<T, BI
 
   if (mode == kModeDelta) {
     T* m = reinterpret_cast<T*>(st.m) + (unsigned long long)sample.row * elems;
+    {
+      const int m_lo = pf_lo + kRowsPerIter * kThreads;           // the first iteration's rows are loaded at once
+      if (pf && pf_hi > m_lo) prefetch_l2(m + (size_t)m_lo * kChunk, (unsigned)(pf_hi - m_lo) * 16u);
+    }
     // whole iterations first (rows without a ragged end: no bounds to check), then the rest
     const int whole_end = min(r_end, st.chunks / kThreads);
     for (; r + kRowsPerIter <= whole_end; r += kRowsPerIter)
@@ -190,6 +199,10 @@ __global__ void __launch_bounds__(kThreads, decode_ctas_per_sm<BITS>()) decode_k
 
   if (mode == kModeDelta) {
     T* m = reinterpret_cast<T*>(st.m) + (unsigned long long)sample.row * elems;
+    {
+      const int m_lo = (r + kRowsPerIter) * kThreads, m_hi = min(st.chunks, r_end * kThreads);
+      if (st.l2_prefetch && tid == 32 && m_hi > m_lo) prefetch_l2(m + (size_t)m_lo * kChunk, (unsigned)(m_hi - m_lo) * 16u);
+    }
     const uint8_t* stream = a.packed + (unsigned long long)(unsigned)y * (unsigned)st.packed_bytes;
     const float* scales = a.scales + (unsigned long long)(unsigned)y * (unsigned)st.groups;
     const bool words_ok = (st.packed_bytes & 3) == 0;

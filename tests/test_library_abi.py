@@ -52,7 +52,7 @@ def test_binding_matches_the_header():
 def test_constants_match_the_header():
     text = open(HEADER).read()
     for name in ("AQ_OK", "AQ_EINVAL", "AQ_ENOMEM", "AQ_ECUDA", "AQ_EUNSUPPORTED", "AQ_DTYPE", "AQ_BATCH",
-                 "AQ_STREAM", "AQ_RAW", "AQ_FIRST_FLAGS", "AQ_ROWS_PER_CTA", "AQ_ROUNDING", "AQ_SEED", "AQ_EPOCH",
+                 "AQ_STREAM", "AQ_RAW", "AQ_FIRST_FLAGS", "AQ_ROWS_PER_CTA", "AQ_ROUNDING", "AQ_SEED", "AQ_EPOCH", "AQ_L2_PREFETCH",
                  "AQ_ROUND_INTERVAL", "AQ_ROUND_STOCHASTIC", "AQ_FP16", "AQ_BF16",
                  "AQ_ST_BAD_ID", "AQ_ST_DUP_ID", "AQ_ST_NO_RAW", "AQ_ST_STAGED"):
         m = re.search(rf"\b{name}\s*=\s*(-?\d+)", text)
