@@ -42,7 +42,7 @@ class GpuSide:
 
 
 def run_boundary(cfg, n_batch=None, epochs=None, check_all_m=True, order_fn=None, act_fn=None, stochastic_seed=None,
-                 hosted=False, prefetch=None):
+                 hosted=False, prefetch=None, l2_prefetch=None):
     """Every call of every epoch: GPU sender -> GPU receiver and oracle sender -> oracle
     receiver; packed, scales, first flags, out and (per epoch) both m arrays and the state
     digests must agree exactly.  prefetch (hosted handles): a function of the call's running
@@ -58,6 +58,9 @@ def run_boundary(cfg, n_batch=None, epochs=None, check_all_m=True, order_fn=None
     out = torch.empty((nb, cfg.seq, cfg.hidden), dtype=cfg.torch_dtype, device="cuda")
     calls = 0
     try:
+        if l2_prefetch is not None:
+            aq.aq_configure(gs.h, aq.AQ_L2_PREFETCH, int(l2_prefetch))
+            aq.aq_configure(gr.h, aq.AQ_L2_PREFETCH, int(l2_prefetch))
         if stochastic_seed is not None:                      # only the sender rounds; the receiver needs no setting
             aq.aq_configure(gs.h, aq.AQ_ROUNDING, aq.AQ_ROUND_STOCHASTIC)
             aq.aq_configure(gs.h, aq.AQ_SEED, stochastic_seed)

@@ -297,6 +297,24 @@ def test_host_buffer_forms_in_slices(n_batch):
         gs.close(), gr.close(), os_.close(), or_.close()
 
 
+def test_l2_prefetch_switch():
+    """AQ_L2_PREFETCH only says whether a CTA asks for its rows ahead of its loads: results are
+    the same with the key at 0, at 1 (the default), and for a hosted store with staged calls."""
+    cfg = synth.shrink(synth.GPT2_XL, 8, seq=160, epochs=3)
+    run_boundary(cfg, n_batch=4, l2_prefetch=0)
+    run_boundary(cfg, n_batch=4, l2_prefetch=1)
+    ragged = synth.Boundary("pf-ragged", 6, 3, 37, 136, "bf16", 3, 8, 3, "outlier", 0.3, seed=43)
+    run_boundary(ragged, l2_prefetch=0)
+    run_boundary(ragged, hosted=True, prefetch=lambda k: True, l2_prefetch=1)
+    run_boundary(ragged, hosted=True, prefetch=lambda k: k % 2 == 0, l2_prefetch=0)
+    h = aq.aq_create(4, 2, 64, 4, 64)
+    try:
+        with pytest.raises(aq.AqError):
+            aq.aq_configure(h, aq.AQ_L2_PREFETCH, 2)
+    finally:
+        aq.aq_destroy(h)
+
+
 def test_two_boundaries_run_side_by_side_on_two_streams():
     """A stage has a boundary on either side: two pairs of handles, each pair on a stream of its
     own, fed without any synchronisation in between.  Handles share no state, so each pair must
