@@ -546,8 +546,8 @@ def main():
     window = min(32, steps_per_epoch)
     with torch.cuda.stream(stream):
         passes = [kernel_pass(total_steps + r * window, window) for r in range(3)]
-    enc_ms = statistics.mean(p[0] for p in passes)
-    dec_ms = statistics.mean(p[1] for p in passes)
+    enc_ms = statistics.median(p[0] for p in passes)          # one disturbed pass must not move the figure
+    dec_ms = statistics.median(p[1] for p in passes)
     status = aq.aq_status(snd) | aq.aq_status(rcv)
     digests_equal = aq.aq_state_checksum(snd) == aq.aq_state_checksum(rcv)
     assert status == 0 and digests_equal, "sender and receiver state diverged"
@@ -603,7 +603,7 @@ def main():
                      "frac": enc_gbs / peak, "peak_kind": peak_kind,
                      "traffic": None if traffic is None else traffic * nb * cfg.elems,
                      "algorithmic_bytes_per_launch": launch_bytes, "avg_launch_ms": enc_ms,
-                     "timing": f"CUDA events around {window * launches_per_step} back-to-back launches of the kernel, 3 passes right after the timed steps",
+                     "timing": f"CUDA events around {window * launches_per_step} back-to-back launches of the kernel, median of 3 passes right after the timed steps",
                      "decode_kernel": {"achieved": dec_gbs, "frac": dec_gbs / peak, "avg_launch_ms": dec_ms}},
         "first_visit_epoch": {"ms": first_ms, "GB/s": first_bytes / (first_ms * 1e-3) / 1e9},
         "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": args.steps * (launches_per_step * 2 + (2 if sweep else 0)),
