@@ -582,7 +582,7 @@ def main():
     enc_gbs = launch_bytes / (enc_ms * 1e-3) / 1e9
     dec_gbs = launch_bytes / (dec_ms * 1e-3) / 1e9
     traffic = NCU_TRAFFIC_BYTES_PER_ELEMENT["encode"] if (args.workload == NCU_TRAFFIC_WORKLOAD and args.rounding == "interval"
-                                                          and not args.m_bits and not args.hosted) else None
+                                                          and not args.m_bits and not args.hosted and not args.no_l2_prefetch) else None
     value = replicas.whole_job_rate(args.steps * step_bytes, world, elapsed_ms) / 1e9
     line = {
         "metric": "activation encode+decode GB/s", "value": value, "unit": "GB/s",
