@@ -101,7 +101,7 @@ __global__ void __launch_bounds__(kThreads, STOCH ? 4 : encode_ctas_per_sm<T, BI
   // the CTA's chunks [pf_lo, pf_hi): its activation rows are asked for before the sample is known
   const int pf_lo = blockIdx.x * plan.rows_per_cta * kThreads;
   const int pf_hi = min(st.chunks, (int)(blockIdx.x + 1) * plan.rows_per_cta * kThreads);
-  const bool pf = st.l2_prefetch && tid == 32;
+  const bool pf = !STOCH && st.l2_prefetch && tid == 32;          // the stochastic kernel is bound by instruction issue
   if (pf && pf_hi > pf_lo) prefetch_l2(act + (size_t)pf_lo * kChunk, (unsigned)(pf_hi - pf_lo) * 16u);
   const Sample sample = open_sample(st, plan, a.ids, y, false, false, a.first_flags);
   const int mode = sample.mode;
