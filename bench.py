@@ -138,6 +138,9 @@ class ClockSampler:
 
     def __enter__(self):
         if self.nv:
+            # the timed loop keeps the interpreter busy; a short switch interval lets this thread in
+            self._switch = sys.getswitchinterval()
+            sys.setswitchinterval(0.0005)
             self._thread = threading.Thread(target=self._run, daemon=True)
             self._thread.start()
         return self
@@ -146,6 +149,7 @@ class ClockSampler:
         self._stop.set()
         if self._thread:
             self._thread.join()
+            sys.setswitchinterval(self._switch)
 
     def summary(self):
         return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
