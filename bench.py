@@ -126,14 +126,17 @@ class ClockSampler:
                 out.append(name)
         return out
 
-    def _run(self):
+    def _sample(self):
         nv = self.nv
+        try:
+            self.samples.append(nv.nvmlDeviceGetClockInfo(self.dev, nv.NVML_CLOCK_SM))
+            self.reasons.update(self._names(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.dev)))
+        except Exception:
+            pass
+
+    def _run(self):
         while not self._stop.is_set():
-            try:
-                self.samples.append(nv.nvmlDeviceGetClockInfo(self.dev, nv.NVML_CLOCK_SM))
-                self.reasons.update(self._names(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.dev)))
-            except Exception:
-                pass
+            self._sample()
             time.sleep(0.002)
 
     def __enter__(self):
@@ -150,6 +153,7 @@ class ClockSampler:
         if self._thread:
             self._thread.join()
             sys.setswitchinterval(self._switch)
+            self._sample()                                    # a very short timed region still gets a reading at its end
 
     def summary(self):
         return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
@@ -511,6 +515,9 @@ def main():
         torch.cuda.synchronize()
         with ClockSampler(local_rank) as clocks:
             wall0 = time.perf_counter()
+            # about 0.1 ms of an idle-spinning kernel ahead of the start event: the host queues the event and the
+            # first launches behind it, so that the clock starts with work waiting and not with launch latency
+            torch.cuda._sleep(200_000)
             t_begin.record(stream)
             for t in range(args.steps):
                 if graphs:
