@@ -517,7 +517,8 @@ def main():
             wall0 = time.perf_counter()
             # about 0.1 ms of an idle-spinning kernel ahead of the start event: the host queues the event and the
             # first launches behind it, so that the clock starts with work waiting and not with launch latency
-            torch.cuda._sleep(200_000)
+            if hasattr(torch.cuda, "_sleep"):
+                torch.cuda._sleep(200_000)
             t_begin.record(stream)
             for t in range(args.steps):
                 if graphs:
