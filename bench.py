@@ -173,7 +173,7 @@ def time_oracle(cfg, budget_s, device, max_samples=256):
     about budget_s seconds of work are done.  Returns (GB/s, samples/s, n_samples, seconds)."""
     import numpy as np
     import oracle
-    from paper_2206_01299_b200 import synth
+    from fixtures import synth
     od = oracle.FP16 if cfg.dtype == "fp16" else oracle.BF16
     small = synth.shrink(cfg, max_samples)
     snd = oracle.Side(max_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, od)
@@ -200,7 +200,7 @@ def run_reference(args, cfg):
     import numpy as np
     import torch
     import oracle
-    from paper_2206_01299_b200 import synth
+    from fixtures import synth
     device = "cuda" if torch.cuda.is_available() else "cpu"
     # calibrate on one full sample, then size the per-step sample so the run stays near two minutes
     _, sps, _, _ = time_oracle(cfg, 0.0, device, max_samples=2)
@@ -255,7 +255,7 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
 
     from dataclasses import replace
-    from paper_2206_01299_b200 import replicas, synth
+    from fixtures import replicas, synth
     global MACRO, M_BITS
     M_BITS = args.m_bits
     recipe, MACRO, label = WORKLOADS[args.workload]
@@ -801,7 +801,7 @@ def run_e2e(aq, torch, cfg, snd, rcv, arena, ids_dev, steps, dist):
 
     dt_serial = timed(run_serial)
     dt = timed(run_pipelined)
-    from paper_2206_01299_b200 import replicas
+    from fixtures import replicas
     dt = replicas.max_over_ranks(dt, dist, "cuda")
     assert aq.aq_status(snd) == 0 and aq.aq_status(rcv) == 0
     assert aq.aq_state_checksum(snd) == aq.aq_state_checksum(rcv)

@@ -20,8 +20,8 @@
  * All arithmetic is IEEE binary32, one rounding per operation (no fused
  * multiply-add), so results are reproducible bit for bit.
  *
- * One handle is ONE copy of the previous-message array m (Algorithm 1: "array
- * of previous messages m initialized to 0"): the sender's or the receiver's
+ * One handle is ONE copy of the previous-message array m that Algorithm 1 sets
+ * up, zero-filled, in its initialisation step: the sender's or the receiver's
  * side of one stage boundary.  A pipeline with K stages uses K-1 independent
  * pairs of handles (appendix A.1).
  *
@@ -96,8 +96,8 @@ enum {
 enum { AQ_FP16 = 0, AQ_BF16 = 1 };
 /*
  * AQ_ROUND_INTERVAL: Q of Section 4.1 as described at the top of this file.
- * AQ_ROUND_STOCHASTIC: the unbiased Q that Theorem 3.1 assumes (its footnote: rounding to the
- * uniform grid "stochastically").  The 2^b levels reach from -s to +s,
+ * AQ_ROUND_STOCHASTIC: the unbiased Q that Theorem 3.1 assumes (its footnote sketches a randomised
+ * rounding onto a uniform grid).  The 2^b levels reach from -s to +s,
  *   Delta = s / (2^(b-1) - 1/2),  k = clamp(floor(d * (1/Delta) + (r - 1/2))),  r uniform in [0,1),
  * so that E[(k + 1/2) * Delta] = d for every element of the group.  Receivers need no setting:
  * aq_decode / aq_dequant_grad rebuild (k + 1/2) * Delta from the Delta they are sent.  r comes
@@ -119,7 +119,7 @@ enum {
 };
 
 /*
- * Algorithm 1, "Initialize": allocates m (n_samples*seq*hidden*2 bytes of device
+ * Initialisation step of Algorithm 1: allocates m (n_samples*seq*hidden*2 bytes of device
  * memory on the current device) filled with zeros, and an empty "seen before"
  * set.  bits in 1..8 is b of the forward quantizer; group in {8,16,32,64,128,256}
  * must divide hidden.  Returns NULL on failure; aq_last_error(NULL) says why.
@@ -202,7 +202,7 @@ void aq_destroy(aq_handle* h);
 int aq_configure(aq_handle* h, int key, int64_t value);
 
 /*
- * Sender side (Algorithm 2, "on network a"; Algorithm 1, the branch on "xi not seen before").  For each
+ * Sender side (Algorithm 2, the part run on network a; Algorithm 1, the test whether xi was seen before).  For each
  * of the n_batch samples, in one fused pass over the data:
  *   first visit  m(xi) <- act (bit copy; the full-precision activation itself is the
  *                message, the caller forwards `act`), codes and scales of the sample = 0;
@@ -213,7 +213,7 @@ int aq_configure(aq_handle* h, int key, int64_t value);
 int aq_encode(aq_handle* h, const void* act, const int32_t* sample_ids, void* packed, float* scales);
 
 /*
- * Receiver side (Algorithm 2, "on network b"): m(xi) <- T(m(xi) + (k+1/2)*Delta) on this
+ * Receiver side (Algorithm 2, the part run on network b): m(xi) <- T(m(xi) + (k+1/2)*Delta) on this
  * handle's own copy of m, and out <- the new m(xi), which network b uses as its forward
  * activation.  First visit: m(xi) <- raw, out <- raw (AQ_RAW).
  * packed, scales (in), sample_ids int32[n_batch] (in), out T[n_batch][seq][hidden] (out).
@@ -221,8 +221,8 @@ int aq_encode(aq_handle* h, const void* act, const int32_t* sample_ids, void* pa
 int aq_decode(aq_handle* h, const void* packed, const float* scales, const int32_t* sample_ids, void* out);
 
 /*
- * Backward direction (Algorithm 1: "Machine b sends Q(gradient of f o b w.r.t. a)"):
- * the same Q applied directly to the gradient; touches no state.  n_elems must be a
+ * Backward direction (Algorithm 1, the message from machine b back to machine a: the quantized
+ * gradient with respect to the activation): the same Q applied directly to the gradient; touches no state.  n_elems must be a
  * multiple of the handle's group; bits in 1..8 may differ from the handle's forward b.
  * grad T[n_elems] (in); packed uint8[n_elems*bits/8], scales float[n_elems/group] (out).
  * n_elems == 0 is a no-op.
@@ -237,7 +237,7 @@ int aq_dequant_grad(aq_handle* h, const void* packed, const float* scales, int64
  *   sum_i mix(i, word_i) + sum_xi mix(2^40 + xi, seen[xi])   (mod 2^64),
  * word_i = the i-th little-endian 32-bit word of m, mix(i, w) = the splitmix64 output
  * function applied to i*0x9E3779B97F4A7C15 + w.  Two handles fed the same id sequence
- * (the two sides of a boundary, Algorithm 2: "networks a and b each maintain a copy")
+ * (the two sides of a boundary: in Algorithm 2 either network keeps its own copy of m)
  * must give the same digest.  Synchronises the stream; *out_host is host memory.
  */
 int aq_state_checksum(aq_handle* h, uint64_t* out_host);

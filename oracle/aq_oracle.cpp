@@ -158,7 +158,7 @@ inline float reconstruct(int32_t k, float delta) {
 
 // ---------------------------------------------------------------------------
 // Unbiased variant of Q (the quantizer that Theorem 3.1 assumes; its footnote
-// sketches it as "rounding to the closest k/2^b, stochastically").  Reading
+// sketches it as a randomised rounding onto the grid of multiples of 2^-b).  Reading
 // fixed here: the 2^b levels are spread evenly over the whole of [-s, s],
 //
 //   Delta = s / (2^(b-1) - 1/2),   level_k = (k + 1/2) * Delta,  k in [-2^(b-1), 2^(b-1)-1]
@@ -277,8 +277,8 @@ int32_t get_code(const uint8_t* stream, int64_t j, int bits) {
 
 // ---------------------------------------------------------------------------
 // State of one side of one boundary: the array m of previous messages, indexed
-// by sample (Algorithm 1, "array of previous messages m initialized to 0"),
-// and the "seen before" set.
+// by sample and zero-filled as Algorithm 1's initialisation step says,
+// and the set of samples seen before.
 // ---------------------------------------------------------------------------
 
 struct Side {
@@ -401,7 +401,7 @@ void* aqo_create(int64_t n_samples, int seq, int hidden, int bits, int group, in
   if (!S) return nullptr;
   S->n_samples = n_samples; S->seq = seq; S->hidden = hidden;
   S->bits = bits; S->group = group; S->dtype = dtype; S->status = 0;
-  S->m.assign((size_t)n_samples * seq * hidden, 0);     // "initialized to 0"
+  S->m.assign((size_t)n_samples * seq * hidden, 0);     // Algorithm 1 starts from an all-zero m
   S->seen.assign((size_t)n_samples, 0);
   return S;
 }
@@ -418,7 +418,7 @@ const uint16_t* aqo_m(void* h) { return ((Side*)h)->m.data(); }
 const uint8_t* aqo_seen(void* h) { return ((Side*)h)->seen.data(); }
 uint32_t aqo_status(void* h) { Side* S = (Side*)h; uint32_t s = S->status; S->status = 0; return s; }
 
-// Sender (Algorithm 2, "on network a"; Algorithm 1, the branch on "xi not seen before").
+// Sender (Algorithm 2, the part run on network a; Algorithm 1, the test whether xi was seen before).
 //   act     [n_batch][seq][hidden]  activation a(xi)
 //   ids     [n_batch]               sample ids xi
 //   packed  [n_batch][seq*hidden*bits/8]   out: bitstream of codes
@@ -508,8 +508,8 @@ void aqo_decode(void* h, const uint8_t* packed, const float* scales, const uint1
   }
 }
 
-// Direct quantization of the backward activation-gradient (Algorithm 1,
-// "Machine b sends Q(grad_a (f o b)|_m)"): same Q, no buffer, no delta.
+// Direct quantization of the backward activation-gradient (Algorithm 1, the
+// message from machine b back to machine a): same Q, no buffer, no delta.
 void aqo_quant_grad(const uint16_t* grad, int64_t n_elems, int bits, int group, int dtype,
                     uint8_t* packed, float* scales) {
   std::vector<float> d(group);
@@ -577,7 +577,7 @@ void* aqo_low_create(int64_t n_samples, int seq, int hidden, int bits, int group
   if (!S) return nullptr;
   S->n_samples = n_samples; S->seq = seq; S->hidden = hidden; S->bits = bits; S->group = group;
   S->dtype = dtype; S->m_bits = m_bits; S->status = 0;
-  S->m_codes.assign((size_t)(n_samples * E * m_bits / 8), 0);     // codes 0, steps 0: "initialized to 0"
+  S->m_codes.assign((size_t)(n_samples * E * m_bits / 8), 0);     // codes 0, steps 0: an all-zero m
   S->m_scales.assign(m_bits == 32 ? 0 : (size_t)(n_samples * E / group), 0.0f);
   S->seen.assign((size_t)n_samples, 0);
   return S;

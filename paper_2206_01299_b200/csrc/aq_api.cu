@@ -296,7 +296,7 @@ static aq_handle* create_handle(int64_t n_samples, int seq, int hidden, int bits
     e = cudaHostAlloc(reinterpret_cast<void**>(&h->m_scales_host), m_scale_bytes, cudaHostAllocMapped | cudaHostAllocPortable);
     if (e == cudaSuccess) e = cudaHostGetDevicePointer(reinterpret_cast<void**>(&st.m_scales), h->m_scales_host, 0);
   }
-  if (e == cudaSuccess && !hosted) e = cudaMemset(st.m, 0, m_bytes);           // "initialized to 0"
+  if (e == cudaSuccess && !hosted) e = cudaMemset(st.m, 0, m_bytes);           // Algorithm 1 starts from an all-zero m
   if (e == cudaSuccess && hosted) memset(h->m_host, 0, m_bytes);
   if (e == cudaSuccess && m_steps && !hosted) e = cudaMemset(st.m_scales, 0, m_scale_bytes);
   if (e == cudaSuccess && m_steps && hosted) memset(h->m_scales_host, 0, m_scale_bytes);

@@ -323,7 +323,7 @@ __device__ __forceinline__ uint4 ld_stream(const void* p) { return __ldcs(reinte
 __device__ __forceinline__ void st_stream(void* p, const uint4& v) { __stcs(reinterpret_cast<uint4*>(p), v); }
 
 
-// ------------------------------------------------------------------ calls and samples (Algorithm 1, "if xi not seen before")
+// ------------------------------------------------------------------ calls and samples (Algorithm 1, the first-visit test)
 
 // Number of the running call, the same in every CTA of the grid, different for every launch on
 // the handle.  The handle keeps one 64-bit arrival counter that only grows.  Each CTA adds its

@@ -5,7 +5,7 @@ import torch
 
 import oracle
 import paper_2206_01299_b200 as aq
-from paper_2206_01299_b200 import synth
+from fixtures import synth
 
 DT = {"fp16": (aq.AQ_FP16, oracle.FP16), "bf16": (aq.AQ_BF16, oracle.BF16)}
 
@@ -13,6 +13,30 @@ DT = {"fp16": (aq.AQ_FP16, oracle.FP16), "bf16": (aq.AQ_BF16, oracle.BF16)}
 def bits16(t: torch.Tensor) -> np.ndarray:
     """16-bit float tensor (any device) -> numpy uint16 bit patterns."""
     return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+GUARD_BYTES = 512
+GUARD_FILL = 0x5A
+
+
+class Guarded:
+    """A device buffer with GUARD_BYTES of a known pattern in front of it and behind it.  `.t` is
+    the buffer itself (the view handed to the library); check() fails when a kernel wrote outside
+    it.  Stands in for a memory checker: a store one word past the end of an output lands here."""
+
+    def __init__(self, shape, dtype, device="cuda"):
+        shape = (shape,) if isinstance(shape, int) else tuple(shape)
+        n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+        self.body = (n + 15) // 16 * 16                       # the tail guard starts at the next 16-byte boundary at the latest
+        self.n = n
+        self.raw = torch.full((GUARD_BYTES + self.body + GUARD_BYTES,), GUARD_FILL, dtype=torch.uint8, device=device)
+        self.t = self.raw[GUARD_BYTES:GUARD_BYTES + n].view(dtype).view(shape)
+
+    def check(self, what=""):
+        front = self.raw[:GUARD_BYTES].cpu().numpy()
+        behind = self.raw[GUARD_BYTES + self.n:].cpu().numpy()
+        assert (front == GUARD_FILL).all(), f"write in front of {what}"
+        assert (behind == GUARD_FILL).all(), f"write behind {what}"
 
 
 class GpuSide:
@@ -24,7 +48,9 @@ class GpuSide:
         aq.aq_configure(self.h, aq.AQ_BATCH, n_batch)
         if stream is not None:
             aq.aq_configure(self.h, aq.AQ_STREAM, stream.cuda_stream)
-        self.first = torch.zeros(max(n_batch, 1), dtype=torch.uint8, device="cuda")
+        self.first_guarded = Guarded(max(n_batch, 1), torch.uint8)
+        self.first = self.first_guarded.t
+        self.first.zero_()
         aq.aq_configure(self.h, aq.AQ_FIRST_FLAGS, self.first)
 
     def close(self):
@@ -41,6 +67,17 @@ class GpuSide:
         return np.stack([self.m_row(i)[0] for i in range(self.cfg.n_samples)])
 
 
+def guarded_outputs(cfg, nb):
+    """(packed, scales, out) of a call of nb samples as Guarded buffers."""
+    return (Guarded((nb, cfg.packed_bytes), torch.uint8), Guarded((nb, cfg.groups), torch.float32),
+            Guarded((nb, cfg.seq, cfg.hidden), cfg.torch_dtype))
+
+
+def check_guards(*guarded):
+    for i, g in enumerate(guarded):
+        g.check(f"output buffer {i}")
+
+
 def run_boundary(cfg, n_batch=None, epochs=None, check_all_m=True, order_fn=None, act_fn=None, stochastic_seed=None,
                  hosted=False, prefetch=None, l2_prefetch=None):
     """Every call of every epoch: GPU sender -> GPU receiver and oracle sender -> oracle
@@ -53,9 +90,10 @@ def run_boundary(cfg, n_batch=None, epochs=None, check_all_m=True, order_fn=None
     gs, gr = GpuSide(cfg, nb, hosted=hosted), GpuSide(cfg, nb, hosted=hosted)
     od = DT[cfg.dtype][1]
     os_, or_ = (oracle.Side(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, od) for _ in range(2))
-    packed = torch.empty((nb, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
-    scales = torch.empty((nb, cfg.groups), dtype=torch.float32, device="cuda")
-    out = torch.empty((nb, cfg.seq, cfg.hidden), dtype=cfg.torch_dtype, device="cuda")
+    g_packed = Guarded((nb, cfg.packed_bytes), torch.uint8)
+    g_scales = Guarded((nb, cfg.groups), torch.float32)
+    g_out = Guarded((nb, cfg.seq, cfg.hidden), cfg.torch_dtype)
+    packed, scales, out = g_packed.t, g_scales.t, g_out.t
     calls = 0
     try:
         if l2_prefetch is not None:
@@ -92,6 +130,9 @@ def run_boundary(cfg, n_batch=None, epochs=None, check_all_m=True, order_fn=None
                 assert np.array_equal(gs.first.cpu().numpy()[:nb], f_o), (epoch, c, "first (sender)")
                 assert np.array_equal(gr.first.cpu().numpy()[:nb], fr_o), (epoch, c, "first (receiver)")
                 assert np.array_equal(bits16(out), out_o), (epoch, c, "out")
+                for g, what in ((g_packed, "packed"), (g_scales, "scales"), (g_out, "out"),
+                                (gs.first_guarded, "first flags (sender)"), (gr.first_guarded, "first flags (receiver)")):
+                    g.check(what)
             assert aq.aq_status(gs.h) == os_.status() and aq.aq_status(gr.h) == or_.status()
             cs = aq.aq_state_checksum(gs.h)
             assert cs == aq.aq_state_checksum(gr.h) == os_.checksum() == or_.checksum(), (epoch, "digest")

@@ -6,8 +6,8 @@ import torch
 
 import oracle
 import paper_2206_01299_b200 as aq
-from paper_2206_01299_b200 import synth
-from codec_harness import DT, bits16
+from fixtures import synth
+from codec_harness import DT, Guarded, bits16, check_guards
 
 pytestmark = pytest.mark.gpu
 
@@ -20,7 +20,9 @@ class LowSide:
                   else aq.aq_create_lowbit(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, m_bits))
         aq.aq_configure(self.h, aq.AQ_DTYPE, DT[cfg.dtype][0])
         aq.aq_configure(self.h, aq.AQ_BATCH, n_batch)
-        self.first = torch.zeros(n_batch, dtype=torch.uint8, device="cuda")
+        self.first_guarded = Guarded(n_batch, torch.uint8)
+        self.first = self.first_guarded.t
+        self.first.zero_()
         aq.aq_configure(self.h, aq.AQ_FIRST_FLAGS, self.first)
         self.code_bytes = cfg.elems * m_bits // 8
         self.n_steps = 0 if m_bits == 32 else cfg.groups
@@ -48,9 +50,10 @@ def run_lowbit(cfg, m_bits, n_batch=None, stochastic_seed=None, hosted=False, pr
     gs, gr = LowSide(cfg, nb, m_bits, hosted), LowSide(cfg, nb, m_bits, hosted)
     od = DT[cfg.dtype][1]
     os_, or_ = (oracle.SideLow(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, od, m_bits) for _ in range(2))
-    packed = torch.empty((nb, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
-    scales = torch.empty((nb, cfg.groups), dtype=torch.float32, device="cuda")
-    out = torch.empty((nb, cfg.seq, cfg.hidden), dtype=cfg.torch_dtype, device="cuda")
+    g_packed = Guarded((nb, cfg.packed_bytes), torch.uint8)
+    g_scales = Guarded((nb, cfg.groups), torch.float32)
+    g_out = Guarded((nb, cfg.seq, cfg.hidden), cfg.torch_dtype)
+    packed, scales, out = g_packed.t, g_scales.t, g_out.t
     calls = 0
     try:
         if stochastic_seed is not None:                      # only the sender rounds
@@ -82,6 +85,9 @@ def run_lowbit(cfg, m_bits, n_batch=None, stochastic_seed=None, hosted=False, pr
                 assert np.array_equal(scales.cpu().numpy().view(np.uint32), s_o.view(np.uint32)), (epoch, c, "scales")
                 assert np.array_equal(gs.first.cpu().numpy(), f_o) and np.array_equal(gr.first.cpu().numpy(), fr_o)
                 assert np.array_equal(bits16(out), out_o), (epoch, c, "out")
+                for g, what in ((g_packed, "packed"), (g_scales, "scales"), (g_out, "out"),
+                                (gs.first_guarded, "first flags (sender)"), (gr.first_guarded, "first flags (receiver)")):
+                    g.check(what)
             for g_side, o_side in ((gs, os_), (gr, or_)):
                 codes, steps, seen = g_side.state()
                 assert np.array_equal(codes, o_side.m_codes()), (epoch, "stored codes")
@@ -155,9 +161,8 @@ def test_bad_ids_import_export_and_unsupported_calls():
     gs, gr = LowSide(cfg, 4, 8), LowSide(cfg, 4, 8)
     os_, or_ = (oracle.SideLow(5, 2, 64, 2, 64, oracle.FP16, 8) for _ in range(2))
     try:
-        packed = torch.empty((4, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
-        scales = torch.empty((4, cfg.groups), dtype=torch.float32, device="cuda")
-        out = torch.empty((4, 2, 64), dtype=torch.float16, device="cuda")
+        guards = (Guarded((4, cfg.packed_bytes), torch.uint8), Guarded((4, cfg.groups), torch.float32), Guarded((4, 2, 64), torch.float16))
+        packed, scales, out = (g.t for g in guards)
         for step, id_list in enumerate([[1, 7, 1, 3], [3, -1, 1, 3], [0, 1, 2, 3]]):
             ids = torch.tensor(id_list, dtype=torch.int32)
             act = synth.activation(cfg, torch.tensor([10, 11, 12, 13]), step, device="cuda")
@@ -166,6 +171,7 @@ def test_bad_ids_import_export_and_unsupported_calls():
             aq.aq_configure(gr.h, aq.AQ_RAW, raw)
             aq.aq_decode(gr.h, packed, scales, ids.cuda(), out)
             torch.cuda.synchronize()
+            check_guards(*guards)
             p_o, s_o, _ = os_.encode(bits16(act), ids.numpy())
             out_o, _ = or_.decode(p_o, s_o, ids.numpy(), raw=bits16(act) if raw is not None else None)
             assert np.array_equal(packed.cpu().numpy(), p_o) and np.array_equal(scales.cpu().numpy(), s_o)
@@ -200,9 +206,8 @@ def test_gpt2_boundary_full_id_space_with_an_8_bit_store():
         pytest.skip("needs 12 GiB of free device memory")
     cfg, per_launch, m_bits = synth.GPT2_XL, 32, 8
     gs, gr = LowSide(cfg, per_launch, m_bits), LowSide(cfg, per_launch, m_bits)
-    packed = torch.empty((per_launch, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
-    scales = torch.empty((per_launch, cfg.groups), dtype=torch.float32, device="cuda")
-    out = torch.empty((per_launch, cfg.seq, cfg.hidden), dtype=cfg.torch_dtype, device="cuda")
+    guards = (Guarded((per_launch, cfg.packed_bytes), torch.uint8), Guarded((per_launch, cfg.groups), torch.float32), Guarded((per_launch, cfg.seq, cfg.hidden), cfg.torch_dtype))
+    packed, scales, out = (g.t for g in guards)
     buf = np.empty(aq.aq_m_bytes_per_sample(gs.h), np.uint8)
     tracked = {}
     try:
@@ -215,6 +220,7 @@ def test_gpt2_boundary_full_id_space_with_an_8_bit_store():
                 aq.aq_configure(gr.h, aq.AQ_RAW, act if epoch == 0 else None)
                 aq.aq_decode(gr.h, packed, scales, ids.cuda(), out)
                 torch.cuda.synchronize()
+                check_guards(*guards)
                 for y in (0, per_launch - 1):
                     sid = int(ids[y])
                     if sid not in tracked:

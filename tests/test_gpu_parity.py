@@ -5,8 +5,8 @@ import torch
 
 import oracle
 import paper_2206_01299_b200 as aq
-from paper_2206_01299_b200 import synth
-from codec_harness import DT, GpuSide, bits16, run_boundary
+from fixtures import synth
+from codec_harness import DT, GpuSide, Guarded, bits16, check_guards, run_boundary
 
 pytestmark = pytest.mark.gpu
 
@@ -66,12 +66,12 @@ def test_backward_workload_full_size():
         n = cfg.elems
         g_np = bits16(grad)
         for bits in cfg.bits:
-            packed = torch.empty(n * bits // 8, dtype=torch.uint8, device="cuda")
-            scales = torch.empty(n // cfg.group, dtype=torch.float32, device="cuda")
-            out = torch.empty(n, dtype=torch.float16, device="cuda")
+            guards = (Guarded(n * bits // 8, torch.uint8), Guarded(n // cfg.group, torch.float32), Guarded(n, torch.float16))
+            packed, scales, out = (g.t for g in guards)
             aq.aq_quant_grad(h, grad, n, bits, packed, scales)
             aq.aq_dequant_grad(h, packed, scales, n, bits, out)
             torch.cuda.synchronize()
+            check_guards(*guards)
             p_o, s_o = oracle.quant_grad(g_np, bits, cfg.group, oracle.FP16)
             o_o = oracle.dequant_grad(p_o, s_o, n, bits, cfg.group, oracle.FP16)
             assert np.array_equal(packed.cpu().numpy(), p_o)
@@ -144,11 +144,13 @@ def test_revisits_of_an_unchanged_activation_send_zeros():
     try:
         ids = torch.tensor([1, 3], dtype=torch.int32, device="cuda")
         act = act_fn(ids.cpu(), 0)
-        packed = torch.full((2, cfg.packed_bytes), 9, dtype=torch.uint8, device="cuda")
-        scales = torch.full((2, cfg.groups), 9.0, device="cuda")
+        guards = (Guarded((2, cfg.packed_bytes), torch.uint8), Guarded((2, cfg.groups), torch.float32))
+        packed, scales = (g.t for g in guards)
+        packed.fill_(9), scales.fill_(9.0)
         aq.aq_encode(side.h, act, ids, packed, scales)
         aq.aq_encode(side.h, act, ids, packed, scales)
         torch.cuda.synchronize()
+        check_guards(*guards)
         assert not packed.any() and not scales.any()
         assert np.array_equal(side.m_row(3)[0], bits16(act[1]))
     finally:
@@ -162,9 +164,8 @@ def test_bad_duplicate_and_rawless_ids_are_skipped_like_the_oracle():
     gs, gr = GpuSide(cfg, 4), GpuSide(cfg, 4)
     os_, or_ = (oracle.Side(5, 2, 64, 2, 64, oracle.FP16) for _ in range(2))
     try:
-        packed = torch.empty((4, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
-        scales = torch.empty((4, cfg.groups), dtype=torch.float32, device="cuda")
-        out = torch.empty((4, 2, 64), dtype=torch.float16, device="cuda")
+        guards = (Guarded((4, cfg.packed_bytes), torch.uint8), Guarded((4, cfg.groups), torch.float32), Guarded((4, 2, 64), torch.float16))
+        packed, scales, out = (g.t for g in guards)
         for step, id_list in enumerate([[1, 7, 1, 3], [3, -1, 1, 3], [0, 1, 2, 3]]):
             ids = torch.tensor(id_list, dtype=torch.int32)
             act = synth.activation(cfg, torch.tensor([10, 11, 12, 13]), step, device="cuda")
@@ -176,6 +177,7 @@ def test_bad_duplicate_and_rawless_ids_are_skipped_like_the_oracle():
             aq.aq_configure(gr.h, aq.AQ_RAW, raw)
             aq.aq_decode(gr.h, packed, scales, ids.cuda(), out)
             torch.cuda.synchronize()
+            check_guards(*guards)
             p_o, s_o, f_o = os_.encode(bits16(act), ids.numpy())
             out_o, fr_o = or_.decode(p_o, s_o, ids.numpy(), raw=bits16(act) if raw is not None else None)
             assert np.array_equal(packed.cpu().numpy(), p_o)
@@ -336,19 +338,20 @@ def test_two_boundaries_run_side_by_side_on_two_streams():
                 ids = synth.epoch_order(c, epoch)[k * c.n_batch:(k + 1) * c.n_batch].contiguous()
                 act = synth.activation(c, ids, epoch, device="cuda")
                 ids_d = ids.cuda()
-                packed = torch.empty((c.n_batch, c.packed_bytes), dtype=torch.uint8, device="cuda")
-                scales = torch.empty((c.n_batch, c.groups), dtype=torch.float32, device="cuda")
-                out = torch.empty_like(act)
+                guards = (Guarded((c.n_batch, c.packed_bytes), torch.uint8), Guarded((c.n_batch, c.groups), torch.float32),
+                          Guarded(tuple(act.shape), act.dtype))
+                packed, scales, out = (g.t for g in guards)
                 torch.cuda.current_stream().synchronize()                 # the inputs are ready; the codec calls are not waited for
                 gs, gr = sides[b]
                 aq.aq_encode(gs.h, act, ids_d, packed, scales)
                 aq.aq_configure(gr.h, aq.AQ_RAW, act)
                 aq.aq_decode(gr.h, packed, scales, ids_d, out)
-                kept[b].append((ids, act, ids_d, packed, scales, out))
+                kept[b].append((ids, act, ids_d, packed, scales, out, guards))
         torch.cuda.synchronize()
         for b, c in enumerate(cfgs):
             o_s, o_r = oracles[b]
-            for ids, act, _, packed, scales, out in kept[b]:
+            for ids, act, _, packed, scales, out, guards in kept[b]:
+                check_guards(*guards)
                 p_o, s_o, _ = o_s.encode(bits16(act), ids.numpy())
                 out_o, _ = o_r.decode(p_o, s_o, ids.numpy(), raw=bits16(act))
                 assert np.array_equal(packed.cpu().numpy(), p_o) and np.array_equal(scales.cpu().numpy(), s_o), c.name
@@ -397,21 +400,21 @@ def test_replayed_cuda_graph_counts_every_replay_as_a_call():
             ids = torch.tensor(ids_list, dtype=torch.int32)
             act = synth.activation(cfg, ids, epoch, device="cuda")
             ids_d = ids.cuda()
-            packed = torch.empty((2, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
-            scales = torch.empty((2, cfg.groups), dtype=torch.float32, device="cuda")
-            out = torch.empty((2, cfg.seq, cfg.hidden), dtype=torch.float16, device="cuda")
+            guards = (Guarded((2, cfg.packed_bytes), torch.uint8), Guarded((2, cfg.groups), torch.float32), Guarded((2, cfg.seq, cfg.hidden), torch.float16))
+            packed, scales, out = (g.t for g in guards)
             torch.cuda.synchronize()
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g, stream=stream):
                 aq.aq_configure(gr.h, aq.AQ_RAW, act)
                 aq.aq_encode(gs.h, act, ids_d, packed, scales)
                 aq.aq_decode(gr.h, packed, scales, ids_d, out)
-            graphs.append((g, ids, act, packed, scales, out, ids_d))     # the graph reads ids_d: keep it alive
+            graphs.append((g, ids, act, packed, scales, out, ids_d, guards))     # the graph reads ids_d: keep it alive
         for which in (0, 0, 1, 0, 1, 1):
-            g, ids, act, packed, scales, out, _ = graphs[which]
+            g, ids, act, packed, scales, out, _, guards = graphs[which]
             aq.aq_configure(gr.h, aq.AQ_RAW, act)            # host-side setting only; the graph holds its own pointer
             g.replay()
             torch.cuda.synchronize()
+            check_guards(*guards, gs.first_guarded, gr.first_guarded)
             p_o, s_o, f_o = os_.encode(bits16(act), ids.numpy())
             out_o, fr_o = or_.decode(p_o, s_o, ids.numpy(), raw=bits16(act))
             assert np.array_equal(packed.cpu().numpy(), p_o)
@@ -458,15 +461,15 @@ def test_stochastic_gradient_quantization_matches_oracle(dtype, bits):
         aq.aq_configure(h, aq.AQ_ROUNDING, aq.AQ_ROUND_STOCHASTIC)
         aq.aq_configure(h, aq.AQ_SEED, 424242)
         grad = _grad_input(n, group, td, 5000 + bits).cuda()
-        packed = torch.empty(n * bits // 8, dtype=torch.uint8, device="cuda")
-        scales = torch.empty(n // group, dtype=torch.float32, device="cuda")
-        out = torch.empty(n, dtype=td, device="cuda")
+        guards = (Guarded(n * bits // 8, torch.uint8), Guarded(n // group, torch.float32), Guarded(n, td))
+        packed, scales, out = (g.t for g in guards)
         seen = []
         for epoch in (3, (1 << 40) + 3):
             aq.aq_configure(h, aq.AQ_EPOCH, epoch)
             aq.aq_quant_grad(h, grad, n, bits, packed, scales)
             aq.aq_dequant_grad(h, packed, scales, n, bits, out)
             torch.cuda.synchronize()
+            check_guards(*guards)
             p_o, s_o = oracle.quant_grad_stochastic(bits16(grad), bits, group, 424242, epoch, DT[dtype][1])
             assert np.array_equal(packed.cpu().numpy(), p_o)
             assert np.array_equal(scales.cpu().numpy().view(np.uint32), s_o.view(np.uint32))
@@ -486,9 +489,8 @@ def test_largest_batch_of_small_samples():
     gs, gr = GpuSide(cfg, 4096), GpuSide(cfg, 4096)
     os_, or_ = (oracle.Side(4096, 1, 64, 4, 64, oracle.FP16) for _ in range(2))
     try:
-        packed = torch.empty((4096, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
-        scales = torch.empty((4096, cfg.groups), dtype=torch.float32, device="cuda")
-        out = torch.empty((4096, 1, 64), dtype=torch.float16, device="cuda")
+        guards = (Guarded((4096, cfg.packed_bytes), torch.uint8), Guarded((4096, cfg.groups), torch.float32), Guarded((4096, 1, 64), torch.float16))
+        packed, scales, out = (g.t for g in guards)
         for epoch in range(3):
             ids = synth.epoch_order(cfg, epoch).clone()
             ids[4000] = ids[17]                       # a repeat far into the call
@@ -498,6 +500,7 @@ def test_largest_batch_of_small_samples():
             aq.aq_configure(gr.h, aq.AQ_RAW, act)
             aq.aq_decode(gr.h, packed, scales, ids.cuda(), out)
             torch.cuda.synchronize()
+            check_guards(*guards)
             p_o, s_o, f_o = os_.encode(bits16(act), ids.numpy())
             out_o, fr_o = or_.decode(p_o, s_o, ids.numpy(), raw=bits16(act))
             assert np.array_equal(packed.cpu().numpy(), p_o) and np.array_equal(scales.cpu().numpy(), s_o)
@@ -527,9 +530,8 @@ def test_rows_per_cta_override_does_not_change_results(rows_per_cta):
     try:
         for h in (gs.h, gr.h):
             aq.aq_configure(h, aq.AQ_ROWS_PER_CTA, rows_per_cta)
-        packed = torch.empty((2, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
-        scales = torch.empty((2, cfg.groups), dtype=torch.float32, device="cuda")
-        out = torch.empty((2, 21, 1000), dtype=torch.float16, device="cuda")
+        guards = (Guarded((2, cfg.packed_bytes), torch.uint8), Guarded((2, cfg.groups), torch.float32), Guarded((2, 21, 1000), torch.float16))
+        packed, scales, out = (g.t for g in guards)
         for epoch in range(3):
             ids = torch.tensor([3, 1], dtype=torch.int32)
             act = synth.activation(cfg, ids, epoch, device="cuda")
@@ -537,6 +539,7 @@ def test_rows_per_cta_override_does_not_change_results(rows_per_cta):
             aq.aq_configure(gr.h, aq.AQ_RAW, act)
             aq.aq_decode(gr.h, packed, scales, ids.cuda(), out)
             torch.cuda.synchronize()
+            check_guards(*guards)
             p_o, s_o, _ = os_.encode(bits16(act), ids.numpy())
             out_o, _ = or_.decode(p_o, s_o, ids.numpy(), raw=bits16(act))
             assert np.array_equal(packed.cpu().numpy(), p_o) and np.array_equal(scales.cpu().numpy(), s_o)

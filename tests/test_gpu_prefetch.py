@@ -7,8 +7,8 @@ import torch
 
 import oracle
 import paper_2206_01299_b200 as aq
-from paper_2206_01299_b200 import synth
-from codec_harness import GpuSide, bits16, run_boundary
+from fixtures import synth
+from codec_harness import GpuSide, Guarded, bits16, check_guards, run_boundary
 
 pytestmark = pytest.mark.gpu
 
@@ -52,9 +52,8 @@ def test_prefetch_of_bad_and_repeated_ids():
     gs, gr = GpuSide(cfg, 6, hosted=True), GpuSide(cfg, 6, hosted=True)
     os_, or_ = (oracle.Side(8, 4, 64, 4, 64, oracle.FP16) for _ in range(2))
     try:
-        packed = torch.empty((6, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
-        scales = torch.empty((6, cfg.groups), dtype=torch.float32, device="cuda")
-        out = torch.empty((6, 4, 64), dtype=torch.float16, device="cuda")
+        guards = (Guarded((6, cfg.packed_bytes), torch.uint8), Guarded((6, cfg.groups), torch.float32), Guarded((6, 4, 64), torch.float16))
+        packed, scales, out = (g.t for g in guards)
         for epoch in range(3):
             ids = torch.tensor([3, 7, 3, -2, 0, 8], dtype=torch.int32)       # a repeat, two out of range
             act = synth.activation(cfg, torch.arange(6), epoch, device="cuda")
@@ -64,6 +63,7 @@ def test_prefetch_of_bad_and_repeated_ids():
             aq.aq_configure(gr.h, aq.AQ_RAW, act)
             aq.aq_decode(gr.h, packed, scales, ids.cuda(), out)
             torch.cuda.synchronize()
+            check_guards(*guards)
             p_o, s_o, f_o = os_.encode(bits16(act), ids.numpy())
             out_o, fr_o = or_.decode(p_o, s_o, ids.numpy(), raw=bits16(act))
             assert np.array_equal(packed.cpu().numpy(), p_o) and np.array_equal(scales.cpu().numpy(), s_o)

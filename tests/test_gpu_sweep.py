@@ -14,8 +14,8 @@ import torch
 
 import oracle
 import paper_2206_01299_b200 as aq
-from paper_2206_01299_b200 import synth
-from codec_harness import DT, GpuSide, bits16
+from fixtures import synth
+from codec_harness import DT, GpuSide, Guarded, bits16, check_guards, guarded_outputs
 
 pytestmark = pytest.mark.gpu
 
@@ -28,15 +28,13 @@ def test_pipeline_sweep_boundary_major():
     bbits = bwd.bits[0]
     assert (fwd0.bits, bbits, fwd0.group) == (3, 6, 64)
     # wire buffers: the sender's and the receiver's ends of the channel
-    tx_p = torch.empty((1, fwd0.packed_bytes), dtype=torch.uint8, device="cuda")
-    tx_s = torch.empty((1, fwd0.groups), dtype=torch.float32, device="cuda")
-    rx_p, rx_s = torch.empty_like(tx_p), torch.empty_like(tx_s)
-    rx_raw = torch.empty((1, seq, fwd0.hidden), dtype=torch.float16, device="cuda")
-    out = torch.empty_like(rx_raw)
-    gtx_p = torch.empty(n * bbits // 8, dtype=torch.uint8, device="cuda")
-    gtx_s = torch.empty(n // bwd.group, dtype=torch.float32, device="cuda")
-    grx_p, grx_s = torch.empty_like(gtx_p), torch.empty_like(gtx_s)
-    gout = torch.empty(n, dtype=torch.float16, device="cuda")
+    guards = [Guarded((1, fwd0.packed_bytes), torch.uint8), Guarded((1, fwd0.groups), torch.float32),       # tx_p, tx_s
+              Guarded((1, fwd0.packed_bytes), torch.uint8), Guarded((1, fwd0.groups), torch.float32),       # rx_p, rx_s
+              Guarded((1, seq, fwd0.hidden), torch.float16), Guarded((1, seq, fwd0.hidden), torch.float16),  # rx_raw, out
+              Guarded(n * bbits // 8, torch.uint8), Guarded(n // bwd.group, torch.float32),                  # gtx_p, gtx_s
+              Guarded(n * bbits // 8, torch.uint8), Guarded(n // bwd.group, torch.float32),                  # grx_p, grx_s
+              Guarded(n, torch.float16)]                                                                     # gout
+    tx_p, tx_s, rx_p, rx_s, rx_raw, out, gtx_p, gtx_s, grx_p, grx_s, gout = (g.t for g in guards)
     digests = []
     for boundary in range(synth.SWEEP_BOUNDARIES):
         cfg = replace(fwd0, stream=boundary)
@@ -65,6 +63,7 @@ def test_pipeline_sweep_boundary_major():
                         grx_s.copy_(gtx_s)
                         aq.aq_dequant_grad(gs.h, grx_p, grx_s, n, bbits, gout)
                         torch.cuda.synchronize()
+                        check_guards(*guards, gs.first_guarded, gr.first_guarded)
                         a_np = bits16(act)
                         p_o, s_o, _ = os_.encode(a_np, ids.numpy())
                         out_o, _ = or_.decode(p_o, s_o, ids.numpy(), raw=a_np if epoch == 0 else None)
@@ -89,13 +88,17 @@ def test_pipeline_sweep_boundary_major():
     assert len(set(digests)) == synth.SWEEP_BOUNDARIES              # every boundary saw its own data
 
 
-def _full_size_sampled(cfg, per_launch, steps, samples_per_launch):
-    """Full id space, the benchmark's launch shape; the oracle follows only the sampled ids."""
+def _full_size_sampled(cfg, per_launch, steps, samples_per_launch, wire=False):
+    """Full id space, the benchmark's launch shape; the oracle follows only the sampled ids.
+    wire: the message crosses aq_wire_copy into the receiver's own buffers (the raw block too, on
+    first visits), as between the two stages of the pipeline sweep."""
     od = DT[cfg.dtype][1]
     gs, gr = GpuSide(cfg, per_launch), GpuSide(cfg, per_launch)
-    packed = torch.empty((per_launch, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
-    scales = torch.empty((per_launch, cfg.groups), dtype=torch.float32, device="cuda")
-    out = torch.empty((per_launch, cfg.seq, cfg.hidden), dtype=cfg.torch_dtype, device="cuda")
+    guards = guarded_outputs(cfg, per_launch)
+    packed, scales, out = (g.t for g in guards)
+    if wire:
+        rx = guarded_outputs(cfg, per_launch)                          # the receiver's codes, steps and raw block
+        guards = guards + rx
     tracked = {}                                                     # sample id -> (oracle sender, oracle receiver)
     try:
         order = synth.epoch_order(cfg, 0)
@@ -104,10 +107,20 @@ def _full_size_sampled(cfg, per_launch, steps, samples_per_launch):
                 ids = order[step * per_launch:(step + 1) * per_launch].contiguous()
                 act = synth.activation(cfg, ids, epoch, device="cuda")
                 aq.aq_encode(gs.h, act, ids.cuda(), packed, scales)
-                aq.aq_configure(gr.h, aq.AQ_RAW, act if epoch == 0 else None)
-                aq.aq_decode(gr.h, packed, scales, ids.cuda(), out)
+                if wire:
+                    first = epoch == 0
+                    aq.aq_wire_copy(gs.h, torch.cuda.current_device(), rx[0].t, rx[1].t, rx[2].t if first else None,
+                                    packed, scales, act if first else None)
+                    aq.aq_configure(gr.h, aq.AQ_RAW, rx[2].t if first else None)
+                    aq.aq_decode(gr.h, rx[0].t, rx[1].t, ids.cuda(), out)
+                else:
+                    aq.aq_configure(gr.h, aq.AQ_RAW, act if epoch == 0 else None)
+                    aq.aq_decode(gr.h, packed, scales, ids.cuda(), out)
                 torch.cuda.synchronize()
+                check_guards(*guards, gs.first_guarded, gr.first_guarded)
                 assert gs.first.cpu().numpy().all() == (epoch == 0)
+                if wire:
+                    assert torch.equal(rx[0].t, packed) and torch.equal(rx[1].t.view(torch.int32), scales.view(torch.int32))
                 for y in np.linspace(0, per_launch - 1, samples_per_launch).astype(int):
                     sid = int(ids[y])
                     if sid not in tracked:
@@ -146,6 +159,38 @@ def test_gpt2_boundary_full_id_space_in_the_benchmark_launch_shape():
     _full_size_sampled(cfg, 32, steps=[0, 1, cfg.n_samples // 32 - 1], samples_per_launch=2)
 
 
+def test_sweep_boundary_full_id_space_in_the_benchmark_launch_shape():
+    """One boundary of the pipeline sweep at full size: 8192 ids (26.8 GB of m per side), a macro-batch of
+    16 micro-batches of 1 x 1024 x 1600 fp16 per launch, 3-bit deltas over the wire copy, three epochs;
+    then the backward direction of one whole macro-batch (26,214,400 gradient elements) in 6 bits."""
+    _needs_gb(60)
+    cfg, per_launch = synth.SWEEP_FWD, synth.SWEEP_MICRO_BATCHES
+    assert (cfg.n_samples, cfg.bits, cfg.group, cfg.elems) == (8192, 3, 64, 1024 * 1600)
+    _full_size_sampled(cfg, per_launch, steps=[0, 3, cfg.n_samples // per_launch - 1], samples_per_launch=2, wire=True)
+    bwd = replace(synth.SWEEP_BWD, n_batch=per_launch)
+    bits, n = bwd.bits[0], bwd.elems
+    assert (bits, n) == (6, 26214400)
+    h = aq.aq_create(1, 1, bwd.group, cfg.bits, bwd.group)
+    try:
+        grad = synth.gradient(bwd, 1, device="cuda")
+        guards = (Guarded(n * bits // 8, torch.uint8), Guarded(n // bwd.group, torch.float32),     # sender's end of the wire
+                  Guarded(n * bits // 8, torch.uint8), Guarded(n // bwd.group, torch.float32),     # receiver's end
+                  Guarded(n, torch.float16))
+        tx_p, tx_s, rx_p, rx_s, gout = (g.t for g in guards)
+        aq.aq_quant_grad(h, grad, n, bits, tx_p, tx_s)
+        rx_p.copy_(tx_p)
+        rx_s.copy_(tx_s)
+        aq.aq_dequant_grad(h, rx_p, rx_s, n, bits, gout)
+        torch.cuda.synchronize()
+        check_guards(*guards)
+        p_o, s_o = oracle.quant_grad(bits16(grad), bits, bwd.group, oracle.FP16)
+        assert np.array_equal(rx_p.cpu().numpy(), p_o)
+        assert np.array_equal(rx_s.cpu().numpy().view(np.uint32), s_o.view(np.uint32))
+        assert np.array_equal(bits16(gout), oracle.dequant_grad(p_o, s_o, n, bits, bwd.group, oracle.FP16))
+    finally:
+        aq.aq_destroy(h)
+
+
 def test_deberta_boundary_full_id_space():
     """32768 ids (25.8 GB of m per side), micro-batch 8 x 256 x 1536 bf16, 2 bit, group 128."""
     _needs_gb(60)
@@ -162,9 +207,8 @@ def test_gpt2_boundary_full_id_space_with_stochastic_rounding():
     gs, gr = GpuSide(cfg, per_launch), GpuSide(cfg, per_launch)
     od = DT[cfg.dtype][1]
     o_s, o_r = (oracle.Side(n_track, cfg.seq, cfg.hidden, cfg.bits, cfg.group, od) for _ in range(2))
-    packed = torch.empty((per_launch, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
-    scales = torch.empty((per_launch, cfg.groups), dtype=torch.float32, device="cuda")
-    out = torch.empty((per_launch, cfg.seq, cfg.hidden), dtype=cfg.torch_dtype, device="cuda")
+    guards = guarded_outputs(cfg, per_launch)
+    packed, scales, out = (g.t for g in guards)
     try:
         aq.aq_configure(gs.h, aq.AQ_ROUNDING, aq.AQ_ROUND_STOCHASTIC)
         aq.aq_configure(gs.h, aq.AQ_SEED, seed)
@@ -182,6 +226,7 @@ def test_gpt2_boundary_full_id_space_with_stochastic_rounding():
                 aq.aq_configure(gr.h, aq.AQ_RAW, act if epoch == 0 else None)
                 aq.aq_decode(gr.h, packed, scales, ids.cuda(), out)
                 torch.cuda.synchronize()
+                check_guards(*guards, gs.first_guarded, gr.first_guarded)
                 for sid, pos in where.items():
                     if pos // per_launch != step:
                         continue

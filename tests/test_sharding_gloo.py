@@ -8,7 +8,7 @@ import torch
 import torch.distributed as dist
 import torch.multiprocessing as mp
 
-from paper_2206_01299_b200 import replicas, synth
+from fixtures import replicas, synth
 
 
 def _free_port():

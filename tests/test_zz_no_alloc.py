@@ -15,7 +15,7 @@ import pytest
 import torch
 
 import paper_2206_01299_b200 as aq
-from paper_2206_01299_b200 import synth
+from fixtures import synth
 
 pytestmark = pytest.mark.gpu
 
