@@ -1,23 +1,32 @@
 #!/usr/bin/env python
 """Benchmark of the AQ-SGD boundary codec on B200.
 
-Workload (default): the GPT2-1.5B-shaped boundary -- hidden 1600, sequence 1024,
+Headline workload (default): the GPT2-1.5B-shaped boundary -- hidden 1600, sequence 1024,
 micro-batch 1, fp16, 4-bit deltas, group 64, 4096 sample ids per side (13.4 GB of m on
 the sender and again on the receiver), a fresh seeded id order per epoch.  One STEP is one
 macro-batch of 32 micro-batches (the paper's GPT2 setting) crossing the boundary:
 aq_encode on the sender handle, then aq_decode on the receiver handle.  Epoch 0 (first
 visits, uncompressed) is run and timed apart; the timed steps are steady-state delta visits
-of epochs 1..4, whose activations are generated into HBM before the clock starts.
+of later epochs, whose activations are generated into HBM before the clock starts.
+
+The timed region of `--steps` K steps is repeated (at least 30 windows, and until half a
+second of GPU time is covered); `ms_per_step` is the median window, with minimum, maximum
+and the number of windows beside it.
 
 One JSON line on stdout (rank 0).  `value` = algorithmic GB/s of encode+decode over the
 timed steps of all ranks; `roofline` = the encode kernel against the measured HBM copy
 peak; `e2e` = the same step through aq_encode_host / aq_decode_host with pinned host
-buffers; `cpu_baseline` = the CPU oracle on a bounded sample of the same workload.
+buffers; `cpu_baseline` = the CPU oracle on a bounded sample of the same workload, on one
+core and on all host cores; `configs` (one GPU only) = the same measurement for the
+DeBERTa-1.5B-shaped boundary, one boundary of the pipeline sweep and the backward path, each
+also with calls of the workload's own micro-batch size.
 
 `--impl reference` times the CPU oracle instead (rank 0 only).
 """
 import argparse
+import hashlib
 import json
+import math
 import os
 import statistics
 import sys
@@ -28,8 +37,8 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-MACRO = 32            # sequences per step: the macro-batch (32 x micro-batch 1 in the paper's GPT2 runs)
-# name -> (recipe in synth, sequences per macro-batch, label); the paper's DeBERTa/QNLI runs use macro-batch 64
+# name -> (recipe in fixtures.synth, sequences per macro-batch, label); the paper's GPT2 runs use macro-batch 32 of
+# micro-batch 1, its DeBERTa/QNLI runs macro-batch 64 of micro-batch 8
 WORKLOADS = {"gpt2": ("GPT2_XL", 32, "GPT2-1.5B-shaped boundary (configs[1])"),
              "deberta": ("DEBERTA_XXL", 64, "DeBERTa-1.5B-shaped boundary (configs[2])"),
              # one of the 8 boundaries of the pipeline sweep (they are independent and alike): per macro-batch of 16
@@ -37,21 +46,35 @@ WORKLOADS = {"gpt2": ("GPT2_XL", 32, "GPT2-1.5B-shaped boundary (configs[1])"),
              "sweep": ("SWEEP_FWD", 16, "one boundary of the pipeline sweep (configs[4]): fwd 3-bit delta + bwd 6-bit direct + wire copies")}
 FALLBACK_HBM_GBS = 6650.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one delta-visit launch of 32 GPT2-shaped sequences
-# (52,428,800 elements), from the ncu capture summarised in profiles/encode_decode_gpt2_boundary_ncu.md;
-# scaled by the elements of a launch.  Set to None when the kernels change after the capture.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = {"encode": 291368192 / 52428800, "decode": 287016960 / 52428800}
-NCU_TRAFFIC_WORKLOAD = "gpt2"
+# DRAM traffic of one delta-visit launch from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum),
+# per element, by workload; reported as roofline.traffic only while the kernel sources still hash to the
+# value recorded with the capture (`python bench.py --kernel-hash` prints the current one).
+NCU_TRAFFIC = {}
+
+
+def kernel_source_hash():
+    """SHA-256 (first 16 hex digits) over the kernel sources that the traffic figures were taken from."""
+    h = hashlib.sha256()
+    for name in ("aq_internal.h", "aq_device.cuh", "aq_kernels.cu"):
+        with open(os.path.join(ROOT, "paper_2206_01299_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
 
 
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=384)
+    ap.add_argument("--steps", type=int, default=64)
     ap.add_argument("--warmup", type=int, default=16)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--workload", default="gpt2", choices=sorted(WORKLOADS), help="the headline workload")
+    ap.add_argument("--configs", default=None, choices=["all", "headline"],
+                    help="all (default on one GPU): also measure the other workloads, reported under `configs`")
+    ap.add_argument("--topology", default="replicas", choices=["replicas", "pipeline"],
+                    help="replicas (default): every rank runs both sides of its own boundary.  pipeline (an even number of "
+                         "ranks): ranks 2p and 2p+1 are the sending and the receiving stage of boundary p, the message "
+                         "travels between them through torch.distributed (paper_2206_01299_b200.link)")
     ap.add_argument("--n-samples", type=int, default=None, help="shrink the id space (profiling runs)")
-    ap.add_argument("--workload", default="gpt2", choices=sorted(WORKLOADS))
     ap.add_argument("--per-launch", type=int, default=0, help="sequences handed to one aq_encode call (0 = the whole macro-batch)")
     ap.add_argument("--graph", action="store_true", help="replay each step as a captured CUDA graph")
     ap.add_argument("--rounding", default="interval", choices=["interval", "stochastic"],
@@ -59,33 +82,31 @@ def parse_args():
     ap.add_argument("--m-bits", type=int, default=0, choices=[0, 2, 4, 8, 32],
                     help="keep the previous messages in this many bits per element (0 = the activation type, 32 = binary32)")
     ap.add_argument("--hosted", action="store_true", help="keep m in page-locked host memory (aq_create_hosted)")
-    ap.add_argument("--no-l2-prefetch", action="store_true", help="AQ_L2_PREFETCH = 0: plain loads only")
-    ap.add_argument("--stage-compute-ms", type=float, default=0.0,
-                    help="stand-in for the stage's own work: a kernel that holds the handles' stream for about this many "
-                         "ms after every step, to see what of the codec's time stays on the critical path")
     ap.add_argument("--prefetch", action="store_true",
                     help="with --hosted: fetch every call's previous messages ahead of it (aq_prefetch); the calls "
                          "then run on staged rows in HBM and write them back behind the caller")
-    ap.add_argument("--rows-per-cta", type=int, default=0, help="AQ_ROWS_PER_CTA of both handles (0 = library default)")
+    ap.add_argument("--stage-compute-ms", type=float, default=0.0,
+                    help="with --hosted: a stand-in for the stage's own work, a kernel that holds the handles' stream "
+                         "for about this many ms after every step (what of the transfers stays on the critical path)")
+    ap.add_argument("--min-timed-ms", type=float, default=500.0, help="repeat the timed region until it covers this much GPU time")
+    ap.add_argument("--max-repeats", type=int, default=400)
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-aux", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=32)
-    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--kernel-hash", action="store_true", help="print the hash of the kernel sources and exit")
     return ap.parse_args()
 
 
-M_BITS = 0            # 0: m kept in the activation type; 2, 4, 8: low-precision store (--m-bits)
-
-
-def bytes_per_element(bits, group):
+def bytes_per_element(bits, group, m_bits=0):
     """Algorithmic HBM bytes per element of a steady-state encode (= of a decode):
     read a (2) + read m (2) + write m (2) + codes (b/8) + scale (4/G); with m kept in z bits:
     a (2) + m read and written (2 * (z/8 + 4/G)) + codes (b/8) + scale (4/G)."""
-    if M_BITS == 32:                                  # binary32 store: no steps
+    if m_bits == 32:                                  # binary32 store: no steps
         return 2.0 + 8.0 + bits / 8.0 + 4.0 / group
-    if M_BITS:
-        return 2.0 + 2.0 * (M_BITS / 8.0 + 4.0 / group) + bits / 8.0 + 4.0 / group
+    if m_bits:
+        return 2.0 + 2.0 * (m_bits / 8.0 + 4.0 / group) + bits / 8.0 + 4.0 / group
     return 6.0 + bits / 8.0 + 4.0 / group
 
 
@@ -194,6 +215,69 @@ def time_oracle(cfg, budget_s, device, max_samples=256):
     return gb / spent, done / spent, done, spent
 
 
+def _oracle_worker(job):
+    """One process of the all-cores leg: the unchanged single-threaded oracle on this worker's own
+    samples (first visits untimed), then, once every worker is ready, delta visits that alternate
+    between two epochs of each sample until the budget is spent.  Returns (visits, seconds)."""
+    path, which, shape, bits, group, dtype, budget_s, ready_at = job
+    import numpy as np
+    import oracle
+    n_ids, seq, hidden = len(which), shape[0], shape[1]
+    acts = np.load(path, mmap_mode="r")                          # [n_pool, 2, seq, hidden] uint16
+    mine = [np.ascontiguousarray(acts[w]) for w in which]
+    snd = oracle.Side(n_ids, seq, hidden, bits, group, dtype)
+    rcv = oracle.Side(n_ids, seq, hidden, bits, group, dtype)
+    for j in range(n_ids):
+        ids = np.array([j], np.int32)
+        p, s, _ = snd.encode(mine[j][0:1], ids)
+        rcv.decode(p, s, ids, raw=mine[j][0:1])
+    while time.time() < ready_at:                                # every worker starts its timed visits together
+        time.sleep(0.005)
+    visits, t0 = 0, time.perf_counter()
+    while time.perf_counter() - t0 < budget_s:
+        j, e = visits % n_ids, 1 - (visits // n_ids) % 2
+        ids = np.array([j], np.int32)
+        p, s, _ = snd.encode(mine[j][e:e + 1], ids)
+        rcv.decode(p, s, ids)
+        visits += 1
+    return visits, time.perf_counter() - t0
+
+
+def time_oracle_all_cores(cfg, budget_s, device):
+    """The same oracle, one worker process per host core, no threading inside it: every worker
+    visits its own samples.  Returns a dict for cpu_baseline.all_cores."""
+    import multiprocessing as mp
+    import tempfile
+    import numpy as np
+    import oracle
+    from fixtures import synth
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+    per_worker = 2
+    pool_ids = min(per_worker * cores, 64)                       # bounded input set: workers beyond 32 share samples
+    small = synth.shrink(cfg, pool_ids)
+    acts = np.empty((pool_ids, 2, cfg.seq, cfg.hidden), np.uint16)
+    for i in range(pool_ids):
+        for e in (0, 1):
+            acts[i, e] = bits16(synth.activation(small, [i], e, device=device))[0]
+    od = oracle.FP16 if cfg.dtype == "fp16" else oracle.BF16
+    with tempfile.TemporaryDirectory() as tmp:
+        path = os.path.join(tmp, "acts.npy")
+        np.save(path, acts)
+        ready_at = time.time() + 6.0 + 0.02 * cores               # start-up of the workers (imports, first visits)
+        jobs = [(path, [(per_worker * w + j) % pool_ids for j in range(per_worker)], (cfg.seq, cfg.hidden), cfg.bits,
+                 cfg.group, od, budget_s, ready_at) for w in range(cores)]
+        ctx = mp.get_context("spawn")
+        with ctx.Pool(cores) as pool:
+            got = pool.map(_oracle_worker, jobs, chunksize=1)
+    visits = sum(v for v, _ in got)
+    secs = max(s for _, s in got)
+    gb = 2 * visits * cfg.elems * bytes_per_element(cfg.bits, cfg.group) / 1e9
+    return {"value": gb / secs, "unit": "GB/s", "cores": cores, "samples_per_s": visits / secs,
+            "sample": f"{cores} worker processes (one per host core, nproc = {cores}), each the single-threaded oracle on "
+                      f"{per_worker} whole sequences of its own ({pool_ids} distinct sequences in all), steady-state "
+                      f"encode+decode visits for {budget_s:.0f} s: {visits} visits"}
+
+
 def run_reference(args, cfg):
     """The oracle as the reference arm: each step = steady-state encode + decode of `rows`
     token rows of one sample (a bounded sample of the macro-batch step), on one host core."""
@@ -248,75 +332,63 @@ def run_reference(args, cfg):
 
 # ------------------------------------------------------------------------------------ GPU arm
 
-def main():
-    args = parse_args()
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+class Env:
+    """What every measurement needs: the process's rank, the process group (or None), the stream."""
 
+    def __init__(self, rank, local_rank, world, dist, stream):
+        self.rank, self.local_rank, self.world, self.dist, self.stream = rank, local_rank, world, dist, stream
+
+
+def measure_boundary(args, env, name, steps, warmup, headline):
+    """One forward boundary at full size (or --n-samples): first-visit epoch, `repeats` timed windows of
+    `steps` steady-state steps, per-kernel durations, calls of the workload's own micro-batch size, and for
+    the headline workload the isolated-call, end-to-end and remaining-kernel figures.  Returns a dict; the
+    handles and every buffer are gone when it returns."""
+    import numpy as np
+    import torch
     from dataclasses import replace
+    import paper_2206_01299_b200 as aq
     from fixtures import replicas, synth
-    global MACRO, M_BITS
-    M_BITS = args.m_bits
-    recipe, MACRO, label = WORKLOADS[args.workload]
+
+    rank, local_rank, world, dist, stream = env.rank, env.local_rank, env.world, env.dist, env.stream
+    recipe, macro, label = WORKLOADS[name]
     cfg = getattr(synth, recipe)
     if args.n_samples:
         cfg = synth.shrink(cfg, args.n_samples)
-
-    if args.impl == "reference":
-        if rank == 0:
-            run_reference(args, cfg)
-        return
-
-    import numpy as np
-    import torch
-    import paper_2206_01299_b200 as aq
-    aq.lib()                                         # fails loudly when the CUDA library is missing
-    assert torch.cuda.is_available(), "bench.py needs a CUDA device; there is no CPU path"
-    torch.cuda.set_device(local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-    # data-parallel replicas: every rank owns its own 4096-id shard of a world-times larger id
-    # space (weak scaling); sample rows never cross ranks, so the data path has no collective
+    # data-parallel replicas: every rank owns its own id shard of a world-times larger id space (weak
+    # scaling); sample rows never cross ranks, so the data path has no collective
     cfg = replicas.shard_for_rank(cfg, rank, world)
+    m_bits = args.m_bits if headline else 0
+    hosted, prefetching = (args.hosted, args.prefetch) if headline else (False, False)
+    stochastic = headline and args.rounding == "stochastic"
+    use_graph = headline and args.graph
 
-    nb = args.per_launch or MACRO
-    assert cfg.n_samples % MACRO == 0 and MACRO % nb == 0
-    steps_per_epoch = cfg.n_samples // MACRO
-    launches_per_step = MACRO // nb
-    total_steps = args.steps + args.warmup
-    # resident steady-state epochs: as many as the timed steps need, at most 4 (2 for the 26 GB boundary)
+    nb = (args.per_launch if headline else 0) or macro
+    assert cfg.n_samples % macro == 0 and macro % nb == 0
+    steps_per_epoch = cfg.n_samples // macro
+    launches_per_step = macro // nb
+    # resident steady-state epochs: at most 4 (2 for the 26 GB boundaries), fewer when the id space is small
     max_arenas = 4 if cfg.n_samples * cfg.elems * 2 < 20e9 else 2
-    n_arenas = min(max_arenas, (total_steps + steps_per_epoch - 1) // steps_per_epoch)
-    stream = torch.cuda.Stream()
-    bpe = bytes_per_element(cfg.bits, cfg.group)
-    step_bytes = 2 * MACRO * cfg.elems * bpe          # encode + decode
+    n_arenas = max(1, min(max_arenas, (steps + warmup + steps_per_epoch - 1) // steps_per_epoch))
+    bpe = bytes_per_element(cfg.bits, cfg.group, m_bits)
+    step_bytes = 2 * macro * cfg.elems * bpe          # encode + decode
 
-    if args.prefetch and not args.hosted:
-        raise SystemExit("--prefetch needs --hosted")
-    if args.hosted and args.m_bits == 32:
-        raise SystemExit("the binary32 store is not offered in host memory")
-    handles = []
-    for _ in range(2):
-        h = (aq.aq_create_hosted_lowbit(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, args.m_bits) if args.m_bits in (2, 4, 8) and args.hosted
-             else aq.aq_create_fp32(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group) if args.m_bits == 32
-             else aq.aq_create_lowbit(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, args.m_bits) if args.m_bits
-             else aq.aq_create_hosted(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group) if args.hosted
+    def create():
+        h = (aq.aq_create_hosted_lowbit(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, m_bits) if m_bits in (2, 4, 8) and hosted
+             else aq.aq_create_fp32(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group) if m_bits == 32
+             else aq.aq_create_lowbit(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, m_bits) if m_bits
+             else aq.aq_create_hosted(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group) if hosted
              else aq.aq_create(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group))
         aq.aq_configure(h, aq.AQ_DTYPE, aq.AQ_FP16 if cfg.dtype == "fp16" else aq.AQ_BF16)
         aq.aq_configure(h, aq.AQ_BATCH, nb)
         aq.aq_configure(h, aq.AQ_STREAM, stream.cuda_stream)
-        if args.rows_per_cta:
-            aq.aq_configure(h, aq.AQ_ROWS_PER_CTA, args.rows_per_cta)
-        if args.no_l2_prefetch:
-            aq.aq_configure(h, aq.AQ_L2_PREFETCH, 0)
-        if args.rounding == "stochastic":
+        if stochastic:
             aq.aq_configure(h, aq.AQ_ROUNDING, aq.AQ_ROUND_STOCHASTIC)
             aq.aq_configure(h, aq.AQ_SEED, 20220601)
-        handles.append(h)
-    snd, rcv = handles
+        return h
+
+    snd, rcv = create(), create()
+    handles = [snd, rcv]
 
     # fp32 running sum A_e of every sample in id order (the recipe's state), advanced one epoch at a time;
     # id spaces too large for that (4 B per element beside the two m arrays) recompute A_e per chunk instead
@@ -343,22 +415,23 @@ def main():
             arena[c:c + 64] = running[order_dev[c:c + 64]].to(cfg.torch_dtype).reshape(-1, cfg.seq, cfg.hidden)
         return arena
 
-    packed = torch.empty((MACRO, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
-    scales = torch.empty((MACRO, cfg.groups), dtype=torch.float32, device="cuda")
-    out = torch.empty((MACRO, cfg.seq, cfg.hidden), dtype=cfg.torch_dtype, device="cuda")
+    packed = torch.empty((macro, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
+    scales = torch.empty((macro, cfg.groups), dtype=torch.float32, device="cuda")
+    out = torch.empty((macro, cfg.seq, cfg.hidden), dtype=cfg.torch_dtype, device="cuda")
 
-    sweep = args.workload == "sweep"
+    sweep = name == "sweep"
     if sweep:
         # receiver's ends of the forward wire, both ends of the backward wire, rotating gradients (4 x 52 MB > L2)
         bw = synth.SWEEP_BWD
-        bbits, n_grad = bw.bits[0], MACRO * cfg.elems
+        bbits, n_grad = bw.bits[0], macro * cfg.elems
         rx_packed, rx_scales = torch.empty_like(packed), torch.empty_like(scales)
-        grads = [synth.gradient(replace(bw, n_batch=MACRO), i, device="cuda") for i in range(4)]
+        grads = [synth.gradient(replace(bw, n_batch=macro), i, device="cuda") for i in range(4)]
         g_tx = (torch.empty(n_grad * bbits // 8, dtype=torch.uint8, device="cuda"), torch.empty(n_grad // bw.group, dtype=torch.float32, device="cuda"))
         g_rx = (torch.empty_like(g_tx[0]), torch.empty_like(g_tx[1]))
         g_out = torch.empty(n_grad, dtype=cfg.torch_dtype, device="cuda")
-        step_bytes += (2 * n_grad * (2 + bbits / 8 + 4 / bw.group)                      # quantize + dequantize
-                       + 2 * (MACRO * (cfg.packed_bytes + cfg.groups * 4))             # forward wire: read + write
+        grad_bytes = n_grad * (2 + bbits / 8 + 4 / bw.group)
+        step_bytes += (2 * grad_bytes                                                  # quantize + dequantize
+                       + 2 * (macro * (cfg.packed_bytes + cfg.groups * 4))             # forward wire: read + write
                        + 2 * (n_grad * bbits // 8 + n_grad // bw.group * 4))           # backward wire
 
     host_ids = {}                                      # device id list -> its host copy (aq_prefetch reads ids on the host)
@@ -374,9 +447,8 @@ def main():
 
     # stand-in for the stage's own work: a kernel that occupies the handles' stream for a fixed number of
     # clock cycles and draws next to no power, so that its duration does not depend on what runs beside it
-    # (dense matrix products throttle under the power cap, by another amount in every mode compared)
     stage_cycles, stage_ms = 0, 0.0
-    if args.stage_compute_ms > 0:
+    if headline and args.stage_compute_ms > 0:
         stage_cycles = int(args.stage_compute_ms * 1e-3 * 1.965e9)
         with torch.cuda.stream(stream):
             torch.cuda._sleep(stage_cycles)
@@ -389,15 +461,15 @@ def main():
         stage_ms = c0.elapsed_time(c1) / 4
 
     def run_step(arena, ids_dev, s, raw=False, nxt=None):
-        """One macro-batch: MACRO micro-batches in launches of nb, each encoded then decoded (the pipeline
+        """One macro-batch: its micro-batches in launches of nb, each encoded then decoded (the pipeline
         sweep: encode, wire, decode, then the gradient of the macro-batch quantized, wired and dequantized).
         nxt = (ids_dev, s) of the step that follows: with --prefetch its rows are asked for as soon as this
         step's calls are issued, so that they travel while the stage computes."""
         for l in range(launches_per_step):
-            lo = s * MACRO + l * nb
+            lo = s * macro + l * nb
             a, i = arena[lo:lo + nb], ids_dev[lo:lo + nb]
             p, sc, o = packed[l * nb:(l + 1) * nb], scales[l * nb:(l + 1) * nb], out[l * nb:(l + 1) * nb]
-            if args.prefetch and ahead["key"] != (ids_dev.data_ptr(), lo):
+            if prefetching and ahead["key"] != (ids_dev.data_ptr(), lo):
                 prefetch(ids_dev, lo)
             aq.aq_encode(snd, a, i, p, sc)
             if raw:
@@ -409,53 +481,69 @@ def main():
             else:
                 aq.aq_decode(rcv, p, sc, i, o)
         ahead["key"] = None
-        if args.prefetch and nxt is not None and launches_per_step == 1:
-            prefetch(nxt[0], nxt[1] * MACRO)
-            ahead["key"] = (nxt[0].data_ptr(), nxt[1] * MACRO)
+        if prefetching and nxt is not None and launches_per_step == 1:
+            prefetch(nxt[0], nxt[1] * macro)
+            ahead["key"] = (nxt[0].data_ptr(), nxt[1] * macro)
         if stage_cycles:
             torch.cuda._sleep(stage_cycles)
         if sweep:
             aq.aq_quant_grad(rcv, grads[s % 4], n_grad, bbits, g_tx[0], g_tx[1])
-            g_rx[0].copy_(g_tx[0], non_blocking=True)    # the backward wire (same stream as the handles)
-            g_rx[1].copy_(g_tx[1], non_blocking=True)
+            aq.aq_wire_copy_grad(rcv, local_rank, g_rx[0], g_rx[1], g_tx[0], g_tx[1], n_grad, bbits)    # the backward wire
             aq.aq_dequant_grad(snd, g_rx[0], g_rx[1], n_grad, bbits, g_out)
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
 
     def kernel_pass(first_step, window):
         """Average duration of one encode launch and of one decode launch: `window` steps whose
         encode launches run back to back between one pair of events, then their decode launches
         between another (the wire buffers of the whole window are kept in between).  An event
         between every two launches would add about 2 us of idle stream time per event."""
-        wp = torch.empty((window, MACRO, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
-        ws = torch.empty((window, MACRO, cfg.groups), dtype=torch.float32, device="cuda")
+        wp = torch.empty((window, macro, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
+        ws = torch.empty((window, macro, cfg.groups), dtype=torch.float32, device="cuda")
         e = [ev(), ev(), ev()]
         e[0].record(stream)
         for w in range(window):
             arena, ids_dev, s = step_source(first_step + w)
             for l in range(launches_per_step):
-                lo = s * MACRO + l * nb
+                lo = s * macro + l * nb
                 aq.aq_encode(snd, arena[lo:lo + nb], ids_dev[lo:lo + nb], wp[w, l * nb:(l + 1) * nb], ws[w, l * nb:(l + 1) * nb])
         e[1].record(stream)
         for w in range(window):
             arena, ids_dev, s = step_source(first_step + w)
             for l in range(launches_per_step):
-                lo = s * MACRO + l * nb
+                lo = s * macro + l * nb
                 aq.aq_decode(rcv, wp[w, l * nb:(l + 1) * nb], ws[w, l * nb:(l + 1) * nb], ids_dev[lo:lo + nb], out[l * nb:(l + 1) * nb])
         e[2].record(stream)
         torch.cuda.synchronize()
         n = window * launches_per_step
         return e[0].elapsed_time(e[1]) / n, e[1].elapsed_time(e[2]) / n
 
-    ev = lambda: torch.cuda.Event(enable_timing=True)
+    def grad_pass(window):
+        """The same for the sweep's backward kernels: `window` quantize launches back to back, then
+        `window` dequantize launches (one wire buffer per rotating gradient)."""
+        tx = [(torch.empty_like(g_tx[0]), torch.empty_like(g_tx[1])) for _ in range(4)]
+        for i in range(4):
+            aq.aq_quant_grad(rcv, grads[i], n_grad, bbits, tx[i][0], tx[i][1])
+        e = [ev(), ev(), ev()]
+        e[0].record(stream)
+        for w in range(window):
+            aq.aq_quant_grad(rcv, grads[w % 4], n_grad, bbits, tx[w % 4][0], tx[w % 4][1])
+        e[1].record(stream)
+        for w in range(window):
+            aq.aq_dequant_grad(snd, tx[w % 4][0], tx[w % 4][1], n_grad, bbits, g_out)
+        e[2].record(stream)
+        torch.cuda.synchronize()
+        return e[0].elapsed_time(e[1]) / window, e[1].elapsed_time(e[2]) / window
 
     # one throw-away visit on a small boundary of the same type, bit width and group: the first launch of a
     # kernel loads its code (milliseconds), which must not count as first-visit time
-    warm = [aq.aq_create_fp32(2, 8, cfg.hidden, cfg.bits, cfg.group) if args.m_bits == 32
-            else aq.aq_create_lowbit(2, 8, cfg.hidden, cfg.bits, cfg.group, args.m_bits) if args.m_bits
+    warm = [aq.aq_create_fp32(2, 8, cfg.hidden, cfg.bits, cfg.group) if m_bits == 32
+            else aq.aq_create_lowbit(2, 8, cfg.hidden, cfg.bits, cfg.group, m_bits) if m_bits
             else aq.aq_create(2, 8, cfg.hidden, cfg.bits, cfg.group) for _ in range(2)]
     for h in warm:
         aq.aq_configure(h, aq.AQ_DTYPE, aq.AQ_FP16 if cfg.dtype == "fp16" else aq.AQ_BF16)
         aq.aq_configure(h, aq.AQ_STREAM, stream.cuda_stream)
-        if args.rounding == "stochastic":
+        if stochastic:
             aq.aq_configure(h, aq.AQ_ROUNDING, aq.AQ_ROUND_STOCHASTIC)
     w_act = torch.zeros((1, 8, cfg.hidden), dtype=cfg.torch_dtype, device="cuda")
     w_ids = torch.zeros(1, dtype=torch.int32, device="cuda")
@@ -496,46 +584,68 @@ def main():
         e = (t // steps_per_epoch) % n_arenas
         return arenas[e], id_lists[e], t % steps_per_epoch
 
+    # ---- the timed region: `repeats` windows of exactly `steps` steps each
     graphs = None
-    if args.graph:
-        # one graph per step (pointers differ from step to step); capture enqueues nothing
+    if use_graph:
+        # one graph per step of a window (pointers differ from step to step); capture enqueues nothing
         graphs = []
-        for t in range(total_steps):
+        for t in range(steps):
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g, stream=stream):
-                run_step(*step_source(t))
+                run_step(*step_source(warmup + t))
             graphs.append(g)
-    t_begin, t_end = ev(), ev()
+    windows_ms, walls_ms = [], []
     with torch.cuda.stream(stream):
-        for t in range(args.warmup):
-            graphs[t].replay() if graphs else run_step(*step_source(t))
-        torch.cuda.synchronize()
-        if dist:
-            dist.barrier()
+        for t in range(warmup):
+            graphs[t % steps].replay() if graphs else run_step(*step_source(t))
         torch.cuda.synchronize()
         with ClockSampler(local_rank) as clocks:
-            wall0 = time.perf_counter()
-            # about 0.1 ms of an idle-spinning kernel ahead of the start event: the host queues the event and the
-            # first launches behind it, so that the clock starts with work waiting and not with launch latency
-            if hasattr(torch.cuda, "_sleep"):
-                torch.cuda._sleep(200_000)
-            t_begin.record(stream)
-            for t in range(args.steps):
-                if graphs:
-                    graphs[args.warmup + t].replay()
-                else:
-                    run_step(*step_source(args.warmup + t), nxt=step_source(args.warmup + t + 1)[1:])
-            t_end.record(stream)
-            torch.cuda.synchronize()
-            wall_ms = (time.perf_counter() - wall0) * 1e3
-        if dist:
-            dist.barrier()
-        torch.cuda.synchronize()
-    # staged calls end with copies on the handles' own copy streams, which the event on `stream` does
-    # not cover: there the step time is the host's, taken between two whole-device synchronisations
-    elapsed_ms = wall_ms if args.prefetch else t_begin.elapsed_time(t_end)
+            repeats, r, t_next = 30, 0, warmup
+            while r < repeats:
+                t_begin, t_end = ev(), ev()
+                if dist:
+                    dist.barrier()
+                torch.cuda.synchronize()
+                wall0 = time.perf_counter()
+                # about 0.1 ms of an idle-spinning kernel ahead of the start event: the host queues the event and the
+                # first launches behind it, so that the clock starts with work waiting and not with launch latency
+                if hasattr(torch.cuda, "_sleep"):
+                    torch.cuda._sleep(200_000)
+                t_begin.record(stream)
+                for t in range(steps):
+                    if graphs:
+                        graphs[t].replay()
+                    else:
+                        run_step(*step_source(t_next + t), nxt=step_source(t_next + t + 1)[1:])
+                t_end.record(stream)
+                torch.cuda.synchronize()
+                walls_ms.append((time.perf_counter() - wall0) * 1e3)
+                if dist:
+                    dist.barrier()
+                torch.cuda.synchronize()
+                # staged calls end with copies on the handles' own copy streams, which the event on `stream` does
+                # not cover: there the window's time is the host's, taken between two whole-device synchronisations
+                windows_ms.append(walls_ms[-1] if prefetching else t_begin.elapsed_time(t_end))
+                t_next += steps
+                r += 1
+                if r == 3:                                        # size the run from the first windows
+                    est = statistics.median(windows_ms)
+                    want = max(30, math.ceil(args.min_timed_ms / max(est, 1e-3)))
+                    if dist:                                      # the same count on every rank
+                        t = torch.tensor([want], device="cuda")
+                        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+                        want = int(t.item())
+                    repeats = min(max(args.max_repeats, 30), want)
+    total_steps = t_next
+    # the slowest rank sets the time of every window
+    if dist:
+        t = torch.tensor(windows_ms, dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        windows_ms = t.cpu().tolist()
+    elapsed_ms = statistics.median(windows_ms)
+
     staged_call_us = None
-    if args.prefetch:
+    if prefetching:
         # the calls' time once their rows have arrived: what stays on the critical path of a pipeline stage
         lat = []
         with torch.cuda.stream(stream):
@@ -543,7 +653,7 @@ def main():
                 run_step(*step_source(total_steps))
             for r in range(8):
                 arena, ids_dev, sidx = step_source(total_steps + 1 + r)
-                lo = sidx * MACRO
+                lo = sidx * macro
                 prefetch(ids_dev, lo)
                 torch.cuda.synchronize()
                 a0, a1 = ev(), ev()
@@ -554,79 +664,223 @@ def main():
                 torch.cuda.synchronize()
                 lat.append(a0.elapsed_time(a1) * 1e3)
         staged_call_us = statistics.median(lat)
-    # per-kernel durations: the steps that follow the timed ones, same handles, same data
+
+    # ---- per-kernel durations: the steps that follow the timed ones, same handles, same data
     window = min(32, steps_per_epoch)
     with torch.cuda.stream(stream):
-        passes = [kernel_pass(total_steps + r * window, window) for r in range(3)]
+        passes = [kernel_pass(total_steps + 2 + r * window, window) for r in range(3)]
+        grad_passes = [grad_pass(32) for r in range(3)] if sweep else None
     enc_ms = statistics.median(p[0] for p in passes)          # one disturbed pass must not move the figure
     dec_ms = statistics.median(p[1] for p in passes)
+
+    # ---- calls of the workload's own micro-batch size, enqueued back to back on the plain stream and as one CUDA graph
+    micro = None
+    if not (hosted or use_graph) and nb != cfg.n_batch:
+        micro = micro_batch_calls(aq, torch, stream, snd, rcv, cfg, step_source, total_steps + 2 + 3 * window, macro, packed, scales, out,
+                                  bpe)
+        for h in handles:
+            aq.aq_configure(h, aq.AQ_BATCH, nb)
+
     status = aq.aq_status(snd) | aq.aq_status(rcv)
     digests_equal = aq.aq_state_checksum(snd) == aq.aq_state_checksum(rcv)
     assert status == 0 and digests_equal, "sender and receiver state diverged"
-
-    elapsed_ms = replicas.max_over_ranks(elapsed_ms, dist, "cuda")
-
-    result_extra = {}
-    if rank == 0 and not args.skip_aux:
-        result_extra["isolated_call"] = isolated_calls(aq, torch, stream, snd, rcv, cfg, arenas[0], id_lists[0])
-        result_extra["aux"] = aux_kernels(aq, torch, synth, stream, snd, cfg)
-
-    # ---- end to end through the host-buffer entry points (pinned host memory both ways)
-    e2e = None
-    if not args.skip_e2e:
-        e2e = run_e2e(aq, torch, cfg, snd, rcv, arenas[0], id_lists[0], args.e2e_steps, dist)
-
-    cpu = None
-    if rank == 0 and not args.skip_cpu:
-        gbs, sps, n, secs = time_oracle(cfg, args.cpu_seconds, "cuda")
-        cpu = {"value": gbs, "unit": "GB/s", "cores": 1, "kind": "oracle", "samples_per_s": sps,
-               "sample": f"steady-state encode+decode of {n} whole sequences ({n * cfg.elems} elements, {secs:.1f} s), single thread"}
-
-    for h in handles:
-        aq.aq_destroy(h)
-    if dist:
-        dist.destroy_process_group()
-    if rank != 0:
-        return
 
     peak, peak_kind = measured_peak()
     launch_bytes = nb * cfg.elems * bpe
     enc_gbs = launch_bytes / (enc_ms * 1e-3) / 1e9
     dec_gbs = launch_bytes / (dec_ms * 1e-3) / 1e9
-    traffic = NCU_TRAFFIC_BYTES_PER_ELEMENT["encode"] if (args.workload == NCU_TRAFFIC_WORKLOAD and args.rounding == "interval"
-                                                          and not args.m_bits and not args.hosted and not args.no_l2_prefetch) else None
-    value = replicas.whole_job_rate(args.steps * step_bytes, world, elapsed_ms) / 1e9
-    line = {
-        "metric": "activation encode+decode GB/s", "value": value, "unit": "GB/s",
-        "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": label, "hidden": cfg.hidden, "seq": cfg.seq,
-                   "micro_batch": cfg.n_batch, "sequences_per_step": MACRO, "sequences_per_launch": nb, "cuda_graph": bool(args.graph), "l2_prefetch": not args.no_l2_prefetch and not args.hosted, "rounding": args.rounding, "m_bits": args.m_bits or 16,
-                   "m_in": ("host memory (page-locked), staged through HBM by aq_prefetch, written back on a copy stream; step time by the host clock" if args.prefetch
-                            else "host memory (page-locked, mapped)" if args.hosted else "HBM"),
-                   "act_dtype": cfg.dtype, "bits": cfg.bits, "group": cfg.group, "n_samples_per_side": cfg.n_samples,
-                   "m_bytes_per_side": cfg.n_samples * (cfg.elems * 2 if not args.m_bits else cfg.elems * args.m_bits // 8 + (0 if args.m_bits == 32 else cfg.groups * 4)), "steady_epochs_resident": n_arenas,
-                   "l2": f"inputs larger than L2 (each step touches {int(MACRO * cfg.elems * 6 / 1e6)} MB of fresh HBM; no flush needed)",
-                   "parallelism": f"dp{world} replicas, no collective"},
-        "samples_per_s": replicas.whole_job_rate(args.steps * MACRO, world, elapsed_ms),
+    value = replicas.whole_job_rate(steps * step_bytes, world, elapsed_ms) / 1e9
+    res = {
+        "workload": label, "value": value, "ms_per_step": elapsed_ms / steps,
+        "timed": {"windows": len(windows_ms), "steps_per_window": steps, "ms_per_step_min": min(windows_ms) / steps,
+                  "ms_per_step_max": max(windows_ms) / steps, "gpu_ms_total": sum(windows_ms)},
+        "samples_per_s": replicas.whole_job_rate(steps * macro, world, elapsed_ms),
         "frac_of_measured_hbm": value / world / peak, "frac_of_8000_spec": value / world / 8000.0,
-        "roofline": {"bound": "hbm", "kernel": "encode_kernel", "achieved": enc_gbs, "peak": peak, "unit": "GB/s",
-                     "frac": enc_gbs / peak, "peak_kind": peak_kind,
-                     "traffic": None if traffic is None else traffic * nb * cfg.elems,
-                     "algorithmic_bytes_per_launch": launch_bytes, "avg_launch_ms": enc_ms,
-                     "timing": f"CUDA events around {window * launches_per_step} back-to-back launches of the kernel, median of 3 passes right after the timed steps",
-                     "decode_kernel": {"achieved": dec_gbs, "frac": dec_gbs / peak, "avg_launch_ms": dec_ms}},
+        "step_bytes": step_bytes, "launch_bytes": launch_bytes, "bytes_per_element": bpe,
+        "encode": {"achieved": enc_gbs, "frac": enc_gbs / peak, "avg_launch_ms": enc_ms},
+        "decode": {"achieved": dec_gbs, "frac": dec_gbs / peak, "avg_launch_ms": dec_ms},
+        "kernel_timing": f"CUDA events around {window * launches_per_step} back-to-back launches of the kernel, median of 3 passes right after the timed steps",
         "first_visit_epoch": {"ms": first_ms, "GB/s": first_bytes / (first_ms * 1e-3) / 1e9},
-        "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": args.steps * (launches_per_step * 2 + (2 if sweep else 0)),
-        "clocks": clocks.summary(),
+        "micro_batch_calls": micro, "clocks": clocks.summary(),
+        "gpu_launches_per_step": launches_per_step * (3 if sweep else 2) + (3 if sweep else 0),
+        "peak": peak, "peak_kind": peak_kind,
+        "shape": {"hidden": cfg.hidden, "seq": cfg.seq, "micro_batch": cfg.n_batch, "sequences_per_step": macro,
+                  "sequences_per_launch": nb, "act_dtype": cfg.dtype, "bits": cfg.bits, "group": cfg.group,
+                  "n_samples_per_side": cfg.n_samples, "steady_epochs_resident": n_arenas},
     }
+    if sweep:
+        q_ms = statistics.median(p[0] for p in grad_passes)
+        d_ms = statistics.median(p[1] for p in grad_passes)
+        res["quant_grad"] = {"bits": bbits, "achieved": grad_bytes / q_ms / 1e6, "frac": grad_bytes / q_ms / 1e6 / peak, "avg_launch_ms": q_ms}
+        res["dequant_grad"] = {"bits": bbits, "achieved": grad_bytes / d_ms / 1e6, "frac": grad_bytes / d_ms / 1e6 / peak, "avg_launch_ms": d_ms}
     if staged_call_us is not None:
-        line["staged_encode_plus_decode_us"] = staged_call_us
+        res["staged_encode_plus_decode_us"] = staged_call_us
     if stage_cycles:
-        line["config"]["stage_compute_ms_per_step"] = stage_ms
-    line.update(result_extra)
-    print(json.dumps(line))
+        res["stage_compute_ms_per_step"] = stage_ms
+
+    if headline:
+        if rank == 0 and not args.skip_aux:
+            res["isolated_call"] = isolated_calls(aq, torch, stream, snd, rcv, cfg, arenas[0], id_lists[0])
+            res["aux"] = aux_kernels(aq, torch, synth, stream, snd, cfg)
+        # ---- end to end through the host-buffer entry points (pinned host memory both ways)
+        res["e2e"] = None
+        if not args.skip_e2e:
+            res["e2e"] = run_e2e(aq, torch, cfg, snd, rcv, arenas[0], id_lists[0], args.e2e_steps, dist, macro, bpe)
+        res["cpu_baseline"] = None
+        if rank == 0 and not args.skip_cpu:
+            gbs, sps, n, secs = time_oracle(cfg, args.cpu_seconds, "cuda")
+            res["cpu_baseline"] = {
+                "value": gbs, "unit": "GB/s", "cores": 1, "kind": "oracle", "samples_per_s": sps,
+                "sample": f"steady-state encode+decode of {n} whole sequences ({n * cfg.elems} elements, {secs:.1f} s), single thread",
+                "all_cores": time_oracle_all_cores(cfg, args.cpu_seconds, "cuda")}
+    res["cfg"] = cfg
+    for h in handles:
+        aq.aq_destroy(h)
+    del arenas, id_lists, packed, scales, out
+    torch.cuda.empty_cache()
+    return res
+
+
+def measure_pipeline(args, env):
+    """One boundary per pair of ranks: rank 2p owns the sender handle and the activations, rank 2p+1 the
+    receiver handle; codes, steps and (epoch 0) the raw blocks cross between the two GPUs through
+    BoundaryLink (NCCL send / recv into the receiver's own buffers), after which aq_decode reads locally.
+    Timed like the replica run: windows of `steps` steps between barriers, the slowest rank sets the time."""
+    import torch
+    import paper_2206_01299_b200 as aq
+    from paper_2206_01299_b200.link import BoundaryLink
+    from fixtures import replicas, synth
+
+    rank, world, dist, stream = env.rank, env.world, env.dist, env.stream
+    assert dist is not None and world % 2 == 0, "--topology pipeline needs an even number of ranks"
+    pair, sender = rank // 2, rank % 2 == 0
+    recipe, macro, label = WORKLOADS[args.workload]
+    cfg = getattr(synth, recipe)
+    if args.n_samples:
+        cfg = synth.shrink(cfg, args.n_samples)
+    cfg = replicas.shard_for_rank(cfg, pair, world // 2)
+    nb, steps, warmup = macro, args.steps, args.warmup
+    steps_per_epoch = cfg.n_samples // macro
+    bpe = bytes_per_element(cfg.bits, cfg.group)
+
+    h = aq.aq_create(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group)
+    aq.aq_configure(h, aq.AQ_DTYPE, aq.AQ_FP16 if cfg.dtype == "fp16" else aq.AQ_BF16)
+    aq.aq_configure(h, aq.AQ_BATCH, nb)
+    aq.aq_configure(h, aq.AQ_STREAM, stream.cuda_stream)
+    first = torch.zeros(nb, dtype=torch.uint8, device="cuda")
+    aq.aq_configure(h, aq.AQ_FIRST_FLAGS, first)
+    link = BoundaryLink(dist, rank + 1 if sender else rank - 1, nb, cfg.packed_bytes, cfg.groups, cfg.elems, cfg.torch_dtype, "cuda")
+    packed = torch.empty((nb, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
+    scales = torch.empty((nb, cfg.groups), dtype=torch.float32, device="cuda")
+    out = torch.empty((nb, cfg.seq, cfg.hidden), dtype=cfg.torch_dtype, device="cuda")
+    orders = [synth.epoch_order(cfg, e) for e in range(2)]
+
+    def arena_of(epoch):
+        a = torch.empty((cfg.n_samples, cfg.seq, cfg.hidden), dtype=cfg.torch_dtype, device="cuda")
+        for c in range(0, cfg.n_samples, 16):
+            a[c:c + 16] = synth.activation(cfg, orders[epoch][c:c + 16], epoch, device="cuda")
+        return a
+
+    def step(epoch, arena, s):
+        ids = orders[epoch][s * macro:(s + 1) * macro]
+        with torch.cuda.stream(stream):
+            if sender:
+                act = arena[s * macro:(s + 1) * macro]
+                aq.aq_encode(h, act, ids.cuda(), packed, scales)
+                stream.synchronize()                      # the link's sends run on the process group's stream
+                link.send(ids, first, packed, scales, act)
+            else:
+                _, _, p, sc, raw = link.recv(expect_ids=ids)
+                aq.aq_configure(h, aq.AQ_RAW, raw)
+                aq.aq_decode(h, p, sc, ids.cuda(), out)
+                stream.synchronize()
+
+    arena = arena_of(0) if sender else None
+    for s in range(steps_per_epoch):                       # epoch 0: first visits, untimed
+        step(0, arena, s)
+    arena = arena_of(1) if sender else None
+    windows_ms, t = [], 0
+    for s in range(warmup):
+        step(1, arena, (t := t + 1) % steps_per_epoch)
+    for r in range(30):
+        dist.barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for s in range(steps):
+            step(1, arena, (t := t + 1) % steps_per_epoch)
+        torch.cuda.synchronize()
+        windows_ms.append((time.perf_counter() - t0) * 1e3)
+    ms = torch.tensor(windows_ms, dtype=torch.float64, device="cuda")
+    dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+    digest = torch.tensor([aq.aq_state_checksum(h) & 0x7FFFFFFFFFFFFFFF], dtype=torch.int64, device="cuda")
+    both = [torch.zeros_like(digest) for _ in range(world)]
+    dist.all_gather(both, digest)
+    assert all(both[2 * p].item() == both[2 * p + 1].item() for p in range(world // 2)), "sender and receiver state diverged"
+    assert aq.aq_status(h) == 0
+    aq.aq_destroy(h)
+    elapsed = statistics.median(ms.cpu().tolist())
+    step_bytes = 2 * macro * cfg.elems * bpe
+    value = (world // 2) * steps * step_bytes / (elapsed * 1e-3) / 1e9
+    wire = macro * (cfg.packed_bytes + cfg.groups * 4) + 4 * (1 + 2 * macro)
+    return {"metric": "activation encode+decode GB/s", "value": value, "unit": "GB/s", "n_gpus": world, "steps": steps,
+            "warmup": warmup, "ms_per_step": elapsed / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": label, "topology": f"pipeline: {world // 2} boundaries, sender and receiver of each on two GPUs, "
+                       "message over torch.distributed send/recv", "sequences_per_step": macro, "wire_bytes_per_step": wire,
+                       "timing": "host clock between barriers, median of 30 windows, slowest rank"},
+            "gpu_launches": 30 * steps}
+
+
+def micro_batch_calls(aq, torch, stream, snd, rcv, cfg, step_source, first_step, macro, packed, scales, out, bpe, steps=24):
+    """Sustained throughput of calls the size of the workload's own micro-batch (1 or 8 sequences): the
+    micro-batches of `steps` macro-batches, each encoded then decoded, enqueued back to back -- once call by
+    call through the binding on the plain stream, once as CUDA graphs of one macro-batch each."""
+    nb = cfg.n_batch
+    for h in (snd, rcv):
+        aq.aq_configure(h, aq.AQ_BATCH, nb)
+    per_step = macro // nb
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def one_step(t):
+        arena, ids_dev, s = step_source(t)
+        for l in range(per_step):
+            lo = s * macro + l * nb
+            aq.aq_encode(snd, arena[lo:lo + nb], ids_dev[lo:lo + nb], packed[l * nb:(l + 1) * nb], scales[l * nb:(l + 1) * nb])
+            aq.aq_decode(rcv, packed[l * nb:(l + 1) * nb], scales[l * nb:(l + 1) * nb], ids_dev[lo:lo + nb], out[l * nb:(l + 1) * nb])
+
+    with torch.cuda.stream(stream):
+        one_step(first_step)
+        torch.cuda.synchronize()
+        a, b = ev(), ev()
+        if hasattr(torch.cuda, "_sleep"):
+            torch.cuda._sleep(2_000_000)                  # a millisecond of queued work ahead of the clock
+        a.record(stream)
+        for t in range(steps):
+            one_step(first_step + 1 + t)
+        b.record(stream)
+        torch.cuda.synchronize()
+        ms_stream = a.elapsed_time(b)
+        graphs = []
+        for t in range(steps):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                one_step(first_step + 1 + steps + t)
+            graphs.append(g)
+        graphs[0].replay()
+        torch.cuda.synchronize()
+        a, b = ev(), ev()
+        a.record(stream)
+        for g in graphs:
+            g.replay()
+        b.record(stream)
+        torch.cuda.synchronize()
+        ms_graph = a.elapsed_time(b)
+    calls = steps * per_step                              # encode + decode pairs
+    pair_bytes = 2 * nb * cfg.elems * bpe
+    return {"sequences_per_call": nb, "calls": 2 * calls,
+            "stream": {"us_per_call": ms_stream * 1e3 / (2 * calls), "GB/s": calls * pair_bytes / ms_stream / 1e6},
+            "graph": {"us_per_call": ms_graph * 1e3 / (2 * calls), "GB/s": calls * pair_bytes / ms_graph / 1e6},
+            "note": "encode then decode of every micro-batch, back to back on one stream; us_per_call counts each encode and each decode"}
 
 
 def isolated_calls(aq, torch, stream, snd, rcv, cfg, arena, ids_dev, reps=40):
@@ -727,12 +981,13 @@ def aux_kernels(aq, torch, synth, stream, h, cfg):
     return res
 
 
-def run_e2e(aq, torch, cfg, snd, rcv, arena, ids_dev, steps, dist):
+def run_e2e(aq, torch, cfg, snd, rcv, arena, ids_dev, steps, dist, macro, bpe):
     """The step through the host-buffer calls: activations start in pinned host memory, codes and
     scales cross to pinned host memory and back (the wire), the reconstructed activation ends in
     pinned host memory.  Uses the handles of the device-resident run (every sample already seen),
     so every timed visit is a steady-state delta visit."""
-    nb = MACRO
+    from fixtures import replicas
+    nb = macro
     for h in (snd, rcv):
         aq.aq_configure(h, aq.AQ_BATCH, nb)
     ids = ids_dev.cpu()
@@ -763,7 +1018,6 @@ def run_e2e(aq, torch, cfg, snd, rcv, arena, ids_dev, steps, dist):
     def run_pipelined(k):
         # the sender's calls in this thread, the receiver's in a second one (the calls release the GIL);
         # a wire buffer goes back to the sender when the receiver has read it
-        import threading
         ready = [threading.Semaphore(0) for _ in range(2)]
         free = [threading.Semaphore(1) for _ in range(2)]
         failed = []
@@ -801,20 +1055,126 @@ def run_e2e(aq, torch, cfg, snd, rcv, arena, ids_dev, steps, dist):
 
     dt_serial = timed(run_serial)
     dt = timed(run_pipelined)
-    from fixtures import replicas
     dt = replicas.max_over_ranks(dt, dist, "cuda")
     assert aq.aq_status(snd) == 0 and aq.aq_status(rcv) == 0
     assert aq.aq_state_checksum(snd) == aq.aq_state_checksum(rcv)
     world = dist.get_world_size() if dist else 1
     act_b = nb * cfg.elems * 2
     wire_b = nb * (cfg.packed_bytes + cfg.groups * 4)
-    step_bytes = 2 * nb * cfg.elems * bytes_per_element(cfg.bits, cfg.group)
+    step_bytes = 2 * nb * cfg.elems * bpe
     return {"value": world * steps * step_bytes / dt / 1e9, "unit": "GB/s", "ms_per_step": dt / steps * 1e3,
             "h2d_bytes_per_step": act_b + wire_b + 2 * nb * 4, "d2h_bytes_per_step": wire_b + act_b,
             "steps": steps, "serial_ms_per_step": dt_serial / steps * 1e3,
             "note": "aq_encode_host + aq_decode_host on pinned host buffers, host clock; the receiver's calls run in a "
                     "second host thread and stream beside the sender's, two wire buffers between them "
                     "(serial_ms_per_step: the two calls one after the other)"}
+
+
+def main():
+    args = parse_args()
+    if args.kernel_hash:
+        print(kernel_source_hash())
+        return
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        if rank == 0:
+            from fixtures import synth
+            cfg = getattr(synth, WORKLOADS[args.workload][0])
+            if args.n_samples:
+                cfg = synth.shrink(cfg, args.n_samples)
+            run_reference(args, cfg)
+        return
+
+    import torch
+    import paper_2206_01299_b200 as aq
+    aq.lib()                                         # fails loudly when the CUDA library is missing
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device; there is no CPU path"
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if args.prefetch and not args.hosted:
+        raise SystemExit("--prefetch needs --hosted")
+    if args.hosted and args.m_bits == 32:
+        raise SystemExit("the binary32 store is not offered in host memory")
+    env = Env(rank, local_rank, world, dist, torch.cuda.Stream())
+
+    if args.topology == "pipeline":
+        line = measure_pipeline(args, env)
+        dist.destroy_process_group()
+        if rank == 0:
+            print(json.dumps(line))
+        return
+
+    head = measure_boundary(args, env, args.workload, args.steps, args.warmup, headline=True)
+    plain = (args.rounding == "interval" and not args.m_bits and not args.hosted and not args.per_launch and not args.graph
+             and not args.n_samples)
+    others = {}
+    which = args.configs or ("all" if world == 1 and plain else "headline")
+    if which == "all" and world == 1:
+        for name in WORKLOADS:
+            if name != args.workload:
+                r = measure_boundary(args, env, name, args.steps, args.warmup, headline=False)
+                r.pop("cfg")
+                others[name] = r
+    if dist:
+        dist.destroy_process_group()
+    if rank != 0:
+        return
+
+    cfg = head.pop("cfg")
+    sh = head["shape"]
+    traffic = None
+    rec = NCU_TRAFFIC.get(args.workload)
+    if rec and plain and rec["kernel_hash"] == kernel_source_hash():
+        traffic = rec["encode_bytes_per_element"] * sh["sequences_per_launch"] * cfg.elems
+    m_state = cfg.n_samples * (cfg.elems * 2 if not args.m_bits else cfg.elems * args.m_bits // 8 + (0 if args.m_bits == 32 else cfg.groups * 4))
+    line = {
+        "metric": "activation encode+decode GB/s", "value": head["value"], "unit": "GB/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": head["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": head["workload"], "hidden": cfg.hidden, "seq": cfg.seq,
+                   "micro_batch": cfg.n_batch, "sequences_per_step": sh["sequences_per_step"],
+                   "sequences_per_launch": sh["sequences_per_launch"],
+                   "launch_shape": (f"one aq_encode / aq_decode call per {sh['sequences_per_launch']} sequences (the macro-batch of "
+                                    f"{sh['sequences_per_step']} micro-batches of {cfg.n_batch}); calls of one micro-batch are under micro_batch_calls"),
+                   "cuda_graph": bool(args.graph), "rounding": args.rounding, "m_bits": args.m_bits or 16,
+                   "m_in": ("host memory (page-locked), staged through HBM by aq_prefetch, written back on a copy stream; step time by the host clock" if args.prefetch
+                            else "host memory (page-locked, mapped)" if args.hosted else "HBM"),
+                   "act_dtype": cfg.dtype, "bits": cfg.bits, "group": cfg.group, "n_samples_per_side": cfg.n_samples,
+                   "m_bytes_per_side": m_state, "steady_epochs_resident": sh["steady_epochs_resident"],
+                   "l2": f"inputs larger than L2 (each step touches {int(sh['sequences_per_step'] * cfg.elems * 6 / 1e6)} MB of fresh HBM; no flush needed)",
+                   "parallelism": f"dp{world} replicas, no collective"},
+        "timed": head["timed"],
+        "samples_per_s": head["samples_per_s"],
+        "frac_of_measured_hbm": head["frac_of_measured_hbm"], "frac_of_8000_spec": head["frac_of_8000_spec"],
+        "roofline": {"bound": "hbm", "kernel": "encode_kernel", "achieved": head["encode"]["achieved"], "peak": head["peak"], "unit": "GB/s",
+                     "frac": head["encode"]["frac"], "peak_kind": head["peak_kind"],
+                     "traffic": traffic, "traffic_from": (rec or {}).get("capture"),
+                     "algorithmic_bytes_per_launch": head["launch_bytes"], "avg_launch_ms": head["encode"]["avg_launch_ms"],
+                     "timing": head["kernel_timing"],
+                     "decode_kernel": head["decode"]},
+        "first_visit_epoch": head["first_visit_epoch"],
+        "micro_batch_calls": head["micro_batch_calls"],
+        "e2e": head.get("e2e"), "cpu_baseline": head.get("cpu_baseline"),
+        "gpu_launches": args.steps * head["gpu_launches_per_step"] * head["timed"]["windows"],
+        "clocks": head["clocks"],
+    }
+    for k in ("quant_grad", "dequant_grad", "staged_encode_plus_decode_us", "stage_compute_ms_per_step", "isolated_call", "aux"):
+        if k in head:
+            line[k] = head[k]
+    if others:
+        line["configs"] = others
+    if "aux" in head:
+        line.setdefault("configs", {})["backward"] = {
+            "workload": "Backward path (configs[3]): 4 x 1024 x 1600 fp16 gradients per call, 8 and 4 bit, group 64; _x16 = 16 such micro-batches in one call",
+            **{k: v for k, v in head["aux"].items() if k != "state_checksum"}}
+    print(json.dumps(line))
 
 
 if __name__ == "__main__":

@@ -87,11 +87,14 @@ enum {
                             or step number; for gradients any number unique to the call); default 0 */
   AQ_ROWS_PER_CTA = 6,   /* tuning: rows (256 chunks = 2048 elements each) that one CTA of aq_encode /
                             aq_decode walks; 0 (default) = chosen from the size of the call (2..4) */
-  AQ_L2_PREFETCH = 10    /* tuning: 1 (default for stores in device memory) = every CTA of aq_encode /
-                            aq_decode asks for its rows of act and m to be brought into L2 before it
-                            loads them (one bulk-prefetch instruction, results unchanged); act must then
-                            be in device memory.  0 = plain loads only (default for hosted stores, whose
-                            staged calls use the value set here) */
+  AQ_L2_PREFETCH = 10,   /* tuning: 1 (default for stores in device memory) = every CTA of aq_encode /
+                            aq_decode asks for its rows of act and m, and every CTA of aq_quant_grad for its
+                            piece of the gradient, to be brought into L2 ahead of its loads (bulk-prefetch
+                            instructions, issued while the previous kernel of the stream drains; results
+                            unchanged); act and grad must then be in device memory.  0 = plain loads only
+                            (default for m of hosted stores, whose staged calls use the value set here) */
+  AQ_RAW_LIST = 11       /* device pointer to an array of n_batch device pointers, or 0: the raw messages
+                            of aq_decode_list, one per sample; a null entry = no raw message for that sample */
 };
 enum { AQ_FP16 = 0, AQ_BF16 = 1 };
 /*
@@ -114,15 +117,21 @@ enum {
   AQ_ST_BAD_ID = 1,      /* a sample id was < 0 or >= n_samples */
   AQ_ST_DUP_ID = 2,      /* an id appeared twice in one call; every occurrence after the first is skipped */
   AQ_ST_NO_RAW = 4,      /* aq_decode met a first-visit sample while AQ_RAW was 0 */
-  AQ_ST_STAGED = 8       /* a call after aq_prefetch brought another id at some position than the one
+  AQ_ST_STAGED = 8,      /* a call after aq_prefetch brought another id at some position than the one
                             prefetched for it; that sample is skipped */
+  AQ_ST_BAD_PTR = 16     /* a list-form call found a null or misaligned pointer in one of its arrays; nothing
+                            is read or written for that sample */
 };
 
 /*
  * Initialisation step of Algorithm 1: allocates m (n_samples*seq*hidden*2 bytes of device
  * memory on the current device) filled with zeros, and an empty "seen before"
- * set.  bits in 1..8 is b of the forward quantizer; group in {8,16,32,64,128,256}
- * must divide hidden.  Returns NULL on failure; aq_last_error(NULL) says why.
+ * set.  bits in 1..8 is b of the forward quantizer; group (a multiple of 8, so that a group
+ * is a whole number of 16-byte pieces and group*bits/8 whole bytes) must divide hidden.  Kernels
+ * exist for groups of 8, 16, 32, 64, 128 and 256 elements -- the lanes that share a group's
+ * maximum are a power of two inside one warp; any other multiple of 8 (24, 40, 48, 96 ...) is a
+ * valid setting of the quantizer that this build refuses with AQ_EUNSUPPORTED.  Returns NULL on
+ * failure; aq_last_error(NULL) and aq_last_error_code(NULL) say why.
  */
 aq_handle* aq_create(int64_t n_samples, int seq, int hidden, int bits, int group);
 
@@ -221,6 +230,24 @@ int aq_encode(aq_handle* h, const void* act, const int32_t* sample_ids, void* pa
 int aq_decode(aq_handle* h, const void* packed, const float* scales, const int32_t* sample_ids, void* out);
 
 /*
+ * List forms of the two calls, for a stage that produces its micro-batches one at a time (GPipe-style
+ * pipeline parallelism, Section 2: the micro-batches of a macro-batch cross the boundary one by one) and
+ * wants several of them, each in a buffer of its own, to go through one launch: instead of one base
+ * pointer per buffer the call takes DEVICE arrays of n_batch device pointers, entry y naming the buffer
+ * of sample y -- act_list[y] T[seq][hidden], packed_list[y] uint8[seq*hidden*bits/8], scales_list[y]
+ * float[seq*hidden/group], out_list[y] T[seq][hidden]; the raw messages of first visits come from
+ * AQ_RAW_LIST.  Every pointer must be 16-byte aligned; the kernels check (the host cannot see the
+ * arrays): a null or misaligned entry skips that sample altogether and sets AQ_ST_BAD_PTR.  Same
+ * kernels, same results as the base-pointer forms on the same samples.  The arrays are read when the
+ * kernel runs and must stay unchanged until then.  16-bit stores only (aq_create, aq_create_hosted);
+ * AQ_EUNSUPPORTED otherwise.
+ */
+int aq_encode_list(aq_handle* h, const void* const* act_list, const int32_t* sample_ids,
+                   void* const* packed_list, float* const* scales_list);
+int aq_decode_list(aq_handle* h, const void* const* packed_list, const float* const* scales_list,
+                   const int32_t* sample_ids, void* const* out_list);
+
+/*
  * Backward direction (Algorithm 1, the message from machine b back to machine a: the quantized
  * gradient with respect to the activation): the same Q applied directly to the gradient; touches no state.  n_elems must be a
  * multiple of the handle's group; bits in 1..8 may differ from the handle's forward b.
@@ -243,22 +270,28 @@ int aq_dequant_grad(aq_handle* h, const void* packed, const float* scales, int64
 int aq_state_checksum(aq_handle* h, uint64_t* out_host);
 
 /*
- * The same digest as aq_state_checksum, for callers that must not allocate device memory
- * when they call: code inside a CUDA-graph capture, a step loop that cannot afford the
- * device-wide synchronisation an allocation may bring, a process whose memory was all handed
- * out at start-up.  (The paper has no counterpart; this entry point exists for such callers
+ * The same digest as aq_state_checksum, for callers that cannot allocate device memory at the
+ * time of the call: a process whose device memory was all handed out at start-up (a framework's
+ * caching pool owns it and cudaMalloc would fail or evict), a step loop that must not take the
+ * device-wide synchronisation that cudaMalloc / cudaFree can bring, a service with a fixed memory
+ * budget per library.  (The paper has no counterpart; this entry point exists for such callers
  * only.)  Its working memory is a fixed array inside the library image -- 512 KiB of device
  * memory that every GPU which loads the library holds until the process exits -- so the call
- * itself runs no cudaMalloc, cudaFree or other allocating routine.
+ * itself runs no cudaMalloc, cudaFree or other allocating routine, and uses none of the handle's
+ * own scratch.
  *   - Limit: m of at most 64 GiB (65536 slabs of 1 MiB, one partial sum each); a larger
- *     state is refused with AQ_EUNSUPPORTED and a message, nothing is launched.
- *   - The first call on each device looks up the array's device address (once per device,
- *     with that device current).  Make that first call outside any stream capture.
+ *     state is refused with AQ_EUNSUPPORTED and a message, nothing is launched.  16-bit stores
+ *     only (aq_create, aq_create_hosted); AQ_EUNSUPPORTED for the low-precision and binary32 stores.
+ *   - The first call on each device does the set-up: it looks up the array's device address
+ *     (once per device, with that device current) and keeps it.  Make that first call before any
+ *     stream capture begins.  A cudaDeviceReset invalidates the address that was kept; do not
+ *     call again after one.
  *   - Every call, on any handle, uses the same array and leaves its partial sums there; each
  *     call rewrites every slot it reads, so nothing has to be cleared.  Calls that overlap
  *     on one GPU (different streams, different threads) race on the array and return
  *     garbage: keep them ordered.
- * Synchronises the handle's stream; *out_host is host memory.
+ * Like aq_state_checksum it queues its kernels on the handle's stream, copies the 8-byte result
+ * to the host and synchronises that stream before it returns; *out_host is host memory.
  */
 int aq_state_checksum_noalloc(aq_handle* h, uint64_t* out_host);
 
@@ -268,6 +301,10 @@ int aq_status(aq_handle* h, uint32_t* bits_host);
 /* Message of the last failed call on this handle; with h == NULL, of the last failed
  * aq_create on this thread.  Never NULL.  The string is owned by the library. */
 const char* aq_last_error(aq_handle* h);
+/* The AQ_E* code that goes with that message (the aq_create family returns NULL, not a code):
+ * AQ_EINVAL for arguments that no quantizer setting can have, AQ_EUNSUPPORTED for a valid setting
+ * without a kernel, AQ_ENOMEM / AQ_ECUDA for the allocation. */
+int aq_last_error_code(aq_handle* h);
 
 /* Bytes of `packed` and floats of `scales` per sample for this handle's forward settings. */
 int64_t aq_packed_bytes_per_sample(aq_handle* h);
@@ -305,6 +342,16 @@ int aq_decode_host(aq_handle* h, const void* packed_host, const float* scales_ho
  */
 int aq_wire_copy(aq_handle* h, int dst_device, void* packed_dst, float* scales_dst, void* raw_dst,
                  const void* packed_src, const float* scales_src, const void* raw_src);
+
+/*
+ * The same wire in the backward direction (Algorithm 2: the receiving stage sends the quantized
+ * gradient of the activation back to the sending stage): copies what aq_quant_grad produced for
+ * n_elems elements at `bits` bits -- n_elems*bits/8 bytes of codes and n_elems/group steps -- to
+ * buffers on dst_device, on the handle's stream.  Same rules as aq_wire_copy.  With both ends on
+ * the handle's own device either call is a single kernel launch.
+ */
+int aq_wire_copy_grad(aq_handle* h, int dst_device, void* packed_dst, float* scales_dst,
+                      const void* packed_src, const float* scales_src, int64_t n_elems, int bits);
 
 /*
  * State access for checkpoints and tests.  Copies one sample's m block

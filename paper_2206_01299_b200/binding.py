@@ -14,10 +14,11 @@ LIB_PATH = os.path.join(HERE, "libaq_b200.so")
 AQ_OK, AQ_EINVAL, AQ_ENOMEM, AQ_ECUDA, AQ_EUNSUPPORTED = 0, -1, -2, -3, -4
 AQ_DTYPE, AQ_BATCH, AQ_STREAM, AQ_RAW, AQ_FIRST_FLAGS, AQ_ROWS_PER_CTA = 1, 2, 3, 4, 5, 6
 AQ_L2_PREFETCH = 10
+AQ_RAW_LIST = 11
 AQ_ROUNDING, AQ_SEED, AQ_EPOCH = 7, 8, 9
 AQ_FP16, AQ_BF16 = 0, 1
 AQ_ROUND_INTERVAL, AQ_ROUND_STOCHASTIC = 0, 1
-AQ_ST_BAD_ID, AQ_ST_DUP_ID, AQ_ST_NO_RAW, AQ_ST_STAGED = 1, 2, 4, 8
+AQ_ST_BAD_ID, AQ_ST_DUP_ID, AQ_ST_NO_RAW, AQ_ST_STAGED, AQ_ST_BAD_PTR = 1, 2, 4, 8, 16
 
 # name -> (restype, argtypes); the load test checks these against the header
 SIGNATURES = {
@@ -30,12 +31,15 @@ SIGNATURES = {
     "aq_configure": (C.c_int, [C.c_void_p, C.c_int, C.c_int64]),
     "aq_encode": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "aq_decode": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "aq_encode_list": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "aq_decode_list": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "aq_quant_grad": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_void_p, C.c_void_p]),
     "aq_dequant_grad": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_void_p]),
     "aq_state_checksum": (C.c_int, [C.c_void_p, C.POINTER(C.c_uint64)]),
     "aq_state_checksum_noalloc": (C.c_int, [C.c_void_p, C.POINTER(C.c_uint64)]),
     "aq_status": (C.c_int, [C.c_void_p, C.POINTER(C.c_uint32)]),
     "aq_last_error": (C.c_char_p, [C.c_void_p]),
+    "aq_last_error_code": (C.c_int, [C.c_void_p]),
     "aq_packed_bytes_per_sample": (C.c_int64, [C.c_void_p]),
     "aq_scales_per_sample": (C.c_int64, [C.c_void_p]),
     "aq_m_bytes_per_sample": (C.c_int64, [C.c_void_p]),
@@ -43,6 +47,7 @@ SIGNATURES = {
     "aq_decode_host": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "aq_wire_copy": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                C.c_void_p]),
+    "aq_wire_copy_grad": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int]),
     "aq_prefetch": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int]),
     "aq_export_sample": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]),
     "aq_import_sample": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p, C.c_uint8]),
@@ -92,39 +97,30 @@ def _check(h, rc):
     return rc
 
 
-def aq_create(n_samples, seq, hidden, bits, group):
-    h = lib().aq_create(n_samples, seq, hidden, bits, group)
+def _created(h):
     if not h:
-        raise AqError(AQ_EINVAL, aq_last_error(None))
+        raise AqError(aq_last_error_code(None), aq_last_error(None))
     return h
+
+
+def aq_create(n_samples, seq, hidden, bits, group):
+    return _created(lib().aq_create(n_samples, seq, hidden, bits, group))
 
 
 def aq_create_hosted(n_samples, seq, hidden, bits, group):
-    h = lib().aq_create_hosted(n_samples, seq, hidden, bits, group)
-    if not h:
-        raise AqError(AQ_EINVAL, aq_last_error(None))
-    return h
+    return _created(lib().aq_create_hosted(n_samples, seq, hidden, bits, group))
 
 
 def aq_create_fp32(n_samples, seq, hidden, bits, group):
-    h = lib().aq_create_fp32(n_samples, seq, hidden, bits, group)
-    if not h:
-        raise AqError(AQ_EINVAL, aq_last_error(None))
-    return h
+    return _created(lib().aq_create_fp32(n_samples, seq, hidden, bits, group))
 
 
 def aq_create_lowbit(n_samples, seq, hidden, bits, group, m_bits):
-    h = lib().aq_create_lowbit(n_samples, seq, hidden, bits, group, m_bits)
-    if not h:
-        raise AqError(AQ_EINVAL, aq_last_error(None))
-    return h
+    return _created(lib().aq_create_lowbit(n_samples, seq, hidden, bits, group, m_bits))
 
 
 def aq_create_hosted_lowbit(n_samples, seq, hidden, bits, group, m_bits):
-    h = lib().aq_create_hosted_lowbit(n_samples, seq, hidden, bits, group, m_bits)
-    if not h:
-        raise AqError(AQ_EINVAL, aq_last_error(None))
-    return h
+    return _created(lib().aq_create_hosted_lowbit(n_samples, seq, hidden, bits, group, m_bits))
 
 
 def aq_destroy(h):
@@ -143,6 +139,15 @@ def aq_encode(h, act, sample_ids, packed, scales):
 
 def aq_decode(h, packed, scales, sample_ids, out):
     return _check(h, lib().aq_decode(h, _ptr(packed), _ptr(scales), _ptr(sample_ids), _ptr(out)))
+
+
+def aq_encode_list(h, act_list, sample_ids, packed_list, scales_list):
+    """The *_list arguments are int64 device tensors holding one device address per sample."""
+    return _check(h, lib().aq_encode_list(h, _ptr(act_list), _ptr(sample_ids), _ptr(packed_list), _ptr(scales_list)))
+
+
+def aq_decode_list(h, packed_list, scales_list, sample_ids, out_list):
+    return _check(h, lib().aq_decode_list(h, _ptr(packed_list), _ptr(scales_list), _ptr(sample_ids), _ptr(out_list)))
 
 
 def aq_quant_grad(h, grad, n_elems, bits, packed, scales):
@@ -176,6 +181,10 @@ def aq_last_error(h):
     return lib().aq_last_error(h).decode()
 
 
+def aq_last_error_code(h):
+    return lib().aq_last_error_code(h)
+
+
 def aq_packed_bytes_per_sample(h):
     return lib().aq_packed_bytes_per_sample(h)
 
@@ -201,6 +210,11 @@ def aq_decode_host(h, packed_host, scales_host, raw_host, sample_ids_host, out_h
 def aq_wire_copy(h, dst_device, packed_dst, scales_dst, raw_dst, packed_src, scales_src, raw_src):
     return _check(h, lib().aq_wire_copy(h, dst_device, _ptr(packed_dst), _ptr(scales_dst), _ptr(raw_dst),
                                         _ptr(packed_src), _ptr(scales_src), _ptr(raw_src)))
+
+
+def aq_wire_copy_grad(h, dst_device, packed_dst, scales_dst, packed_src, scales_src, n_elems, bits):
+    return _check(h, lib().aq_wire_copy_grad(h, dst_device, _ptr(packed_dst), _ptr(scales_dst), _ptr(packed_src),
+                                             _ptr(scales_src), n_elems, bits))
 
 
 def aq_prefetch(h, sample_ids_host):

@@ -22,6 +22,7 @@ struct aq_handle {
   int device = 0;
   cudaStream_t stream = nullptr;
   const void* raw = nullptr;
+  const void* const* raw_list = nullptr;     // AQ_RAW_LIST: the raw messages of a list-form decode
   uint8_t* first_flags = nullptr;
   unsigned long long* sum_dev = nullptr;     // scratch of aq_state_checksum
   void* m_host = nullptr;                    // hosted store: the pinned host block that st.m maps
@@ -60,14 +61,17 @@ struct aq_handle {
   cudaStream_t in_stream = nullptr, out_stream = nullptr;
   cudaEvent_t ev_begin = nullptr, ev_in[kSlices] = {}, ev_done[kSlices] = {};
   char err[256] = {0};
+  int err_code = AQ_OK;                      // code of the call that wrote err
 };
 
 namespace {
 
 thread_local char g_create_err[256] = "";
+thread_local int g_create_code = AQ_OK;
 
 int fail(aq_handle* h, int code, const char* fmt, ...) {
   char* dst = h ? h->err : g_create_err;
+  (h ? h->err_code : g_create_code) = code;
   va_list ap;
   va_start(ap, fmt);
   vsnprintf(dst, 256, fmt, ap);
@@ -246,13 +250,20 @@ aq_handle* aq_create_lowbit(int64_t n_samples, int seq, int hidden, int bits, in
 static aq_handle* create_handle(int64_t n_samples, int seq, int hidden, int bits, int group, int m_bits,
                                 bool hosted) {
   g_create_err[0] = 0;
+  g_create_code = AQ_OK;
   const int lanes = lanes_for_group(group);
   if (n_samples <= 0 || seq <= 0 || hidden <= 0) { fail(nullptr, AQ_EINVAL, "n_samples, seq and hidden must be positive"); return nullptr; }
   if (n_samples > 0x7fffffffll) { fail(nullptr, AQ_EINVAL, "n_samples must fit the int32 sample ids"); return nullptr; }
   if ((long long)seq * hidden > (1ll << 30)) { fail(nullptr, AQ_EINVAL, "seq*hidden must not exceed 2^30 elements per sample"); return nullptr; }
   if (bits < 1 || bits > 8) { fail(nullptr, AQ_EINVAL, "bits must be in 1..8 (got %d)", bits); return nullptr; }
-  if (!lanes) { fail(nullptr, AQ_EINVAL, "group must be one of 8,16,32,64,128,256 (got %d)", group); return nullptr; }
+  if (group <= 0 || group % 8) { fail(nullptr, AQ_EINVAL, "group must be a positive multiple of 8 (got %d)", group); return nullptr; }
   if (hidden % group) { fail(nullptr, AQ_EINVAL, "group %d does not divide hidden %d", group, hidden); return nullptr; }
+  if (!lanes) {
+    // a valid quantizer setting that no kernel is built for: the lanes that share a group's maximum must be
+    // a power of two within one warp
+    fail(nullptr, AQ_EUNSUPPORTED, "group %d: this build has kernels for groups of 8, 16, 32, 64, 128 and 256 elements only", group);
+    return nullptr;
+  }
   aq_handle* h = new (std::nothrow) aq_handle();
   if (!h) { fail(nullptr, AQ_ENOMEM, "host allocation failed"); return nullptr; }
   h->seq = seq; h->hidden = hidden; h->bits = bits; h->group = group;
@@ -363,6 +374,9 @@ int aq_configure(aq_handle* h, int key, int64_t value) {
       if (value & 15) return fail(h, AQ_EINVAL, "AQ_RAW pointer must be 16-byte aligned");
       h->raw = reinterpret_cast<const void*>(static_cast<intptr_t>(value));
       return AQ_OK;
+    case AQ_RAW_LIST:
+      h->raw_list = reinterpret_cast<const void* const*>(static_cast<intptr_t>(value));
+      return AQ_OK;
     case AQ_FIRST_FLAGS:
       h->first_flags = reinterpret_cast<uint8_t*>(static_cast<intptr_t>(value));
       return AQ_OK;
@@ -411,15 +425,17 @@ static int launch_decode_call(aq_handle* h, const aq::DecodeArgs& a) {
   return AQ_OK;
 }
 
-int aq_encode(aq_handle* h, const void* act, const int32_t* sample_ids, void* packed, float* scales) {
+static int encode_call(aq_handle* h, const void* act, const int32_t* sample_ids, void* packed, float* scales, bool lists,
+                       const char* who) {
   if (!h) return fail(nullptr, AQ_EINVAL, "null handle");
   if (h->n_batch == 0) return AQ_OK;
-  if (!act || !sample_ids || !packed || !scales) return fail(h, AQ_EINVAL, "aq_encode: null pointer");
-  if (!aligned16(act) || !aligned16(packed) || !aligned16(scales))
-    return fail(h, AQ_EINVAL, "aq_encode: act, packed and scales must be 16-byte aligned");
+  if (!act || !sample_ids || !packed || !scales) return fail(h, AQ_EINVAL, "%s: null pointer", who);
+  if (!lists && (!aligned16(act) || !aligned16(packed) || !aligned16(scales)))
+    return fail(h, AQ_EINVAL, "%s: act, packed and scales must be 16-byte aligned", who);
+  if (lists && h->st.m_bits) return fail(h, AQ_EUNSUPPORTED, "%s: the list form is built for the 16-bit store only", who);
   DeviceGuard g(h->device);
   aq::EncodeArgs a{act, sample_ids, static_cast<uint8_t*>(packed), scales, h->first_flags, h->n_batch,
-                   h->rounding == AQ_ROUND_STOCHASTIC, h->seed, h->epoch};
+                   h->rounding == AQ_ROUND_STOCHASTIC, h->seed, h->epoch, lists};
   if (h->prefetch_pending)
     return run_staged(h, [&](const aq::State& st) {
       return h->st.m_bits ? aq::launch_encode_lowbit(h->dtype, h->bits, st, a, h->stream)
@@ -428,20 +444,43 @@ int aq_encode(aq_handle* h, const void* act, const int32_t* sample_ids, void* pa
   return launch_encode_call(h, a);
 }
 
-int aq_decode(aq_handle* h, const void* packed, const float* scales, const int32_t* sample_ids, void* out) {
+int aq_encode(aq_handle* h, const void* act, const int32_t* sample_ids, void* packed, float* scales) {
+  return encode_call(h, act, sample_ids, packed, scales, false, "aq_encode");
+}
+
+int aq_encode_list(aq_handle* h, const void* const* act_list, const int32_t* sample_ids, void* const* packed_list,
+                   float* const* scales_list) {
+  return encode_call(h, act_list, sample_ids, const_cast<void**>(packed_list),
+                     reinterpret_cast<float*>(const_cast<float**>(scales_list)), true, "aq_encode_list");
+}
+
+static int decode_call(aq_handle* h, const void* packed, const float* scales, const int32_t* sample_ids, void* out, bool lists,
+                       const char* who) {
   if (!h) return fail(nullptr, AQ_EINVAL, "null handle");
   if (h->n_batch == 0) return AQ_OK;
-  if (!packed || !scales || !sample_ids || !out) return fail(h, AQ_EINVAL, "aq_decode: null pointer");
-  if (!aligned16(packed) || !aligned16(scales) || !aligned16(out))
-    return fail(h, AQ_EINVAL, "aq_decode: packed, scales and out must be 16-byte aligned");
+  if (!packed || !scales || !sample_ids || !out) return fail(h, AQ_EINVAL, "%s: null pointer", who);
+  if (!lists && (!aligned16(packed) || !aligned16(scales) || !aligned16(out)))
+    return fail(h, AQ_EINVAL, "%s: packed, scales and out must be 16-byte aligned", who);
+  if (lists && h->st.m_bits) return fail(h, AQ_EUNSUPPORTED, "%s: the list form is built for the 16-bit store only", who);
   DeviceGuard g(h->device);
-  aq::DecodeArgs a{static_cast<const uint8_t*>(packed), scales, h->raw, sample_ids, out, h->first_flags, h->n_batch};
+  aq::DecodeArgs a{static_cast<const uint8_t*>(packed), scales, lists ? static_cast<const void*>(h->raw_list) : h->raw, sample_ids,
+                   out, h->first_flags, h->n_batch, lists};
   if (h->prefetch_pending)
     return run_staged(h, [&](const aq::State& st) {
       return h->st.m_bits ? aq::launch_decode_lowbit(h->dtype, h->bits, st, a, h->stream)
                           : aq::launch_decode(h->dtype, h->bits, st, a, h->stream);
     });
   return launch_decode_call(h, a);
+}
+
+int aq_decode(aq_handle* h, const void* packed, const float* scales, const int32_t* sample_ids, void* out) {
+  return decode_call(h, packed, scales, sample_ids, out, false, "aq_decode");
+}
+
+int aq_decode_list(aq_handle* h, const void* const* packed_list, const float* const* scales_list, const int32_t* sample_ids,
+                   void* const* out_list) {
+  return decode_call(h, packed_list, reinterpret_cast<const float*>(scales_list), sample_ids, const_cast<void**>(out_list), true,
+                     "aq_decode_list");
 }
 
 static int check_grad_args(aq_handle* h, const void* a, const void* b, const void* c, int64_t n_elems, int bits) {
@@ -462,7 +501,8 @@ int aq_quant_grad(aq_handle* h, const void* grad, int64_t n_elems, int bits, voi
   if (stochastic && n_elems / aq::kChunk > 0xFFFFFFFFll)
     return fail(h, AQ_EINVAL, "aq_quant_grad: stochastic rounding numbers chunks with 32 bits (n_elems < 2^35)");
   AQ_CUDA(h, aq::launch_quant_grad(h->dtype, bits, h->st.lanes_per_group, grad, n_elems,
-                                   static_cast<uint8_t*>(packed), scales, stochastic, h->seed, h->epoch, h->stream));
+                                   static_cast<uint8_t*>(packed), scales, stochastic, h->seed, h->epoch, h->l2_prefetch,
+                                   h->stream));
   return AQ_OK;
 }
 
@@ -502,6 +542,7 @@ int aq_status(aq_handle* h, uint32_t* bits_host) {
 }
 
 const char* aq_last_error(aq_handle* h) { return h ? h->err : g_create_err; }
+int aq_last_error_code(aq_handle* h) { return h ? h->err_code : g_create_code; }
 
 int64_t aq_packed_bytes_per_sample(aq_handle* h) { return h ? h->st.packed_bytes : 0; }
 int64_t aq_scales_per_sample(aq_handle* h) { return h ? h->st.groups : 0; }
@@ -669,6 +710,22 @@ int aq_prefetch(aq_handle* h, const int32_t* sample_ids_host, int n) {
   return AQ_OK;
 }
 
+// The byte ranges of a message from the handle's device to dst_device, on the handle's stream: one
+// kernel launch when both ends are on the handle's device and every range is made of whole,
+// aligned 16-byte pieces; otherwise one copy per range (peer copies into the receiver's memory).
+static int wire_ranges(aq_handle* h, int dst_device, const void* const* src, void* const* dst, const size_t* bytes, int n) {
+  bool by_kernel = dst_device == h->device;
+  for (int k = 0; k < n; ++k)
+    by_kernel = by_kernel && bytes[k] % 16 == 0 && aligned16(src[k]) && aligned16(dst[k]);
+  if (by_kernel) {
+    AQ_CUDA(h, aq::launch_wire_copy(src, dst, bytes, n, h->stream));
+    return AQ_OK;
+  }
+  for (int k = 0; k < n; ++k)
+    AQ_CUDA(h, cudaMemcpyPeerAsync(dst[k], dst_device, src[k], h->device, bytes[k], h->stream));
+  return AQ_OK;
+}
+
 int aq_wire_copy(aq_handle* h, int dst_device, void* packed_dst, float* scales_dst, void* raw_dst,
                  const void* packed_src, const float* scales_src, const void* raw_src) {
   if (!h) return fail(nullptr, AQ_EINVAL, "null handle");
@@ -680,12 +737,27 @@ int aq_wire_copy(aq_handle* h, int dst_device, void* packed_dst, float* scales_d
   if (dst_device < 0 || dst_device >= n_dev) return fail(h, AQ_EINVAL, "aq_wire_copy: no device %d", dst_device);
   DeviceGuard g(h->device);
   const size_t nb = (size_t)h->n_batch;
-  AQ_CUDA(h, cudaMemcpyPeerAsync(packed_dst, dst_device, packed_src, h->device, nb * (size_t)h->st.packed_bytes, h->stream));
-  AQ_CUDA(h, cudaMemcpyPeerAsync(scales_dst, dst_device, scales_src, h->device,
-                                 nb * (size_t)h->st.groups * sizeof(float), h->stream));
-  if (raw_src)
-    AQ_CUDA(h, cudaMemcpyPeerAsync(raw_dst, dst_device, raw_src, h->device, nb * (size_t)h->st.elems * 2, h->stream));
-  return AQ_OK;
+  const void* src[3] = {packed_src, scales_src, raw_src};
+  void* dst[3] = {packed_dst, scales_dst, raw_dst};
+  const size_t bytes[3] = {nb * (size_t)h->st.packed_bytes, nb * (size_t)h->st.groups * sizeof(float), nb * (size_t)h->st.elems * 2};
+  return wire_ranges(h, dst_device, src, dst, bytes, raw_src ? 3 : 2);
+}
+
+int aq_wire_copy_grad(aq_handle* h, int dst_device, void* packed_dst, float* scales_dst, const void* packed_src,
+                      const float* scales_src, int64_t n_elems, int bits) {
+  if (!h) return fail(nullptr, AQ_EINVAL, "null handle");
+  if (bits < 1 || bits > 8) return fail(h, AQ_EINVAL, "bits must be in 1..8 (got %d)", bits);
+  if (n_elems < 0 || n_elems % h->group) return fail(h, AQ_EINVAL, "n_elems must be a non-negative multiple of group %d", h->group);
+  if (n_elems == 0) return AQ_OK;
+  if (!packed_dst || !scales_dst || !packed_src || !scales_src) return fail(h, AQ_EINVAL, "aq_wire_copy_grad: null pointer");
+  int n_dev = 0;
+  AQ_CUDA(h, cudaGetDeviceCount(&n_dev));
+  if (dst_device < 0 || dst_device >= n_dev) return fail(h, AQ_EINVAL, "aq_wire_copy_grad: no device %d", dst_device);
+  DeviceGuard g(h->device);
+  const void* src[2] = {packed_src, scales_src};
+  void* dst[2] = {packed_dst, scales_dst};
+  const size_t bytes[2] = {(size_t)n_elems * (size_t)bits / 8, (size_t)(n_elems / h->group) * sizeof(float)};
+  return wire_ranges(h, dst_device, src, dst, bytes, 2);
 }
 
 int aq_export_sample(aq_handle* h, int64_t sample_id, void* m_host, uint8_t* seen_host) {

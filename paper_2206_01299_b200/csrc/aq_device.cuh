@@ -17,8 +17,8 @@ constexpr unsigned kFullMask = 0xffffffffu;
 constexpr int kChunksPerThread = 3;                      // grad kernels: chunks per thread (measured: 2, 3, 4)
 constexpr int kChunksPerCta = kThreads * kChunksPerThread;
 
-enum { kModeDelta = 0, kModeFirst = 1, kModeSkip = 2 };
-enum { kStBadId = 1, kStDupId = 2, kStNoRaw = 4, kStStaged = 8 };
+enum { kModeDelta = 0, kModeFirst = 1, kModeSkip = 2, kModeNothing = 3 };   // kModeNothing: not even zeros can be written
+enum { kStBadId = 1, kStDupId = 2, kStNoRaw = 4, kStStaged = 8, kStBadPtr = 16 };
 
 // What the launch layer decides for one encode / decode launch.
 struct LaunchPlan {
@@ -51,6 +51,16 @@ template <> struct Conv<__half> {
     for (int i = 0; i < 4; ++i) h[i] = __floats2half2_rn(f[2 * i], f[2 * i + 1]);
     return v;
   }
+  // d[j] = a_j - m[j]: the mixed-precision subtraction widens a_j exactly and rounds the
+  // difference once, the same number as converting first and subtracting in binary32
+  static __device__ __forceinline__ void diff(const uint4& a, const float (&m)[8], float (&d)[8]) {
+    const uint32_t w[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tsub.rn.f32.f16 %0, lo, %3;\n\tsub.rn.f32.f16 %1, hi, %4;\n\t}"
+          : "=f"(d[2 * i]), "=f"(d[2 * i + 1])
+          : "r"(w[i]), "f"(m[2 * i]), "f"(m[2 * i + 1]));
+  }
 };
 
 template <> struct Conv<__nv_bfloat16> {
@@ -69,6 +79,14 @@ template <> struct Conv<__nv_bfloat16> {
 #pragma unroll
     for (int i = 0; i < 4; ++i) h[i] = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
     return v;
+  }
+  static __device__ __forceinline__ void diff(const uint4& a, const float (&m)[8], float (&d)[8]) {
+    const uint32_t w[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tsub.rn.f32.bf16 %0, lo, %3;\n\tsub.rn.f32.bf16 %1, hi, %4;\n\t}"
+          : "=f"(d[2 * i]), "=f"(d[2 * i + 1])
+          : "r"(w[i]), "f"(m[2 * i]), "f"(m[2 * i + 1]));
   }
 };
 
@@ -179,6 +197,26 @@ __device__ __forceinline__ void quantize8(const float (&d)[8], float s, const ui
   }
 }
 
+// quantize8 for the type at hand.  The wide type (bf16: differences span the whole binary32 exponent
+// range) needs the two guards of quantize8 only when a step is extreme; whenever every lane of the
+// warp has a step in [2^-125, 2^100] (or a dead group) the narrow form computes the same numbers --
+// its reciprocal is normal, so the lower clamp cannot bind, and half the step is exact, so the fused
+// reconstruction rounds the same product once -- and the warp takes it.
+template <int BITS, bool WIDE, bool STOCH>
+__device__ __forceinline__ void quantize8_for(const float (&d)[8], float s, const uint4& noise, float& delta,
+                                              unsigned long long& codes, float (&q)[8]) {
+  if constexpr (!WIDE || STOCH) {
+    quantize8<BITS, WIDE, STOCH>(d, s, noise, delta, codes, q);
+  } else {
+    const float dl = __fmul_rn(s, 1.0f / (float)(1 << (BITS - 1)));
+    const bool tame = !(dl >= FLT_MIN) || (dl >= 0x1p-125f && dl <= 0x1p100f);
+    if (__all_sync(kFullMask, tame))
+      quantize8<BITS, false, false>(d, s, noise, delta, codes, q);
+    else
+      quantize8<BITS, true, false>(d, s, noise, delta, codes, q);
+  }
+}
+
 // Philox4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw, SC 2011): the 128 random bits of one
 // chunk.  key = the seed's two words; counter = { chunk index in the stream, stream id (sample
 // id, or 0xFFFFFFFF for gradients), epoch low word, epoch high word }.  Element j of the chunk
@@ -240,7 +278,24 @@ __device__ __forceinline__ void store_codes(uint8_t* stream, long long chunk, in
   } else {
     constexpr int kBitsPerLane = 8 * BITS;
     constexpr int kWords = 8 * BITS;
-    if (warp_words) {   // uniform over the warp: all 32 lanes active, base word-aligned
+    if (warp_words && BITS == 3) {
+      // four lanes hold 96 bits = three whole words: lane q of the quad builds word q from its own
+      // 24 bits and those of lane q + 1 (one shuffle), the fourth lane stores nothing
+      const uint32_t own = (uint32_t)v;
+      const uint32_t nxt = __shfl_down_sync(kFullMask, own, 1);
+      const int q = lane & 3;
+      const uint32_t word = (own >> (8 * q)) | (nxt << (24 - 8 * q));
+      if (q < 3) reinterpret_cast<uint32_t*>(stream + (chunk >> 2) * 12)[q] = word;
+    } else if (warp_words && BITS == 6) {
+      // two lanes hold 96 bits = three whole words: the even lane stores words 0 and 1 (its own 48
+      // bits and the low 16 of its neighbour's), the odd lane word 2 (its own high 32)
+      const uint32_t lo = (uint32_t)v, hi = (uint32_t)(v >> 32);
+      const uint32_t other = __shfl_xor_sync(kFullMask, lo, 1);
+      const bool odd = lane & 1;
+      uint32_t* w = reinterpret_cast<uint32_t*>(stream + (chunk >> 1) * 12);
+      w[odd ? 2 : 0] = odd ? ((lo >> 16) | (hi << 16)) : lo;
+      if (!odd) w[1] = hi | (other << 16);
+    } else if (warp_words) {   // uniform over the warp: all 32 lanes active, base word-aligned
       uint32_t* wbase = reinterpret_cast<uint32_t*>(stream + (chunk - lane) * BITS);
 #pragma unroll
       for (int r = 0; r < (kWords + 31) / 32; ++r) {
@@ -289,7 +344,20 @@ __device__ __forceinline__ unsigned long long load_codes(const uint8_t* stream, 
     constexpr int kWords = 8 * BITS;
     constexpr int kNeed = (BITS == 7) ? 3 : 2;      // words a lane's field can straddle
     unsigned long long v = 0ull;
-    if (warp_words) {
+    if (warp_words && BITS == 3) {
+      // lane q of a quad owns bits [24q, 24q + 24) of the quad's three words: it reads the two
+      // words that hold them (no exchange between lanes) and shifts its field down
+      const uint32_t* w = reinterpret_cast<const uint32_t*>(stream + (chunk >> 2) * 12);
+      const int q = lane & 3;
+      const uint32_t a = __ldg(w + max(q - 1, 0)), b = __ldg(w + min(q, 2));
+      v = __funnelshift_r(a, b, (24 * q) & 31) & 0xFFFFFFu;
+    } else if (warp_words && BITS == 6) {
+      // the even lane of a pair owns bits [0, 48) of the pair's three words, the odd lane bits [48, 96)
+      const int odd = lane & 1;
+      const uint32_t* w = reinterpret_cast<const uint32_t*>(stream + (chunk >> 1) * 12) + odd;
+      const uint32_t a = __ldg(w), b = __ldg(w + 1);
+      v = ((((unsigned long long)b << 32) | a) >> (16 * odd)) & 0xFFFFFFFFFFFFull;
+    } else if (warp_words) {
       const uint32_t* wbase = reinterpret_cast<const uint32_t*>(stream + (chunk - lane) * BITS);
       const uint32_t w0 = (lane < kWords) ? wbase[lane] : 0u;
       uint32_t w1 = 0u;
@@ -353,12 +421,42 @@ __device__ __forceinline__ void overlap_with_neighbours() {
   asm volatile("griddepcontrol.launch_dependents;");
   asm volatile("griddepcontrol.wait;" ::: "memory");
 }
+// The two halves of the above: between them a CTA may issue hints (prefetches into L2), nothing
+// whose value it keeps -- L2 is the point of coherence, so a line fetched early is updated in
+// place by the writes of the kernel that is still running.
+__device__ __forceinline__ void let_dependents_launch() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void wait_for_predecessor() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// Issued by one thread of the CTA ahead of wait_for_predecessor: asks for the CTA's rows of m(xi)
+// -- chunks [lo, hi) of the sample at position y of the call -- to be brought into L2.  While
+// the CTA is waiting for the previous kernel of the stream to drain, the memory system is not
+// busy; when the wait is over the real loads find the rows in L2.  The id and the stamp are read
+// past L1 (they may not be final yet) and only steer the hint: an id out of range or a sample
+// that looks unseen asks for nothing.
+template <typename T>
+__device__ __forceinline__ void prefetch_rows_of_m(const State& st, const int32_t* ids, int y, int lo, int hi) {
+  if (hi <= lo) return;
+  const int32_t id = __ldcg(ids + y);
+  if (id < 0 || (long long)id >= st.n_samples) return;
+  if (__ldcg(st.seen + id) == 0ull) return;
+  const unsigned long long row = st.slot_ids ? (unsigned long long)(unsigned)y : (unsigned long long)(unsigned)id;
+  const T* m = reinterpret_cast<const T*>(st.m) + row * (unsigned long long)st.elems;
+  prefetch_l2(m + (size_t)lo * kChunk, (unsigned)(hi - lo) * 16u);
+}
 
 // What a CTA knows about its sample after open_sample.
 struct Sample {
   int mode;
   int32_t id;
   unsigned row;   // the sample's row of st.m: its id, or its position in the call when m(xi) was staged
+  const void* buf[4];   // list form of the calls: the sample's own buffers, in the order of BufferLists
+};
+
+// The pointer arrays of a list-form call (null entries of `list`: that buffer is not used by the
+// call); `needed`: a null pointer in the array is an error, not "absent".
+struct BufferLists {
+  const void* const* list[4];
+  bool needed[4];
 };
 
 // Sample y of the call, resolved by warp 0 for the whole CTA (one barrier): its id, whether it
@@ -368,14 +466,31 @@ struct Sample {
 // first row also records the visit: status bit of a skipped sample, first-visit flag, stamp.
 // With staged messages (st.slot_ids set) row y of st.m holds m of sample slot_ids[y]; a call
 // that brings another id to that position skips the sample.
+// List form (lists != null): lane 0 also fetches the sample's buffer pointers; one that is
+// missing or not 16-byte aligned makes the sample kModeNothing (nothing read or written for it).
+// raw_at: which of the lists holds the raw message of a first visit (-1: none); a null entry
+// there means "no raw message for this sample".
 __device__ __forceinline__ Sample open_sample(const State& st, const LaunchPlan& plan,
                                               const int32_t* __restrict__ ids, int y, bool need_raw,
-                                              bool have_raw, uint8_t* first_flags) {
+                                              bool have_raw, uint8_t* first_flags,
+                                              const BufferLists* lists = nullptr, int raw_at = -1) {
   __shared__ Sample s_sample;
   if (threadIdx.x < 32) {
     const int lane = threadIdx.x;
     unsigned long long call = 0ull;
     if (lane == 0) call = take_call_number(st, plan);
+    const void* buf[4] = {nullptr, nullptr, nullptr, nullptr};
+    bool bad_ptr = false;
+    if (lists && lane == 0) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if (lists->list[k]) buf[k] = lists->list[k][y];
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if (lists->list[k])
+          bad_ptr |= (reinterpret_cast<uintptr_t>(buf[k]) & 15u) != 0 || (lists->needed[k] && buf[k] == nullptr);
+      if (raw_at >= 0) have_raw = buf[raw_at] != nullptr;
+    }
     const int32_t id = ids[y];
     const bool in_range = id >= 0 && (long long)id < st.n_samples;
     int dup = 0;
@@ -386,7 +501,10 @@ __device__ __forceinline__ Sample open_sample(const State& st, const LaunchPlan&
     if (lane == 0) {
       int mode;
       unsigned why = 0u;
-      if (!in_range) {
+      if (bad_ptr) {
+        mode = kModeNothing;
+        why = kStBadPtr;
+      } else if (!in_range) {
         mode = kModeSkip;
         why = kStBadId;
       } else if (dup) {
@@ -406,6 +524,8 @@ __device__ __forceinline__ Sample open_sample(const State& st, const LaunchPlan&
       s_sample.mode = mode;
       s_sample.id = id;
       s_sample.row = st.slot_ids ? (unsigned)y : (unsigned)id;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) s_sample.buf[k] = buf[k];
       if (blockIdx.x == 0) {                     // once per sample and call
         if (why) atomicOr(st.status, why);
         if (first_flags) first_flags[y] = (uint8_t)(mode == kModeFirst);

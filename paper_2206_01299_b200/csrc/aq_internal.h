@@ -44,6 +44,8 @@ struct State {
                                   // running call: row y holds m of sample slot_ids[y] (hosted store, prefetched)
 };
 
+// A call names its buffers either by one base pointer each (sample y at base + y * its size) or,
+// when `lists` is set, by device arrays of n_batch pointers, one buffer per sample.
 struct EncodeArgs {
   const void* act;
   const int32_t* ids;
@@ -53,16 +55,25 @@ struct EncodeArgs {
   int n_batch;
   bool stochastic;                  // unbiased stochastic rounding instead of the interval number
   unsigned long long seed, epoch;   // its generator key and the caller's call counter
+  bool lists;                       // act, packed, scales are arrays of pointers (act_list() etc.)
+  __host__ __device__ const void* const* act_list() const { return static_cast<const void* const*>(act); }
+  __host__ __device__ const void* const* packed_list() const { return reinterpret_cast<const void* const*>(packed); }
+  __host__ __device__ const void* const* scales_list() const { return reinterpret_cast<const void* const*>(scales); }
 };
 
 struct DecodeArgs {
   const uint8_t* packed;
   const float* scales;
-  const void* raw;         // may be null
+  const void* raw;         // may be null (as a list: the array itself, or single entries of it)
   const int32_t* ids;
   void* out;
   uint8_t* first_flags;    // may be null
   int n_batch;
+  bool lists;              // packed, scales, raw, out are arrays of pointers
+  __host__ __device__ const void* const* packed_list() const { return reinterpret_cast<const void* const*>(packed); }
+  __host__ __device__ const void* const* scales_list() const { return reinterpret_cast<const void* const*>(scales); }
+  __host__ __device__ const void* const* raw_list() const { return static_cast<const void* const*>(raw); }
+  __host__ __device__ const void* const* out_list() const { return static_cast<const void* const*>(out); }
 };
 
 cudaError_t launch_encode(int dtype, int bits, const State& st, const EncodeArgs& a, cudaStream_t s);
@@ -71,13 +82,16 @@ cudaError_t launch_encode_lowbit(int dtype, int bits, const State& st, const Enc
 cudaError_t launch_decode_lowbit(int dtype, int bits, const State& st, const DecodeArgs& a, cudaStream_t s);
 cudaError_t launch_quant_grad(int dtype, int bits, int lanes_per_group, const void* grad,
                               long long n_elems, uint8_t* packed, float* scales, bool stochastic,
-                              unsigned long long seed, unsigned long long epoch, cudaStream_t s);
+                              unsigned long long seed, unsigned long long epoch, int l2_prefetch, cudaStream_t s);
 cudaError_t launch_dequant_grad(int dtype, int bits, int lanes_per_group, const uint8_t* packed,
                                 const float* scales, long long n_elems, void* out, cudaStream_t s);
 // Rows of `row_bytes` bytes moved by one kernel (in 16-, 4- or 1-byte pieces, as the size and the bases allow): gather: dst row y <- src row
 // ids[y]; scatter: dst row ids[y] <- src row y; entries with ids[y] < 0 are left out.
 cudaError_t launch_copy_rows(const void* src, void* dst, const int32_t* ids, int n, long long row_bytes, bool gather,
                              cudaStream_t s);
+// Up to three byte ranges (sizes multiples of 16, bases 16-byte aligned, all on the current device) copied by
+// one kernel launch.
+cudaError_t launch_wire_copy(const void* const* src, void* const* dst, const size_t* bytes, int n_ranges, cudaStream_t s);
 // *sum_dev += digest of (m, seen); the caller zeroes *sum_dev first.
 cudaError_t launch_checksum(const State& st, unsigned long long* sum_dev, cudaStream_t s);
 

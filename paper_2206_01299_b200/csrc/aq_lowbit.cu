@@ -45,7 +45,7 @@ __device__ __forceinline__ void lowbit_put(const State& st, uint8_t* m_codes, fl
     const float s2 = group_max_any(abs_max8(m_new), st.lanes_per_group);
     unsigned long long km2;
     float dm2, unused[8];
-    quantize8<MBITS, true, false>(m_new, s2, make_uint4(0, 0, 0, 0), dm2, km2, unused);
+    quantize8_for<MBITS, true, false>(m_new, s2, make_uint4(0, 0, 0, 0), dm2, km2, unused);
     store_codes<MBITS>(m_codes, c, lane, write, false, km2);
     if (write && (lane & (st.lanes_per_group - 1)) == 0) m_scales[c >> st.lg_shift] = dm2;
   }
@@ -106,7 +106,7 @@ __device__ __forceinline__ void lowbit_rows(const State& st, const EncodeArgs& e
         const float s = group_max_any(abs_max8(d), st.lanes_per_group);
         uint4 noise = make_uint4(0, 0, 0, 0);                // the message's rounding; the store's stays deterministic
         if constexpr (STOCH) noise = chunk_noise(ea.seed, ea.epoch, stream_id, (uint32_t)c);
-        quantize8<BITS, true, STOCH>(d, s, noise, delta[i], codes, q);
+        quantize8_for<BITS, true, STOCH>(d, s, noise, delta[i], codes, q);
       } else {
         dequantize8<BITS>(kw[i], delta[i], q);
       }

@@ -1,12 +1,14 @@
 // aq_state_checksum_noalloc: the state digest for callers that must not allocate.
 //
-// Who needs it: code that runs where device allocation is off limits -- inside a region that is
-// being captured into a CUDA graph, in a step loop that may not take the allocator's device-wide
-// synchronisation, or in a process whose memory budget was handed out at start-up and has no
-// room left for a library to claim more.  Such a caller cannot give this library a chance to
-// cudaMalloc its working memory, so the working memory of this entry point is part of the
-// library image: a fixed array in device memory that every GPU holds from the moment the
-// library is loaded on it until the process exits.
+// Who needs it: code that runs where device allocation is off limits -- a process whose device
+// memory was all handed out at start-up (a caching pool owns it; a cudaMalloc from a library would
+// fail or force the pool to give memory back), a step loop that may not take the device-wide
+// synchronisation cudaMalloc and cudaFree can bring, a service that gives every library a fixed
+// memory budget.  Such a caller cannot give this library a chance to cudaMalloc its working
+// memory, so the working memory of this entry point is part of the library image: a fixed array
+// in device memory that every GPU holds from the moment the library is loaded on it until the
+// process exits.  The call still synchronises the handle's stream and returns the digest in host
+// memory, exactly like aq_state_checksum.
 //
 // The digest is the one aq_state_checksum returns.  It is formed in two steps: every CTA sums
 // the mixed words of one slab of m into its own slot of the fixed array, then one CTA adds the
@@ -77,7 +79,9 @@ __global__ void __launch_bounds__(aq::kThreads) digest_finish_kernel(const unsig
 
 // Device address of the fixed array on `device` (which must be current).  In host code the
 // array's name is only a handle for the runtime; the address a kernel can use has to be asked
-// for, once per device.
+// for, once per device.  The first call of the entry point on a device does this and should come
+// before any stream capture begins; the address is kept until the process ends (a cudaDeviceReset
+// would make it stale).
 std::mutex g_setup_lock;
 unsigned long long* g_scratch_addr[kMaxDevices] = {nullptr};
 

@@ -30,7 +30,7 @@ def _grad_input(n, group, dtype, seed):
 
 @pytest.mark.parametrize("dtype", ["fp16", "bf16"])
 @pytest.mark.parametrize("bits", range(1, 9))
-@pytest.mark.parametrize("group,n_groups", [(8, 1), (8, 333), (64, 4097), (128, 777), (256, 130)])
+@pytest.mark.parametrize("group,n_groups", [(8, 1), (8, 333), (16, 1), (16, 333), (32, 77), (64, 4097), (128, 777), (256, 130)])
 def test_quant_and_dequant_grad_match_oracle(dtype, bits, group, n_groups):
     td = torch.float16 if dtype == "fp16" else torch.bfloat16
     n = group * n_groups                               # ragged: not a multiple of the CTA tile
@@ -199,8 +199,12 @@ def test_bad_duplicate_and_rawless_ids_are_skipped_like_the_oracle():
 def test_host_side_argument_errors():
     with pytest.raises(aq.AqError):
         aq.aq_create(4, 2, 100, 4, 64)          # group does not divide hidden
-    with pytest.raises(aq.AqError):
-        aq.aq_create(4, 2, 96, 4, 24)           # unsupported group
+    with pytest.raises(aq.AqError) as e:
+        aq.aq_create(4, 2, 96, 4, 24)           # a valid group that no kernel is built for
+    assert e.value.code == aq.AQ_EUNSUPPORTED and "24" in str(e.value)
+    with pytest.raises(aq.AqError) as e:
+        aq.aq_create(4, 2, 96, 4, 12)           # not a whole number of 16-byte pieces
+    assert e.value.code == aq.AQ_EINVAL
     with pytest.raises(aq.AqError):
         aq.aq_create(0, 2, 64, 4, 64)
     h = aq.aq_create(4, 2, 64, 4, 64)

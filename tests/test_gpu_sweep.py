@@ -59,8 +59,7 @@ def test_pipeline_sweep_boundary_major():
                         # backward: receiver -> channel -> sender
                         grad = synth.gradient(bwd, call, device="cuda", stream=boundary)
                         aq.aq_quant_grad(gr.h, grad, n, bbits, gtx_p, gtx_s)
-                        grx_p.copy_(gtx_p)
-                        grx_s.copy_(gtx_s)
+                        aq.aq_wire_copy_grad(gr.h, 0, grx_p, grx_s, gtx_p, gtx_s, n, bbits)
                         aq.aq_dequant_grad(gs.h, grx_p, grx_s, n, bbits, gout)
                         torch.cuda.synchronize()
                         check_guards(*guards, gs.first_guarded, gr.first_guarded)
@@ -86,6 +85,45 @@ def test_pipeline_sweep_boundary_major():
             os_.close()
             or_.close()
     assert len(set(digests)) == synth.SWEEP_BOUNDARIES              # every boundary saw its own data
+
+
+def test_wire_copies_of_odd_sizes_and_bad_arguments():
+    """Messages whose byte counts are not multiples of 16 travel by plain copies instead of the one-launch
+    kernel: the bytes that arrive are the same, and nothing lands outside the receiver's buffers."""
+    cfg = synth.Boundary("wire-odd", 4, 2, 3, 64, "fp16", 3, 64, 2, "normal", 0.1, seed=55)     # 72 bytes of codes per sample
+    gs = GpuSide(cfg, 2)
+    try:
+        tx = guarded_outputs(cfg, 2)
+        rx = guarded_outputs(cfg, 2)
+        ids = torch.tensor([1, 3], dtype=torch.int32, device="cuda")
+        for epoch in range(2):
+            act = synth.activation(cfg, [1, 3], epoch, device="cuda")
+            for g in rx:
+                g.t.view(torch.uint8).fill_(0xEE)
+            aq.aq_encode(gs.h, act, ids, tx[0].t, tx[1].t)
+            aq.aq_wire_copy(gs.h, 0, rx[0].t, rx[1].t, rx[2].t if epoch == 0 else None, tx[0].t, tx[1].t, act if epoch == 0 else None)
+            torch.cuda.synchronize()
+            check_guards(*tx, *rx)
+            assert torch.equal(rx[0].t, tx[0].t) and torch.equal(rx[1].t.view(torch.int32), tx[1].t.view(torch.int32))
+            assert torch.equal(rx[2].t, act) == (epoch == 0)
+        n, bits = 3 * 64, 5                                          # 120 bytes of codes, 12 bytes of steps
+        grad = torch.randn(n, device="cuda").half()
+        g_tx = (Guarded(n * bits // 8, torch.uint8), Guarded(n // 64, torch.float32))
+        g_rx = (Guarded(n * bits // 8, torch.uint8), Guarded(n // 64, torch.float32))
+        aq.aq_quant_grad(gs.h, grad, n, bits, g_tx[0].t, g_tx[1].t)
+        aq.aq_wire_copy_grad(gs.h, 0, g_rx[0].t, g_rx[1].t, g_tx[0].t, g_tx[1].t, n, bits)
+        torch.cuda.synchronize()
+        check_guards(*g_tx, *g_rx)
+        assert torch.equal(g_rx[0].t, g_tx[0].t) and torch.equal(g_rx[1].t, g_tx[1].t)
+        aq.aq_wire_copy_grad(gs.h, 0, None, None, None, None, 0, bits)                # nothing to move
+        with pytest.raises(aq.AqError):
+            aq.aq_wire_copy_grad(gs.h, 0, g_rx[0].t, g_rx[1].t, g_tx[0].t, g_tx[1].t, n + 1, bits)
+        with pytest.raises(aq.AqError):
+            aq.aq_wire_copy_grad(gs.h, 99, g_rx[0].t, g_rx[1].t, g_tx[0].t, g_tx[1].t, n, bits)
+        with pytest.raises(aq.AqError):
+            aq.aq_wire_copy(gs.h, 0, rx[0].t, rx[1].t, rx[2].t, tx[0].t, tx[1].t, None)
+    finally:
+        gs.close()
 
 
 def _full_size_sampled(cfg, per_launch, steps, samples_per_launch, wire=False):
@@ -178,8 +216,7 @@ def test_sweep_boundary_full_id_space_in_the_benchmark_launch_shape():
                   Guarded(n, torch.float16))
         tx_p, tx_s, rx_p, rx_s, gout = (g.t for g in guards)
         aq.aq_quant_grad(h, grad, n, bits, tx_p, tx_s)
-        rx_p.copy_(tx_p)
-        rx_s.copy_(tx_s)
+        aq.aq_wire_copy_grad(h, torch.cuda.current_device(), rx_p, rx_s, tx_p, tx_s, n, bits)
         aq.aq_dequant_grad(h, rx_p, rx_s, n, bits, gout)
         torch.cuda.synchronize()
         check_guards(*guards)

@@ -54,7 +54,7 @@ def test_constants_match_the_header():
     for name in ("AQ_OK", "AQ_EINVAL", "AQ_ENOMEM", "AQ_ECUDA", "AQ_EUNSUPPORTED", "AQ_DTYPE", "AQ_BATCH",
                  "AQ_STREAM", "AQ_RAW", "AQ_FIRST_FLAGS", "AQ_ROWS_PER_CTA", "AQ_ROUNDING", "AQ_SEED", "AQ_EPOCH", "AQ_L2_PREFETCH",
                  "AQ_ROUND_INTERVAL", "AQ_ROUND_STOCHASTIC", "AQ_FP16", "AQ_BF16",
-                 "AQ_ST_BAD_ID", "AQ_ST_DUP_ID", "AQ_ST_NO_RAW", "AQ_ST_STAGED"):
+                 "AQ_ST_BAD_ID", "AQ_ST_DUP_ID", "AQ_ST_NO_RAW", "AQ_ST_STAGED", "AQ_ST_BAD_PTR", "AQ_RAW_LIST"):
         m = re.search(rf"\b{name}\s*=\s*(-?\d+)", text)
         assert m, name
         assert getattr(aq, name) == int(m.group(1)), name

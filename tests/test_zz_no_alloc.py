@@ -1,9 +1,9 @@
 """aq_state_checksum_noalloc against aq_state_checksum, through the C ABI.
 
-The entry point under test serves callers that may not allocate device memory at the time
-of the call (inside a graph capture, in a loop that cannot take an allocator's
-synchronisation, in a process with no memory left to hand out): its scratch is a fixed
-array in the library image.  The digest must be the same 64 bits that the allocating entry
+The entry point under test serves callers that cannot allocate device memory at the time
+of the call (a process whose memory a caching pool handed out at start-up, a loop that cannot
+take an allocator's device-wide synchronisation, a service with a fixed memory budget per
+library): its scratch is a fixed array in the library image.  The digest must be the same 64 bits that the allocating entry
 point returns -- the tolerance of every other digest test here: bit-exact -- and because the
 fixed array keeps the previous call's contents, the check is made on consecutive calls, on
 states of different sizes, and after the state changed.
@@ -11,9 +11,13 @@ states of different sizes, and after the state changed.
 This file sorts last on purpose: a run that stops at the first failure has then already
 run every other test.
 """
+import ctypes
+
+import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2206_01299_b200 as aq
 from fixtures import synth
 
@@ -84,3 +88,42 @@ def test_noalloc_digest_rejects_null_output():
         assert "null" in aq.aq_last_error(h)
     finally:
         aq.aq_destroy(h)
+
+
+def test_noalloc_digest_refuses_the_stores_it_is_not_built_for():
+    for create in (lambda: aq.aq_create_lowbit(4, 2, 64, 4, 64, 8), lambda: aq.aq_create_fp32(4, 2, 64, 4, 64)):
+        h = create()
+        try:
+            rc = aq.lib().aq_state_checksum_noalloc(h, ctypes.byref(ctypes.c_uint64(0)))
+            assert rc == aq.AQ_EUNSUPPORTED
+            assert "store" in aq.aq_last_error(h)
+        finally:
+            aq.aq_destroy(h)
+
+
+def test_noalloc_digest_of_a_hosted_store_after_a_staged_call():
+    """m in page-locked host memory, visited through aq_prefetch: the digest call has to wait for the rows
+    that are still travelling back to the host block, and must then equal the allocating digest and the
+    oracle's, on a stream of the caller's own, with a ragged bf16 state."""
+    cfg = synth.Boundary("noalloc-hosted", 6, 3, 37, 136, "bf16", 3, 8, 2, "outlier", 0.3, seed=94)
+    stream = torch.cuda.Stream()
+    h = aq.aq_create_hosted(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group)
+    o = oracle.Side(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, oracle.BF16)
+    try:
+        aq.aq_configure(h, aq.AQ_DTYPE, aq.AQ_BF16)
+        aq.aq_configure(h, aq.AQ_BATCH, cfg.n_batch)
+        aq.aq_configure(h, aq.AQ_STREAM, stream.cuda_stream)
+        packed = torch.empty((cfg.n_batch, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
+        scales = torch.empty((cfg.n_batch, cfg.groups), dtype=torch.float32, device="cuda")
+        for epoch, id_list in [(0, [5, 0, 2]), (1, [2, 5, 0]), (1, [1, 3, 4])]:
+            ids = torch.tensor(id_list, dtype=torch.int32)
+            act = synth.activation(cfg, ids, epoch, device="cuda")
+            torch.cuda.synchronize()
+            aq.aq_prefetch(h, ids)
+            aq.aq_encode(h, act, ids.cuda(), packed, scales)
+            got = aq.aq_state_checksum_noalloc(h)                       # no synchronisation in between: the write-back is in flight
+            o.encode(act.view(torch.int16).cpu().numpy().view(np.uint16), ids.numpy())
+            assert got == o.checksum() == aq.aq_state_checksum(h) == aq.aq_state_checksum_noalloc(h)
+    finally:
+        aq.aq_destroy(h)
+        o.close()
