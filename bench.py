@@ -49,7 +49,10 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of one delta-visit launch from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum),
 # per element, by workload; reported as roofline.traffic only while the kernel sources still hash to the
 # value recorded with the capture (`python bench.py --kernel-hash` prints the current one).
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    "gpt2": {"kernel_hash": "b5d74788fc8525c8", "encode_bytes_per_element": (209755904 + 78299648) / 52428800,
+             "capture": "ncu --set full, encode_kernel<__half,4,8,0>, one launch of 32 sequences on the 128-id case"},
+}
 
 
 def kernel_source_hash():
@@ -417,7 +420,11 @@ def measure_boundary(args, env, name, steps, warmup, headline):
 
     packed = torch.empty((macro, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
     scales = torch.empty((macro, cfg.groups), dtype=torch.float32, device="cuda")
-    out = torch.empty((macro, cfg.seq, cfg.hidden), dtype=cfg.torch_dtype, device="cuda")
+    # the receiver's output rotates over buffers that together exceed twice the L2, so that no launch finds the
+    # lines it is about to overwrite still dirty in cache
+    n_outs = max(2, math.ceil(2 * 126e6 / (macro * cfg.elems * 2)) + 1)
+    outs = [torch.empty((macro, cfg.seq, cfg.hidden), dtype=cfg.torch_dtype, device="cuda") for _ in range(n_outs)]
+    out = outs[0]
 
     sweep = name == "sweep"
     if sweep:
@@ -428,7 +435,7 @@ def measure_boundary(args, env, name, steps, warmup, headline):
         grads = [synth.gradient(replace(bw, n_batch=macro), i, device="cuda") for i in range(4)]
         g_tx = (torch.empty(n_grad * bbits // 8, dtype=torch.uint8, device="cuda"), torch.empty(n_grad // bw.group, dtype=torch.float32, device="cuda"))
         g_rx = (torch.empty_like(g_tx[0]), torch.empty_like(g_tx[1]))
-        g_out = torch.empty(n_grad, dtype=cfg.torch_dtype, device="cuda")
+        g_outs = [torch.empty(n_grad, dtype=cfg.torch_dtype, device="cuda") for _ in range(n_outs)]
         grad_bytes = n_grad * (2 + bbits / 8 + 4 / bw.group)
         step_bytes += (2 * grad_bytes                                                  # quantize + dequantize
                        + 2 * (macro * (cfg.packed_bytes + cfg.groups * 4))             # forward wire: read + write
@@ -468,7 +475,7 @@ def measure_boundary(args, env, name, steps, warmup, headline):
         for l in range(launches_per_step):
             lo = s * macro + l * nb
             a, i = arena[lo:lo + nb], ids_dev[lo:lo + nb]
-            p, sc, o = packed[l * nb:(l + 1) * nb], scales[l * nb:(l + 1) * nb], out[l * nb:(l + 1) * nb]
+            p, sc, o = packed[l * nb:(l + 1) * nb], scales[l * nb:(l + 1) * nb], outs[s % n_outs][l * nb:(l + 1) * nb]
             if prefetching and ahead["key"] != (ids_dev.data_ptr(), lo):
                 prefetch(ids_dev, lo)
             aq.aq_encode(snd, a, i, p, sc)
@@ -489,7 +496,7 @@ def measure_boundary(args, env, name, steps, warmup, headline):
         if sweep:
             aq.aq_quant_grad(rcv, grads[s % 4], n_grad, bbits, g_tx[0], g_tx[1])
             aq.aq_wire_copy_grad(rcv, local_rank, g_rx[0], g_rx[1], g_tx[0], g_tx[1], n_grad, bbits)    # the backward wire
-            aq.aq_dequant_grad(snd, g_rx[0], g_rx[1], n_grad, bbits, g_out)
+            aq.aq_dequant_grad(snd, g_rx[0], g_rx[1], n_grad, bbits, g_outs[s % n_outs])
 
     ev = lambda: torch.cuda.Event(enable_timing=True)
 
@@ -512,7 +519,8 @@ def measure_boundary(args, env, name, steps, warmup, headline):
             arena, ids_dev, s = step_source(first_step + w)
             for l in range(launches_per_step):
                 lo = s * macro + l * nb
-                aq.aq_decode(rcv, wp[w, l * nb:(l + 1) * nb], ws[w, l * nb:(l + 1) * nb], ids_dev[lo:lo + nb], out[l * nb:(l + 1) * nb])
+                aq.aq_decode(rcv, wp[w, l * nb:(l + 1) * nb], ws[w, l * nb:(l + 1) * nb], ids_dev[lo:lo + nb],
+                             outs[w % n_outs][l * nb:(l + 1) * nb])
         e[2].record(stream)
         torch.cuda.synchronize()
         n = window * launches_per_step
@@ -520,17 +528,18 @@ def measure_boundary(args, env, name, steps, warmup, headline):
 
     def grad_pass(window):
         """The same for the sweep's backward kernels: `window` quantize launches back to back, then
-        `window` dequantize launches (one wire buffer per rotating gradient)."""
-        tx = [(torch.empty_like(g_tx[0]), torch.empty_like(g_tx[1])) for _ in range(4)]
-        for i in range(4):
-            aq.aq_quant_grad(rcv, grads[i], n_grad, bbits, tx[i][0], tx[i][1])
+        `window` dequantize launches; gradients, wire buffers and outputs rotate over sets larger than L2."""
+        n_tx = math.ceil(2 * 126e6 / (n_grad * bbits // 8)) + 1
+        tx = [(torch.empty_like(g_tx[0]), torch.empty_like(g_tx[1])) for _ in range(n_tx)]
+        for i in range(n_tx):
+            aq.aq_quant_grad(rcv, grads[i % 4], n_grad, bbits, tx[i][0], tx[i][1])
         e = [ev(), ev(), ev()]
         e[0].record(stream)
         for w in range(window):
-            aq.aq_quant_grad(rcv, grads[w % 4], n_grad, bbits, tx[w % 4][0], tx[w % 4][1])
+            aq.aq_quant_grad(rcv, grads[w % 4], n_grad, bbits, tx[w % n_tx][0], tx[w % n_tx][1])
         e[1].record(stream)
         for w in range(window):
-            aq.aq_dequant_grad(snd, tx[w % 4][0], tx[w % 4][1], n_grad, bbits, g_out)
+            aq.aq_dequant_grad(snd, tx[w % n_tx][0], tx[w % n_tx][1], n_grad, bbits, g_outs[w % n_outs])
         e[2].record(stream)
         torch.cuda.synchronize()
         return e[0].elapsed_time(e[1]) / window, e[1].elapsed_time(e[2]) / window
@@ -569,6 +578,8 @@ def measure_boundary(args, env, name, steps, warmup, headline):
     first_ms = e0.elapsed_time(e1)
     aq.aq_configure(rcv, aq.AQ_RAW, None)
     first_bytes = cfg.n_samples * cfg.elems * ((4 + cfg.bits / 8 + 4 / cfg.group) + 6)
+    if sweep:                                          # the steps of that epoch also carry the wires and the gradient kernels
+        first_bytes += steps_per_epoch * (step_bytes - 2 * macro * cfg.elems * bpe)
     del arena0
 
     # ---- steady-state epochs: inputs resident in HBM before the clock starts
@@ -676,7 +687,7 @@ def measure_boundary(args, env, name, steps, warmup, headline):
     # ---- calls of the workload's own micro-batch size, enqueued back to back on the plain stream and as one CUDA graph
     micro = None
     if not (hosted or use_graph) and nb != cfg.n_batch:
-        micro = micro_batch_calls(aq, torch, stream, snd, rcv, cfg, step_source, total_steps + 2 + 3 * window, macro, packed, scales, out,
+        micro = micro_batch_calls(aq, torch, stream, snd, rcv, cfg, step_source, total_steps + 2 + 3 * window, macro, packed, scales, outs,
                                   bpe)
         for h in handles:
             aq.aq_configure(h, aq.AQ_BATCH, nb)
@@ -736,7 +747,7 @@ def measure_boundary(args, env, name, steps, warmup, headline):
     res["cfg"] = cfg
     for h in handles:
         aq.aq_destroy(h)
-    del arenas, id_lists, packed, scales, out
+    del arenas, id_lists, packed, scales, out, outs
     torch.cuda.empty_cache()
     return res
 
@@ -831,7 +842,7 @@ def measure_pipeline(args, env):
             "gpu_launches": 30 * steps}
 
 
-def micro_batch_calls(aq, torch, stream, snd, rcv, cfg, step_source, first_step, macro, packed, scales, out, bpe, steps=24):
+def micro_batch_calls(aq, torch, stream, snd, rcv, cfg, step_source, first_step, macro, packed, scales, outs, bpe, steps=24):
     """Sustained throughput of calls the size of the workload's own micro-batch (1 or 8 sequences): the
     micro-batches of `steps` macro-batches, each encoded then decoded, enqueued back to back -- once call by
     call through the binding on the plain stream, once as CUDA graphs of one macro-batch each."""
@@ -846,7 +857,8 @@ def micro_batch_calls(aq, torch, stream, snd, rcv, cfg, step_source, first_step,
         for l in range(per_step):
             lo = s * macro + l * nb
             aq.aq_encode(snd, arena[lo:lo + nb], ids_dev[lo:lo + nb], packed[l * nb:(l + 1) * nb], scales[l * nb:(l + 1) * nb])
-            aq.aq_decode(rcv, packed[l * nb:(l + 1) * nb], scales[l * nb:(l + 1) * nb], ids_dev[lo:lo + nb], out[l * nb:(l + 1) * nb])
+            aq.aq_decode(rcv, packed[l * nb:(l + 1) * nb], scales[l * nb:(l + 1) * nb], ids_dev[lo:lo + nb],
+                         outs[t % len(outs)][l * nb:(l + 1) * nb])
 
     with torch.cuda.stream(stream):
         one_step(first_step)

@@ -86,7 +86,7 @@ enum {
                             independent random numbers need different values (for activations the epoch
                             or step number; for gradients any number unique to the call); default 0 */
   AQ_ROWS_PER_CTA = 6,   /* tuning: rows (256 chunks = 2048 elements each) that one CTA of aq_encode /
-                            aq_decode walks; 0 (default) = chosen from the size of the call (2..4) */
+                            aq_decode walks; 0 (default) = chosen from the size of the call (1..4) */
   AQ_L2_PREFETCH = 10,   /* tuning: 1 (default for stores in device memory) = every CTA of aq_encode /
                             aq_decode asks for its rows of act and m, and every CTA of aq_quant_grad for its
                             piece of the gradient, to be brought into L2 ahead of its loads (bulk-prefetch
@@ -151,16 +151,21 @@ aq_handle* aq_create_hosted(int64_t n_samples, int seq, int hidden, int bits, in
  * call ahead of time (Section 3.3 and the appendix on offloading: the previous messages are
  * prefetched from host memory while the preceding stages compute, so the transfer is off the
  * critical path).  sample_ids_host int32[n] (host; copied before the call returns), n must equal
- * AQ_BATCH now and at that call.  The call returns at once; on a copy stream of the handle's
- * own, behind everything issued so far on the handle's stream, each sample's row of m is copied
- * into a staging block in device memory (n rows, allocated at the first use and when n grows):
- * by one copy per row, or by one kernel when there are more than 64 rows or rows under 64 KB.
+ * AQ_BATCH now and at that call.  The call returns at once; on a stream of the handle's own
+ * each sample's row of m is copied into a staging block in device memory (n rows, allocated at
+ * the first use and when n grows): by one copy per row, or by one kernel when there are more than
+ * 64 rows or rows under 64 KB.  Two staging blocks are used in turn and the rows travel home on a
+ * second stream, so the fetch for call N+1 may be asked for as soon as call N is issued: it runs
+ * beside call N's kernel and beside the write-back of call N's rows (both directions of the host
+ * link at once) and waits only for what it must -- the write-back of the block it reuses, the
+ * write-back of call N where both calls touch a sample, and calls that worked on the host block in
+ * place.
  * The next aq_encode / aq_decode (aq_encode_host / aq_decode_host too) then
  *   - waits on the device, not on the host, until the rows have arrived,
  *   - runs the same kernel on the staged rows at device-memory speed, with the same results as
  *     on the host block in place, and
- *   - starts the copy of the rows back to host memory on the copy stream, again without
- *     blocking the caller; every later call that touches m waits for it on the device.
+ *   - starts the copy of the rows back to host memory on the second stream, again without
+ *     blocking the caller; every later call that touches m in place waits for it on the device.
  * That call must bring the prefetched ids, position by position: a sample whose id differs is
  * skipped (codes and scales zero, m untouched, as for a bad id) and AQ_ST_STAGED is set.  Ids
  * out of range and repeated ids are not fetched and the call reports them as always.  Between

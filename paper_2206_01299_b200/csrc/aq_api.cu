@@ -27,28 +27,36 @@ struct aq_handle {
   unsigned long long* sum_dev = nullptr;     // scratch of aq_state_checksum
   void* m_host = nullptr;                    // hosted store: the pinned host block that st.m maps
   float* m_scales_host = nullptr;            // ... and the one that st.m_scales maps (low-precision hosted store)
-  // hosted store, staged visits: aq_prefetch copies the next call's m(xi) into `slots` on
-  // copy_stream, the call works there and copies the rows back on copy_stream afterwards
-  cudaStream_t copy_stream = nullptr;
+  // hosted store, staged visits: aq_prefetch copies the next call's m(xi) into a staging block in device
+  // memory on fetch_stream, the call works there and copies the rows back on store_stream afterwards.  Two
+  // blocks are used in turn, so that the rows of call N+1 arrive while call N computes and while its rows
+  // travel home, and the two directions of the host link work at the same time.
+  struct Stage {
+    void* slots = nullptr;                   // [batch] rows of m (16-bit values, or the codes of a low-precision store)
+    float* slot_scales = nullptr;            // [batch][groups] steps of those rows (low-precision store)
+    int32_t* d_slot_ids = nullptr;           // [batch] ids as given to aq_prefetch
+    int32_t* d_copy_ids = nullptr;           // [batch] the same with -1 where no row is to be moved
+    int batch = 0;
+    std::vector<int32_t> ids;                // per slot: the sample whose row it holds, -1 = nothing to copy
+    bool rows_by_kernel = false;             // how this block's rows travel (see aq_prefetch)
+    cudaEvent_t ev_staged = nullptr;         // fetch_stream: the prefetched rows are in HBM
+    cudaEvent_t ev_computed = nullptr;       // the handle's stream: the call that used them is done
+    cudaEvent_t ev_written = nullptr;        // store_stream: its rows are back in host memory
+    bool writeback_issued = false;
+  };
+  static constexpr int kStages = 2;
+  Stage stage[kStages];
+  int next_stage = 0;                        // the block that the next aq_prefetch fills
+  int pending_stage = -1;                    // the block of the pending prefetch, -1 = none
+  cudaStream_t fetch_stream = nullptr, store_stream = nullptr;
   cudaEvent_t ev_settled = nullptr;          // the handle's stream, when aq_prefetch was called
-  cudaEvent_t ev_staged = nullptr;           // copy_stream: the prefetched rows are in HBM
-  cudaEvent_t ev_computed = nullptr;         // the handle's stream: the call that used them is done
-  cudaEvent_t ev_written = nullptr;          // copy_stream: its rows are back in host memory
-  void* slots = nullptr;                     // [slots_batch] rows of m (16-bit values, or the codes of a low-precision store)
-  float* slot_scales = nullptr;              // [slots_batch][groups] steps of those rows (low-precision store)
-  int32_t* d_slot_ids = nullptr;             // [slots_batch] ids as given to aq_prefetch
-  int32_t* d_copy_ids = nullptr;             // [slots_batch] the same with -1 where no row is to be moved
-  bool rows_by_kernel = false;               // how the pending prefetch's rows travel (see aq_prefetch)
-  int slots_batch = 0;
-  std::vector<int32_t> staged_ids;           // per slot: the sample whose row it holds, -1 = nothing to copy
   // the ids travel to d_slot_ids from page-locked blocks used in turn (a pageable source would
-  // make the copy wait on the host for copy_stream to drain); an event says when one is free again
+  // make the copy wait on the host for fetch_stream to drain); an event says when one is free again
   static constexpr int kIdRing = 4;
   int32_t* ids_pinned[kIdRing] = {nullptr, nullptr, nullptr, nullptr};
   cudaEvent_t ev_ids_sent[kIdRing] = {nullptr, nullptr, nullptr, nullptr};
   unsigned prefetches = 0;
-  bool prefetch_pending = false;
-  bool writeback_issued = false;
+  bool inplace_since_fetch = true;           // a call worked on the host block in place since the last prefetch was issued
   // staging for the host-buffer entry points, sized for staged_batch samples
   int staged_batch = 0;
   void* d_act = nullptr;      // also raw / out
@@ -152,61 +160,65 @@ bool sliceable(const aq_handle* h, const int32_t* ids_host) {
   return true;
 }
 
-// Hosted store: rows that a staged call updated travel back to host memory on copy_stream.
+// Hosted store: rows that staged calls updated travel back to host memory on store_stream.
 // Whatever touches the host block next on the handle's stream waits for them on the device.
 cudaError_t settle(aq_handle* h) {
-  if (!h->writeback_issued) return cudaSuccess;
-  return cudaStreamWaitEvent(h->stream, h->ev_written, 0);
+  for (aq_handle::Stage& sg : h->stage) {
+    if (!sg.writeback_issued) continue;
+    const cudaError_t e = cudaStreamWaitEvent(h->stream, sg.ev_written, 0);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 
-// The rows of the pending prefetch between the host blocks and the staging blocks, on
-// copy_stream: in = host to staging.  A low-precision store has two blocks, codes and steps.
-int move_rows(aq_handle* h, bool in) {
-  const int n = (int)h->staged_ids.size();
+// The rows of one staging block between the host blocks and the block, on `stream`: in = host to
+// staging.  A low-precision store has two blocks, codes and steps.
+int move_rows(aq_handle* h, aq_handle::Stage& sg, bool in, cudaStream_t stream) {
+  const int n = (int)sg.ids.size();
   const size_t bytes = (size_t)h->st.m_bytes, step_bytes = (size_t)h->st.groups * sizeof(float);
   const cudaMemcpyKind kind = in ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToHost;
-  if (h->rows_by_kernel) {
-    AQ_CUDA(h, aq::launch_copy_rows(in ? h->st.m : h->slots, in ? h->slots : h->st.m, h->d_copy_ids, n, (long long)bytes, in,
-                                    h->copy_stream));
+  if (sg.rows_by_kernel) {
+    AQ_CUDA(h, aq::launch_copy_rows(in ? h->st.m : sg.slots, in ? sg.slots : h->st.m, sg.d_copy_ids, n, (long long)bytes, in, stream));
     if (h->m_scales_host)
-      AQ_CUDA(h, aq::launch_copy_rows(in ? h->st.m_scales : h->slot_scales, in ? h->slot_scales : h->st.m_scales, h->d_copy_ids,
-                                      n, (long long)step_bytes, in, h->copy_stream));
+      AQ_CUDA(h, aq::launch_copy_rows(in ? h->st.m_scales : sg.slot_scales, in ? sg.slot_scales : h->st.m_scales, sg.d_copy_ids,
+                                      n, (long long)step_bytes, in, stream));
     return AQ_OK;
   }
   for (int j = 0; j < n; ++j) {
-    const int32_t id = h->staged_ids[j];
+    const int32_t id = sg.ids[j];
     if (id < 0) continue;
     char* host_row = static_cast<char*>(h->m_host) + (size_t)id * bytes;
-    char* slot_row = static_cast<char*>(h->slots) + (size_t)j * bytes;
-    AQ_CUDA(h, cudaMemcpyAsync(in ? slot_row : host_row, in ? host_row : slot_row, bytes, kind, h->copy_stream));
+    char* slot_row = static_cast<char*>(sg.slots) + (size_t)j * bytes;
+    AQ_CUDA(h, cudaMemcpyAsync(in ? slot_row : host_row, in ? host_row : slot_row, bytes, kind, stream));
     if (h->m_scales_host) {
       float* host_steps = h->m_scales_host + (size_t)id * (size_t)h->st.groups;
-      float* slot_steps = h->slot_scales + (size_t)j * (size_t)h->st.groups;
-      AQ_CUDA(h, cudaMemcpyAsync(in ? slot_steps : host_steps, in ? host_steps : slot_steps, step_bytes, kind, h->copy_stream));
+      float* slot_steps = sg.slot_scales + (size_t)j * (size_t)h->st.groups;
+      AQ_CUDA(h, cudaMemcpyAsync(in ? slot_steps : host_steps, in ? host_steps : slot_steps, step_bytes, kind, stream));
     }
   }
   return AQ_OK;
 }
 
-// A staged call: `launch` runs on the prefetched rows in HBM, then the rows go home.
+// A staged call: `launch` runs on the prefetched rows in HBM, then the rows go home on store_stream.
 template <typename Launch>
 int run_staged(aq_handle* h, Launch launch) {
-  h->prefetch_pending = false;
-  if ((int)h->staged_ids.size() != h->n_batch)
-    return fail(h, AQ_EINVAL, "the pending aq_prefetch was for %d samples, AQ_BATCH is %d", (int)h->staged_ids.size(), h->n_batch);
+  aq_handle::Stage& sg = h->stage[h->pending_stage];
+  h->pending_stage = -1;
+  if ((int)sg.ids.size() != h->n_batch)
+    return fail(h, AQ_EINVAL, "the pending aq_prefetch was for %d samples, AQ_BATCH is %d", (int)sg.ids.size(), h->n_batch);
   aq::State st = h->st;
-  st.m = h->slots;
-  if (h->m_scales_host) st.m_scales = h->slot_scales;
-  st.slot_ids = h->d_slot_ids;
+  st.m = sg.slots;
+  if (h->m_scales_host) st.m_scales = sg.slot_scales;
+  st.slot_ids = sg.d_slot_ids;
   st.l2_prefetch = h->l2_prefetch;                    // the staged rows are in device memory
-  AQ_CUDA(h, cudaStreamWaitEvent(h->stream, h->ev_staged, 0));
+  AQ_CUDA(h, cudaStreamWaitEvent(h->stream, sg.ev_staged, 0));
   AQ_CUDA(h, launch(st));
-  AQ_CUDA(h, cudaEventRecord(h->ev_computed, h->stream));
-  AQ_CUDA(h, cudaStreamWaitEvent(h->copy_stream, h->ev_computed, 0));
-  const int rc = move_rows(h, false);
+  AQ_CUDA(h, cudaEventRecord(sg.ev_computed, h->stream));
+  AQ_CUDA(h, cudaStreamWaitEvent(h->store_stream, sg.ev_computed, 0));
+  const int rc = move_rows(h, sg, false, h->store_stream);
   if (rc != AQ_OK) return rc;
-  AQ_CUDA(h, cudaEventRecord(h->ev_written, h->copy_stream));
-  h->writeback_issued = true;
+  AQ_CUDA(h, cudaEventRecord(sg.ev_written, h->store_stream));
+  sg.writeback_issued = true;
   return AQ_OK;
 }
 
@@ -290,9 +302,12 @@ static aq_handle* create_handle(int64_t n_samples, int seq, int hidden, int bits
     // page-locked host memory that the GPU addresses directly: the kernels stream m over the bus
     e = cudaHostAlloc(&h->m_host, m_bytes, cudaHostAllocMapped | cudaHostAllocPortable);
     if (e == cudaSuccess) e = cudaHostGetDevicePointer(&st.m, h->m_host, 0);
-    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking);
-    for (cudaEvent_t* ev : {&h->ev_settled, &h->ev_staged, &h->ev_computed, &h->ev_written})
-      if (e == cudaSuccess) e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->fetch_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->store_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_settled, cudaEventDisableTiming);
+    for (aq_handle::Stage& sg : h->stage)
+      for (cudaEvent_t* ev : {&sg.ev_staged, &sg.ev_computed, &sg.ev_written})
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming);
     for (int i = 0; i < aq_handle::kIdRing; ++i) {
       if (e == cudaSuccess) e = cudaHostAlloc(reinterpret_cast<void**>(&h->ids_pinned[i]), 2 * aq::kMaxBatch * sizeof(int32_t), cudaHostAllocPortable);
       if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_ids_sent[i], cudaEventDisableTiming);
@@ -334,12 +349,16 @@ void aq_destroy(aq_handle* h) {
     cudaEventDestroy(h->ev_begin);
     for (int i = 0; i < aq_handle::kSlices; ++i) { cudaEventDestroy(h->ev_in[i]); cudaEventDestroy(h->ev_done[i]); }
   }
-  if (h->copy_stream) {
-    cudaStreamSynchronize(h->copy_stream);
-    cudaStreamDestroy(h->copy_stream);
-    cudaEventDestroy(h->ev_settled); cudaEventDestroy(h->ev_staged);
-    cudaEventDestroy(h->ev_computed); cudaEventDestroy(h->ev_written);
-    cudaFree(h->slots); cudaFree(h->slot_scales); cudaFree(h->d_slot_ids); cudaFree(h->d_copy_ids);
+  if (h->fetch_stream) {
+    cudaStreamSynchronize(h->fetch_stream);
+    cudaStreamSynchronize(h->store_stream);
+    cudaStreamDestroy(h->fetch_stream);
+    cudaStreamDestroy(h->store_stream);
+    cudaEventDestroy(h->ev_settled);
+    for (aq_handle::Stage& sg : h->stage) {
+      cudaEventDestroy(sg.ev_staged); cudaEventDestroy(sg.ev_computed); cudaEventDestroy(sg.ev_written);
+      cudaFree(sg.slots); cudaFree(sg.slot_scales); cudaFree(sg.d_slot_ids); cudaFree(sg.d_copy_ids);
+    }
     for (int i = 0; i < aq_handle::kIdRing; ++i) {
       cudaFreeHost(h->ids_pinned[i]);
       cudaEventDestroy(h->ev_ids_sent[i]);
@@ -407,6 +426,7 @@ int aq_configure(aq_handle* h, int key, int64_t value) {
 
 static int launch_encode_call(aq_handle* h, const aq::EncodeArgs& a) {
   AQ_CUDA(h, settle(h));
+  h->inplace_since_fetch = true;
   if (h->st.m_bits) {
     AQ_CUDA(h, aq::launch_encode_lowbit(h->dtype, h->bits, h->st, a, h->stream));
     return AQ_OK;
@@ -417,6 +437,7 @@ static int launch_encode_call(aq_handle* h, const aq::EncodeArgs& a) {
 
 static int launch_decode_call(aq_handle* h, const aq::DecodeArgs& a) {
   AQ_CUDA(h, settle(h));
+  h->inplace_since_fetch = true;
   if (h->st.m_bits) {
     AQ_CUDA(h, aq::launch_decode_lowbit(h->dtype, h->bits, h->st, a, h->stream));
     return AQ_OK;
@@ -436,7 +457,7 @@ static int encode_call(aq_handle* h, const void* act, const int32_t* sample_ids,
   DeviceGuard g(h->device);
   aq::EncodeArgs a{act, sample_ids, static_cast<uint8_t*>(packed), scales, h->first_flags, h->n_batch,
                    h->rounding == AQ_ROUND_STOCHASTIC, h->seed, h->epoch, lists};
-  if (h->prefetch_pending)
+  if (h->pending_stage >= 0)
     return run_staged(h, [&](const aq::State& st) {
       return h->st.m_bits ? aq::launch_encode_lowbit(h->dtype, h->bits, st, a, h->stream)
                           : aq::launch_encode(h->dtype, h->bits, st, a, h->stream);
@@ -465,7 +486,7 @@ static int decode_call(aq_handle* h, const void* packed, const float* scales, co
   DeviceGuard g(h->device);
   aq::DecodeArgs a{static_cast<const uint8_t*>(packed), scales, lists ? static_cast<const void*>(h->raw_list) : h->raw, sample_ids,
                    out, h->first_flags, h->n_batch, lists};
-  if (h->prefetch_pending)
+  if (h->pending_stage >= 0)
     return run_staged(h, [&](const aq::State& st) {
       return h->st.m_bits ? aq::launch_decode_lowbit(h->dtype, h->bits, st, a, h->stream)
                           : aq::launch_decode(h->dtype, h->bits, st, a, h->stream);
@@ -669,44 +690,60 @@ int aq_prefetch(aq_handle* h, const int32_t* sample_ids_host, int n) {
   if (!sample_ids_host) return fail(h, AQ_EINVAL, "aq_prefetch: null pointer");
   DeviceGuard g(h->device);
   const size_t bytes = (size_t)h->st.m_bytes;
-  if (h->slots_batch < n) {
-    AQ_CUDA(h, cudaStreamSynchronize(h->copy_stream));
+  // a prefetch that replaces a pending one reuses its block; otherwise the blocks take turns
+  const int which = h->pending_stage >= 0 ? h->pending_stage : h->next_stage;
+  aq_handle::Stage& sg = h->stage[which];
+  aq_handle::Stage& other = h->stage[1 - which];
+  if (sg.batch < n) {
+    AQ_CUDA(h, cudaStreamSynchronize(h->fetch_stream));
+    AQ_CUDA(h, cudaStreamSynchronize(h->store_stream));
     AQ_CUDA(h, cudaStreamSynchronize(h->stream));
-    cudaFree(h->slots); cudaFree(h->slot_scales); cudaFree(h->d_slot_ids); cudaFree(h->d_copy_ids);
-    h->slots = nullptr; h->slot_scales = nullptr; h->d_slot_ids = nullptr; h->d_copy_ids = nullptr; h->slots_batch = 0;
-    AQ_CUDA(h, cudaMalloc(&h->slots, (size_t)n * bytes));
+    cudaFree(sg.slots); cudaFree(sg.slot_scales); cudaFree(sg.d_slot_ids); cudaFree(sg.d_copy_ids);
+    sg.slots = nullptr; sg.slot_scales = nullptr; sg.d_slot_ids = nullptr; sg.d_copy_ids = nullptr; sg.batch = 0;
+    AQ_CUDA(h, cudaMalloc(&sg.slots, (size_t)n * bytes));
     if (h->m_scales_host)
-      AQ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&h->slot_scales), (size_t)n * (size_t)h->st.groups * sizeof(float)));
-    AQ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&h->d_slot_ids), (size_t)n * sizeof(int32_t)));
-    AQ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&h->d_copy_ids), (size_t)n * sizeof(int32_t)));
-    h->slots_batch = n;
+      AQ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&sg.slot_scales), (size_t)n * (size_t)h->st.groups * sizeof(float)));
+    AQ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&sg.d_slot_ids), (size_t)n * sizeof(int32_t)));
+    AQ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&sg.d_copy_ids), (size_t)n * sizeof(int32_t)));
+    sg.batch = n;
   }
   // rows to move: every id once (the kernels skip an id's later occurrences and ids out of range)
-  h->staged_ids.assign(sample_ids_host, sample_ids_host + n);
+  sg.ids.assign(sample_ids_host, sample_ids_host + n);
   std::unordered_set<int32_t> taken;
-  for (int32_t& id : h->staged_ids)
+  for (int32_t& id : sg.ids)
     if (id < 0 || (long long)id >= h->st.n_samples || !taken.insert(id).second) id = -1;
-  // the copies start once everything issued so far on the handle's stream is done (it may
-  // write the host block in place, and an earlier staged call still owns the slots until
-  // its write-back, which copy_stream runs first)
-  AQ_CUDA(h, cudaEventRecord(h->ev_settled, h->stream));
-  AQ_CUDA(h, cudaStreamWaitEvent(h->copy_stream, h->ev_settled, 0));
+  // What the copies have to wait for, on the device: the block's own rows of two calls ago going home;
+  // the other block's rows going home when that call updates a sample that is fetched again here;
+  // and, when a call has worked on the host block in place since the last prefetch, everything
+  // issued so far on the handle's stream.  Not the call that is computing on the other block.
+  if (sg.writeback_issued) AQ_CUDA(h, cudaStreamWaitEvent(h->fetch_stream, sg.ev_written, 0));
+  if (other.writeback_issued) {
+    bool shared = false;
+    for (int32_t id : other.ids) shared = shared || (id >= 0 && taken.count(id));
+    if (shared) AQ_CUDA(h, cudaStreamWaitEvent(h->fetch_stream, other.ev_written, 0));
+  }
+  if (h->inplace_since_fetch) {
+    AQ_CUDA(h, cudaEventRecord(h->ev_settled, h->stream));
+    AQ_CUDA(h, cudaStreamWaitEvent(h->fetch_stream, h->ev_settled, 0));
+    h->inplace_since_fetch = false;
+  }
   const int ring = (int)(h->prefetches++ % aq_handle::kIdRing);
   AQ_CUDA(h, cudaEventSynchronize(h->ev_ids_sent[ring]));      // long done, unless kIdRing prefetches are queued
   int32_t* copy_ids_pinned = h->ids_pinned[ring] + aq::kMaxBatch;
   memcpy(h->ids_pinned[ring], sample_ids_host, (size_t)n * sizeof(int32_t));
-  memcpy(copy_ids_pinned, h->staged_ids.data(), (size_t)n * sizeof(int32_t));
-  AQ_CUDA(h, cudaMemcpyAsync(h->d_slot_ids, h->ids_pinned[ring], (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice, h->copy_stream));
-  AQ_CUDA(h, cudaMemcpyAsync(h->d_copy_ids, copy_ids_pinned, (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice, h->copy_stream));
-  AQ_CUDA(h, cudaEventRecord(h->ev_ids_sent[ring], h->copy_stream));
+  memcpy(copy_ids_pinned, sg.ids.data(), (size_t)n * sizeof(int32_t));
+  AQ_CUDA(h, cudaMemcpyAsync(sg.d_slot_ids, h->ids_pinned[ring], (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice, h->fetch_stream));
+  AQ_CUDA(h, cudaMemcpyAsync(sg.d_copy_ids, copy_ids_pinned, (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice, h->fetch_stream));
+  AQ_CUDA(h, cudaEventRecord(h->ev_ids_sent[ring], h->fetch_stream));
   // a few large rows: one copy per row through the copy engines, the faster way over the host
   // link; many rows or small ones: one kernel that reads the mapped host block, since a copy
   // call costs microseconds of host time each
-  h->rows_by_kernel = n > 64 || bytes < (64u << 10);
-  const int rc = move_rows(h, true);
+  sg.rows_by_kernel = n > 64 || bytes < (64u << 10);
+  const int rc = move_rows(h, sg, true, h->fetch_stream);
   if (rc != AQ_OK) return rc;
-  AQ_CUDA(h, cudaEventRecord(h->ev_staged, h->copy_stream));
-  h->prefetch_pending = true;
+  AQ_CUDA(h, cudaEventRecord(sg.ev_staged, h->fetch_stream));
+  if (h->pending_stage < 0) h->next_stage = 1 - which;
+  h->pending_stage = which;
   return AQ_OK;
 }
 
@@ -788,6 +825,7 @@ int aq_import_sample(aq_handle* h, int64_t sample_id, const void* m_host, uint8_
   if (!m_host) return fail(h, AQ_EINVAL, "aq_import_sample: null pointer");
   DeviceGuard g(h->device);
   AQ_CUDA(h, settle(h));
+  h->inplace_since_fetch = true;
   const size_t bytes = (size_t)h->st.m_bytes;
   const unsigned long long stamp = seen ? aq::kImportedStamp : 0ull;
   AQ_CUDA(h, cudaMemcpyAsync(static_cast<char*>(h->st.m) + (size_t)sample_id * bytes, m_host, bytes,

@@ -170,3 +170,65 @@ def test_prefetch_argument_checks():
         assert aq.aq_status(hosted) == 0
     finally:
         aq.aq_destroy(dev), aq.aq_destroy(hosted)
+
+
+@pytest.mark.parametrize("m_bits", [0, 8])
+def test_prefetch_issued_while_the_previous_call_is_in_flight(m_bits):
+    """The order a pipeline stage uses: the rows of call N+1 are asked for as soon as call N is
+    issued, with no synchronisation anywhere -- the fetch runs beside call N's kernel and beside the
+    write-back of its rows, on the second staging block.  Consecutive calls share a sample now and
+    then (the fetch then has to wait for that row to come home), a call in between works on the host
+    block in place, and one prefetch is replaced before it is used.  Every output is kept and compared
+    at the end."""
+    cfg = synth.Boundary("staged-overlap", 24, 4, 24, 1536, "bf16" if m_bits else "fp16", 4, 64, 1, "normal", 0.1, seed=519)
+    nb, n_calls = 4, 18
+    if m_bits:
+        create = lambda: aq.aq_create_hosted_lowbit(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, m_bits)
+        o_side = lambda: oracle.SideLow(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, oracle.BF16, m_bits)
+    else:
+        create = lambda: aq.aq_create_hosted(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group)
+        o_side = lambda: oracle.Side(cfg.n_samples, cfg.seq, cfg.hidden, cfg.bits, cfg.group, oracle.FP16)
+    stream = torch.cuda.Stream()
+    hs, hr = create(), create()
+    os_, or_ = o_side(), o_side()
+    rng = np.random.default_rng(519)
+    calls = []
+    for c in range(n_calls):
+        ids = rng.choice(cfg.n_samples, nb, replace=False).astype(np.int32)
+        if c % 3 == 1 and int(calls[-1][0][2]) not in ids[1:]:
+            ids[0] = calls[-1][0][2]                              # a sample of the call before
+        calls.append((torch.from_numpy(ids), synth.activation(cfg, torch.arange(nb) + 4 * c, c % 3, device="cuda")))
+    outs = [(torch.empty((nb, cfg.packed_bytes), dtype=torch.uint8, device="cuda"),
+             torch.empty((nb, cfg.groups), dtype=torch.float32, device="cuda"),
+             torch.empty((nb, cfg.seq, cfg.hidden), dtype=cfg.torch_dtype, device="cuda")) for _ in range(n_calls)]
+    ids_dev = [c[0].cuda() for c in calls]
+    torch.cuda.synchronize()
+    try:
+        for h in (hs, hr):
+            aq.aq_configure(h, aq.AQ_DTYPE, aq.AQ_BF16 if m_bits else aq.AQ_FP16)
+            aq.aq_configure(h, aq.AQ_BATCH, nb)
+            aq.aq_configure(h, aq.AQ_STREAM, stream.cuda_stream)
+        in_place = {7, 13}                                        # these calls fetch nothing ahead
+        aq.aq_prefetch(hs, calls[0][0]), aq.aq_prefetch(hr, calls[0][0])
+        for c, (ids, act) in enumerate(calls):
+            packed, scales, out = outs[c]
+            aq.aq_encode(hs, act, ids_dev[c], packed, scales)
+            aq.aq_configure(hr, aq.AQ_RAW, act)
+            aq.aq_decode(hr, packed, scales, ids_dev[c], out)
+            if c + 1 < n_calls and c + 1 not in in_place:
+                if c == 4:                                        # a prefetch for other samples, replaced before its call
+                    aq.aq_prefetch(hs, calls[c][0]), aq.aq_prefetch(hr, calls[c][0])
+                aq.aq_prefetch(hs, calls[c + 1][0]), aq.aq_prefetch(hr, calls[c + 1][0])
+        torch.cuda.synchronize()
+        for c, (ids, act) in enumerate(calls):
+            a_np = bits16(act)
+            p_o, s_o, _ = os_.encode(a_np, ids.numpy())
+            out_o, _ = or_.decode(p_o, s_o, ids.numpy(), raw=a_np)
+            packed, scales, out = outs[c]
+            assert np.array_equal(packed.cpu().numpy(), p_o), (c, "packed")
+            assert np.array_equal(scales.cpu().numpy().view(np.uint32), s_o.view(np.uint32)), (c, "scales")
+            assert np.array_equal(bits16(out), out_o), (c, "out")
+        assert aq.aq_status(hs) == 0 and aq.aq_status(hr) == 0
+        assert aq.aq_state_checksum(hs) == aq.aq_state_checksum(hr) == os_.checksum() == or_.checksum()
+    finally:
+        aq.aq_destroy(hs), aq.aq_destroy(hr), os_.close(), or_.close()
