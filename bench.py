@@ -77,6 +77,9 @@ def parse_args():
                     help="replicas (default): every rank runs both sides of its own boundary.  pipeline (an even number of "
                          "ranks): ranks 2p and 2p+1 are the sending and the receiving stage of boundary p, the message "
                          "travels between them through torch.distributed (paper_2206_01299_b200.link)")
+    ap.add_argument("--backend", default="nccl", choices=["nccl", "gloo"],
+                    help="process-group backend for N > 1.  gloo lets several ranks share one GPU (rank -> device "
+                         "rank %% device count): a functional check of the multi-rank paths where only one GPU is at hand")
     ap.add_argument("--n-samples", type=int, default=None, help="shrink the id space (profiling runs)")
     ap.add_argument("--per-launch", type=int, default=0, help="sequences handed to one aq_encode call (0 = the whole macro-batch)")
     ap.add_argument("--graph", action="store_true", help="replay each step as a captured CUDA graph")
@@ -684,6 +687,14 @@ def measure_boundary(args, env, name, steps, warmup, headline):
     enc_ms = statistics.median(p[0] for p in passes)          # one disturbed pass must not move the figure
     dec_ms = statistics.median(p[1] for p in passes)
 
+    # ---- the same steps with the two sides on streams of their own
+    overlapped = None
+    if not (hosted or use_graph or prefetching or stochastic or m_bits) and launches_per_step == 1:
+        overlapped = two_stream_steps(aq, torch, snd, rcv, cfg, step_source, total_steps + 2 + 3 * window, macro, outs, stream,
+                                      steps=max(steps, 32), reps=5)
+        overlapped["GB/s"] = 2 * macro * cfg.elems * bpe / overlapped["ms_per_step"] / 1e6
+        overlapped["frac_of_measured_hbm"] = overlapped["GB/s"] / measured_peak()[0]
+
     # ---- calls of the workload's own micro-batch size, enqueued back to back on the plain stream and as one CUDA graph
     micro = None
     if not (hosted or use_graph) and nb != cfg.n_batch:
@@ -712,7 +723,7 @@ def measure_boundary(args, env, name, steps, warmup, headline):
         "decode": {"achieved": dec_gbs, "frac": dec_gbs / peak, "avg_launch_ms": dec_ms},
         "kernel_timing": f"CUDA events around {window * launches_per_step} back-to-back launches of the kernel, median of 3 passes right after the timed steps",
         "first_visit_epoch": {"ms": first_ms, "GB/s": first_bytes / (first_ms * 1e-3) / 1e9},
-        "micro_batch_calls": micro, "clocks": clocks.summary(),
+        "micro_batch_calls": micro, "two_streams": overlapped, "clocks": clocks.summary(),
         "gpu_launches_per_step": launches_per_step * (3 if sweep else 2) + (3 if sweep else 0),
         "peak": peak, "peak_kind": peak_kind,
         "shape": {"hidden": cfg.hidden, "seq": cfg.seq, "micro_batch": cfg.n_batch, "sequences_per_step": macro,
@@ -780,7 +791,8 @@ def measure_pipeline(args, env):
     aq.aq_configure(h, aq.AQ_STREAM, stream.cuda_stream)
     first = torch.zeros(nb, dtype=torch.uint8, device="cuda")
     aq.aq_configure(h, aq.AQ_FIRST_FLAGS, first)
-    link = BoundaryLink(dist, rank + 1 if sender else rank - 1, nb, cfg.packed_bytes, cfg.groups, cfg.elems, cfg.torch_dtype, "cuda")
+    wire_dev = "cuda" if args.backend == "nccl" else "cpu"       # gloo moves host memory only
+    link = BoundaryLink(dist, rank + 1 if sender else rank - 1, nb, cfg.packed_bytes, cfg.groups, cfg.elems, cfg.torch_dtype, wire_dev)
     packed = torch.empty((nb, cfg.packed_bytes), dtype=torch.uint8, device="cuda")
     scales = torch.empty((nb, cfg.groups), dtype=torch.float32, device="cuda")
     out = torch.empty((nb, cfg.seq, cfg.hidden), dtype=cfg.torch_dtype, device="cuda")
@@ -802,6 +814,8 @@ def measure_pipeline(args, env):
                 link.send(ids, first, packed, scales, act)
             else:
                 _, _, p, sc, raw = link.recv(expect_ids=ids)
+                if wire_dev == "cpu":
+                    p, sc, raw = p.cuda(), sc.cuda(), (None if raw is None else raw.cuda())
                 aq.aq_configure(h, aq.AQ_RAW, raw)
                 aq.aq_decode(h, p, sc, ids.cuda(), out)
                 stream.synchronize()
@@ -821,9 +835,9 @@ def measure_pipeline(args, env):
             step(1, arena, (t := t + 1) % steps_per_epoch)
         torch.cuda.synchronize()
         windows_ms.append((time.perf_counter() - t0) * 1e3)
-    ms = torch.tensor(windows_ms, dtype=torch.float64, device="cuda")
+    ms = torch.tensor(windows_ms, dtype=torch.float64, device=wire_dev)
     dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-    digest = torch.tensor([aq.aq_state_checksum(h) & 0x7FFFFFFFFFFFFFFF], dtype=torch.int64, device="cuda")
+    digest = torch.tensor([aq.aq_state_checksum(h) & 0x7FFFFFFFFFFFFFFF], dtype=torch.int64, device=wire_dev)
     both = [torch.zeros_like(digest) for _ in range(world)]
     dist.all_gather(both, digest)
     assert all(both[2 * p].item() == both[2 * p + 1].item() for p in range(world // 2)), "sender and receiver state diverged"
@@ -840,6 +854,50 @@ def measure_pipeline(args, env):
                        "message over torch.distributed send/recv", "sequences_per_step": macro, "wire_bytes_per_step": wire,
                        "timing": "host clock between barriers, median of 30 windows, slowest rank"},
             "gpu_launches": 30 * steps}
+
+
+def two_stream_steps(aq, torch, snd, rcv, cfg, step_source, first_step, macro, outs, home_stream, steps, reps):
+    """Encode and decode of consecutive steps on two streams, the way two stages on two devices work: the
+    receiver decodes message t while the sender already encodes message t+1 (two wire buffers; events hand
+    a buffer from one stream to the other and back).  The forward codec only (no wire copy, no gradients),
+    same handles and data as the timed steps; median of `reps` runs of `steps` steps, by events."""
+    sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+    wires = [(torch.empty((macro, cfg.packed_bytes), dtype=torch.uint8, device="cuda"),
+              torch.empty((macro, cfg.groups), dtype=torch.float32, device="cuda")) for _ in range(2)]
+    torch.cuda.synchronize()
+    aq.aq_configure(snd, aq.AQ_STREAM, sa.cuda_stream)
+    aq.aq_configure(rcv, aq.AQ_STREAM, sb.cuda_stream)
+    times, t0 = [], first_step
+    for rep in range(reps + 1):
+        enc_done = [torch.cuda.Event() for _ in range(steps)]
+        dec_done = [torch.cuda.Event() for _ in range(steps)]
+        begin, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        if hasattr(torch.cuda, "_sleep"):
+            with torch.cuda.stream(sa):
+                torch.cuda._sleep(400_000)                # work queued on both streams before the clock starts
+        begin.record(sa)
+        sb.wait_event(begin)
+        for t in range(steps):
+            arena, ids_dev, s = step_source(t0 + t)
+            lo = s * macro
+            p, sc = wires[t % 2]
+            if t >= 2:
+                sa.wait_event(dec_done[t - 2])            # the receiver has read this wire buffer
+            aq.aq_encode(snd, arena[lo:lo + macro], ids_dev[lo:lo + macro], p, sc)
+            enc_done[t].record(sa)
+            sb.wait_event(enc_done[t])
+            aq.aq_decode(rcv, p, sc, ids_dev[lo:lo + macro], outs[t % len(outs)])
+            dec_done[t].record(sb)
+        end.record(sb)
+        torch.cuda.synchronize()
+        if rep:                                           # the first run warms the streams up
+            times.append(begin.elapsed_time(end) / steps)
+        t0 += steps
+    aq.aq_configure(snd, aq.AQ_STREAM, home_stream.cuda_stream)
+    aq.aq_configure(rcv, aq.AQ_STREAM, home_stream.cuda_stream)
+    return {"ms_per_step": statistics.median(times), "steps": steps, "runs": reps,
+            "note": "sender and receiver handles on two streams, two wire buffers: decode of step t beside encode of step t+1"}
 
 
 def micro_batch_calls(aq, torch, stream, snd, rcv, cfg, step_source, first_step, macro, packed, scales, outs, bpe, steps=24):
@@ -1104,11 +1162,15 @@ def main():
     import paper_2206_01299_b200 as aq
     aq.lib()                                         # fails loudly when the CUDA library is missing
     assert torch.cuda.is_available(), "bench.py needs a CUDA device; there is no CPU path"
+    local_rank = local_rank % torch.cuda.device_count() if args.backend == "gloo" else local_rank
     torch.cuda.set_device(local_rank)
     dist = None
     if world > 1:
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        if args.backend == "nccl":
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        else:
+            dist.init_process_group("gloo")
     if args.prefetch and not args.hosted:
         raise SystemExit("--prefetch needs --hosted")
     if args.hosted and args.m_bits == 32:

@@ -264,8 +264,10 @@ __device__ __forceinline__ void dequantize8(unsigned long long codes, float delt
 // A chunk (8 elements) owns BITS whole bytes at byte offset chunk*BITS of its sample's
 // stream; a full warp owns 32*BITS contiguous bytes = 8*BITS words.
 
-template <int BITS>
-__device__ __forceinline__ void store_codes(uint8_t* stream, long long chunk, int lane, bool active,
+// Idx: the type chunks are numbered with (int inside a sample, wider in the gradient kernel that
+// numbers a whole call): offsets are formed in that type, so 32-bit numbering costs no 64-bit arithmetic.
+template <int BITS, typename Idx>
+__device__ __forceinline__ void store_codes(uint8_t* stream, Idx chunk, int lane, bool active,
                                             bool warp_words, unsigned long long v) {
   if constexpr (BITS == 8) {
     if (active) *reinterpret_cast<uint2*>(stream + chunk * 8) = make_uint2((unsigned)v, (unsigned)(v >> 32));
@@ -326,8 +328,8 @@ __device__ __forceinline__ void store_codes(uint8_t* stream, long long chunk, in
   }
 }
 
-template <int BITS>
-__device__ __forceinline__ unsigned long long load_codes(const uint8_t* stream, long long chunk, int lane,
+template <int BITS, typename Idx>
+__device__ __forceinline__ unsigned long long load_codes(const uint8_t* stream, Idx chunk, int lane,
                                                          bool active, bool warp_words) {
   if constexpr (BITS == 8) {
     if (!active) return 0ull;

@@ -653,8 +653,9 @@ cudaError_t launch_dequant_grad(int dtype, int bits, int lanes_per_group, const 
   if (n_elems <= 0) return cudaSuccess;
   int lg_shift = 0;
   while ((1 << lg_shift) < lanes_per_group) ++lg_shift;
-  // slices of at most 2^30 chunks, each a multiple of a CTA's chunks and therefore of a group and a warp
-  const long long slice = (1ll << 30) / kChunksPerCta * kChunksPerCta;
+  // slices of at most 2^27 chunks (byte offsets into the codes then fit 32 bits), each a multiple of a CTA's
+  // chunks and therefore of a group and a warp
+  const long long slice = (1ll << 27) / kChunksPerCta * kChunksPerCta;
   for (long long done = 0, chunks = n_elems / kChunk; done < chunks; done += slice) {
     const unsigned n = (unsigned)(chunks - done < slice ? chunks - done : slice);
     const uint8_t* p = packed + done * bits;

@@ -27,7 +27,10 @@ import torch
 class BoundaryLink:
     def __init__(self, dist, peer, n_batch, packed_bytes, groups, elems, act_dtype, device="cpu", group=None):
         """dist: torch.distributed (initialised); peer: the rank at the other end of the boundary;
-        sizes per sample as aq_packed_bytes_per_sample / aq_scales_per_sample report them."""
+        sizes per sample as aq_packed_bytes_per_sample / aq_scales_per_sample report them; device: where
+        the message travels from and to ("cuda" with NCCL: straight between the GPUs' memories; "cpu"
+        with gloo: the sender's parts are copied to the host first, and the receiver copies what
+        arrived to its GPU before it decodes)."""
         self.dist, self.peer, self.group = dist, peer, group
         self.n_batch, self.packed_bytes, self.groups, self.elems = n_batch, packed_bytes, groups, elems
         self.act_dtype, self.device = act_dtype, torch.device(device)
@@ -46,11 +49,11 @@ class BoundaryLink:
         ids = ids.to(self.device, torch.int32).reshape(n)
         flags = first_flags.to(self.device).reshape(-1)[:n].to(torch.int32)
         header = torch.cat([torch.tensor([n], dtype=torch.int32, device=self.device), ids, flags])
-        parts = [header, packed.reshape(n, self.packed_bytes), scales.reshape(n, self.groups)]
+        parts = [header, packed.reshape(n, self.packed_bytes).to(self.device), scales.reshape(n, self.groups).to(self.device)]
         first = torch.nonzero(flags.cpu(), as_tuple=False).reshape(-1)          # host read: sizes the message
         if first.numel():
-            rows = act.reshape(n, self.elems).index_select(0, first.to(self.device))
-            parts.append(rows.contiguous())
+            rows = act.reshape(n, self.elems).index_select(0, first.to(act.device))
+            parts.append(rows.contiguous().to(self.device))
         return parts
 
     def unframe(self, header, raw_rows):
