@@ -695,6 +695,14 @@ def measure_boundary(args, env, name, steps, warmup, headline):
         overlapped["GB/s"] = 2 * macro * cfg.elems * bpe / overlapped["ms_per_step"] / 1e6
         overlapped["frac_of_measured_hbm"] = overlapped["GB/s"] / measured_peak()[0]
 
+    # ---- the same steps through the list forms: every sequence of the macro-batch named by a pointer of its own
+    listed = None
+    if overlapped is not None:
+        listed = list_form_steps(aq, torch, snd, rcv, cfg, step_source, total_steps + 2 + 3 * window, macro, packed, scales, outs,
+                                 stream, steps=max(steps, 32), reps=5)
+        listed["GB/s"] = 2 * macro * cfg.elems * bpe / listed["ms_per_step"] / 1e6
+        listed["frac_of_measured_hbm"] = listed["GB/s"] / measured_peak()[0]
+
     # ---- calls of the workload's own micro-batch size, enqueued back to back on the plain stream and as one CUDA graph
     micro = None
     if not (hosted or use_graph) and nb != cfg.n_batch:
@@ -723,7 +731,7 @@ def measure_boundary(args, env, name, steps, warmup, headline):
         "decode": {"achieved": dec_gbs, "frac": dec_gbs / peak, "avg_launch_ms": dec_ms},
         "kernel_timing": f"CUDA events around {window * launches_per_step} back-to-back launches of the kernel, median of 3 passes right after the timed steps",
         "first_visit_epoch": {"ms": first_ms, "GB/s": first_bytes / (first_ms * 1e-3) / 1e9},
-        "micro_batch_calls": micro, "two_streams": overlapped, "clocks": clocks.summary(),
+        "micro_batch_calls": micro, "two_streams": overlapped, "list_form": listed, "clocks": clocks.summary(),
         "gpu_launches_per_step": launches_per_step * (3 if sweep else 2) + (3 if sweep else 0),
         "peak": peak, "peak_kind": peak_kind,
         "shape": {"hidden": cfg.hidden, "seq": cfg.seq, "micro_batch": cfg.n_batch, "sequences_per_step": macro,
@@ -898,6 +906,40 @@ def two_stream_steps(aq, torch, snd, rcv, cfg, step_source, first_step, macro, o
     aq.aq_configure(rcv, aq.AQ_STREAM, home_stream.cuda_stream)
     return {"ms_per_step": statistics.median(times), "steps": steps, "runs": reps,
             "note": "sender and receiver handles on two streams, two wire buffers: decode of step t beside encode of step t+1"}
+
+
+def list_form_steps(aq, torch, snd, rcv, cfg, step_source, first_step, macro, packed, scales, outs, stream, steps, reps):
+    """The timed step through aq_encode_list / aq_decode_list: the macro-batch's sequences are handed over as
+    `macro` separate buffers (here: the rows of the arena and of the wire and output buffers, each named by its
+    own pointer), one launch per side.  Same stream, same data as the timed steps; median of `reps` runs."""
+    row = lambda t: torch.tensor([t[y].data_ptr() for y in range(macro)], dtype=torch.int64, device="cuda")
+    packed_l, scales_l = row(packed), row(scales)
+    outs_l = [row(o) for o in outs]
+    acts_l = {}
+    for t in range(steps):                                   # pointer arrays of the steps, built before the clock starts
+        arena, ids_dev, s = step_source(first_step + t)
+        key = (arena.data_ptr(), s)
+        if key not in acts_l:
+            acts_l[key] = row(arena[s * macro:(s + 1) * macro])
+    torch.cuda.synchronize()
+    times = []
+    with torch.cuda.stream(stream):
+        for rep in range(reps + 1):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            if hasattr(torch.cuda, "_sleep"):
+                torch.cuda._sleep(400_000)
+            a.record(stream)
+            for t in range(steps):
+                arena, ids_dev, s = step_source(first_step + t)
+                ids = ids_dev[s * macro:(s + 1) * macro]
+                aq.aq_encode_list(snd, acts_l[(arena.data_ptr(), s)], ids, packed_l, scales_l)
+                aq.aq_decode_list(rcv, packed_l, scales_l, ids, outs_l[t % len(outs_l)])
+            b.record(stream)
+            torch.cuda.synchronize()
+            if rep:
+                times.append(a.elapsed_time(b) / steps)
+    return {"ms_per_step": statistics.median(times), "steps": steps, "runs": reps,
+            "note": "aq_encode_list + aq_decode_list, one pointer per sequence of the macro-batch"}
 
 
 def micro_batch_calls(aq, torch, stream, snd, rcv, cfg, step_source, first_step, macro, packed, scales, outs, bpe, steps=24):
@@ -1234,7 +1276,7 @@ def main():
                      "timing": head["kernel_timing"],
                      "decode_kernel": head["decode"]},
         "first_visit_epoch": head["first_visit_epoch"],
-        "micro_batch_calls": head["micro_batch_calls"],
+        "micro_batch_calls": head["micro_batch_calls"], "two_streams": head.get("two_streams"), "list_form": head.get("list_form"),
         "e2e": head.get("e2e"), "cpu_baseline": head.get("cpu_baseline"),
         "gpu_launches": args.steps * head["gpu_launches_per_step"] * head["timed"]["windows"],
         "clocks": head["clocks"],

@@ -228,11 +228,13 @@ def test_sweep_boundary_full_id_space_in_the_benchmark_launch_shape():
         aq.aq_destroy(h)
 
 
-def test_deberta_boundary_full_id_space():
-    """32768 ids (25.8 GB of m per side), micro-batch 8 x 256 x 1536 bf16, 2 bit, group 128."""
+@pytest.mark.parametrize("per_launch", [8, 64])
+def test_deberta_boundary_full_id_space(per_launch):
+    """32768 ids (25.8 GB of m per side), 256 x 1536 bf16, 2 bit, group 128: calls of its micro-batch of 8
+    sequences, and of the 64 sequences (a macro-batch) that the benchmark hands to one launch."""
     _needs_gb(60)
     cfg = synth.DEBERTA_XXL
-    _full_size_sampled(cfg, cfg.n_batch, steps=[0, 7, cfg.n_samples // cfg.n_batch - 1], samples_per_launch=3)
+    _full_size_sampled(cfg, per_launch, steps=[0, 7, cfg.n_samples // per_launch - 1], samples_per_launch=3)
 
 
 def test_gpt2_boundary_full_id_space_with_stochastic_rounding():
