@@ -552,13 +552,18 @@ void aqo_dequant_grad(const uint8_t* packed, const float* scales, int64_t n_elem
 }
 
 // Order-independent 64-bit digest of the whole state: the m array read as
-// little-endian 32-bit words (word i = elements 2i, 2i+1), plus the seen set.
+// little-endian 64-bit words (word i = elements 4i .. 4i+3; a last word that
+// the array does not fill is completed with zeros -- the library's shapes,
+// multiples of 8 elements per sample, have none), plus the seen set.
+// (The digest is a requirement of this build, not of the paper: any fixed
+// mixer serves as long as both sides of a comparison use the same one.)
 uint64_t aqo_state_checksum(void* h) {
   Side* S = (Side*)h;
   uint64_t sum = 0;
-  const int64_t nwords = (int64_t)S->m.size() / 2;
+  const int64_t n = (int64_t)S->m.size(), nwords = (n + 3) / 4;
   for (int64_t i = 0; i < nwords; ++i) {
-    const uint32_t w = (uint32_t)S->m[2 * i] | ((uint32_t)S->m[2 * i + 1] << 16);
+    uint64_t w = 0;
+    for (int e = 0; e < 4 && 4 * i + e < n; ++e) w |= (uint64_t)S->m[4 * i + e] << (16 * e);
     sum += mix64((uint64_t)i, w);
   }
   for (int64_t x = 0; x < S->n_samples; ++x)

@@ -352,7 +352,8 @@ def test_checksum_definition_and_sensitivity():
     act = _rand_act(rng, (2, 2, 8), FP16)
     side.encode(act, np.array([2, 0], np.int32))
     m = side.m().reshape(-1)
-    words = m[0::2].astype(np.uint64) | (m[1::2].astype(np.uint64) << np.uint64(16))
+    words = sum(m[e::4].astype(np.uint64) << np.uint64(16 * e) for e in range(4))      # little-endian 64-bit words
+    assert np.array_equal(words, np.ascontiguousarray(m).view(np.uint64))
     want = sum(oracle.mix64(i, int(w)) for i, w in enumerate(words))
     want += sum(oracle.mix64((1 << 40) + x, int(f)) for x, f in enumerate(side.seen()))
     assert side.checksum() == want % (1 << 64)
