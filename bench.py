@@ -1267,6 +1267,8 @@ def main():
                    "l2": f"inputs larger than L2 (each step touches {int(sh['sequences_per_step'] * cfg.elems * 6 / 1e6)} MB of fresh HBM; no flush needed)",
                    "parallelism": f"dp{world} replicas, no collective"},
         "timed": head["timed"],
+        # step time x median sampled SM clock: compares runs taken at different clocks under the power cap
+        "sm_kcycles_per_step": (head["ms_per_step"] * head["clocks"]["sm_mhz"] if head["clocks"]["sm_mhz"] else None),
         "samples_per_s": head["samples_per_s"],
         "frac_of_measured_hbm": head["frac_of_measured_hbm"], "frac_of_8000_spec": head["frac_of_8000_spec"],
         "roofline": {"bound": "hbm", "kernel": "encode_kernel", "achieved": head["encode"]["achieved"], "peak": head["peak"], "unit": "GB/s",

@@ -267,7 +267,7 @@ int aq_dequant_grad(aq_handle* h, const void* packed, const float* scales, int64
 /*
  * 64-bit digest of the whole state, independent of summation order:
  *   sum_i mix(i, word_i) + sum_xi mix(2^40 + xi, seen[xi])   (mod 2^64),
- * word_i = the i-th little-endian 32-bit word of m, mix(i, w) = the splitmix64 output
+ * word_i = the i-th little-endian 64-bit word of m (four elements), mix(i, w) = the splitmix64 output
  * function applied to i*0x9E3779B97F4A7C15 + w.  Two handles fed the same id sequence
  * (the two sides of a boundary: in Algorithm 2 either network keeps its own copy of m)
  * must give the same digest.  Synchronises the stream; *out_host is host memory.

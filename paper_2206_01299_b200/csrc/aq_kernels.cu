@@ -498,14 +498,14 @@ __device__ __forceinline__ unsigned long long mix64(unsigned long long index, un
 }
 
 __global__ void __launch_bounds__(kThreads) checksum_kernel(const State st, unsigned long long* sum_out) {
-  const long long n_vec = st.n_samples * (long long)st.chunks;      // 16-byte pieces = 4 words each
+  const long long n_vec = st.n_samples * (long long)st.chunks;      // 16-byte pieces = two 64-bit words each
   const uint4* mv = reinterpret_cast<const uint4*>(st.m);
   const long long stride = (long long)gridDim.x * kThreads;
   unsigned long long acc = 0ull;
   for (long long v = (long long)blockIdx.x * kThreads + threadIdx.x; v < n_vec; v += stride) {
     const uint4 w = __ldcs(mv + v);
-    const unsigned long long i = (unsigned long long)v * 4ull;
-    acc += mix64(i, w.x) + mix64(i + 1, w.y) + mix64(i + 2, w.z) + mix64(i + 3, w.w);
+    const unsigned long long i = (unsigned long long)v * 2ull;
+    acc += mix64(i, ((unsigned long long)w.y << 32) | w.x) + mix64(i + 1, ((unsigned long long)w.w << 32) | w.z);
   }
   for (long long x = (long long)blockIdx.x * kThreads + threadIdx.x; x < st.n_samples; x += stride)
     acc += mix64((1ull << 40) + (unsigned long long)x, st.seen[x] != 0ull ? 1ull : 0ull);

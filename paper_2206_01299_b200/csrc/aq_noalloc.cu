@@ -57,8 +57,8 @@ __global__ void __launch_bounds__(aq::kThreads) digest_slabs_kernel(const uint4*
   unsigned long long acc = 0ull;
   for (long long v = v0 + threadIdx.x; v < v1; v += aq::kThreads) {
     const uint4 w = __ldcs(mv + v);
-    const unsigned long long i = (unsigned long long)v * 4ull;
-    acc += mix64(i, w.x) + mix64(i + 1, w.y) + mix64(i + 2, w.z) + mix64(i + 3, w.w);
+    const unsigned long long i = (unsigned long long)v * 2ull;           // two 64-bit words per piece
+    acc += mix64(i, ((unsigned long long)w.y << 32) | w.x) + mix64(i + 1, ((unsigned long long)w.w << 32) | w.z);
   }
   const unsigned long long t = cta_sum(acc, part);
   if (threadIdx.x == 0) slot[blockIdx.x] = t;
