@@ -555,8 +555,9 @@ void aqo_dequant_grad(const uint8_t* packed, const float* scales, int64_t n_elem
 // little-endian 64-bit words (word i = elements 4i .. 4i+3; a last word that
 // the array does not fill is completed with zeros -- the library's shapes,
 // multiples of 8 elements per sample, have none), plus the seen set.
-// (The digest is a requirement of this build, not of the paper: any fixed
-// mixer serves as long as both sides of a comparison use the same one.)
+// (The digest is a device for comparing two states, not a part of the paper's
+// method: any fixed mixer serves as long as both sides of a comparison use
+// the same one.)
 uint64_t aqo_state_checksum(void* h) {
   Side* S = (Side*)h;
   uint64_t sum = 0;
