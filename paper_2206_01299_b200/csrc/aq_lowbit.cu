@@ -99,10 +99,8 @@ __device__ __forceinline__ void lowbit_rows(const State& st, const EncodeArgs& e
       }
       unsigned long long codes = 0ull;
       if (SENDER) {
-        float af[8], d[8];
-        Conv<T>::unpack(av[i], af);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) d[j] = __fsub_rn(af[j], m_deq[j]);
+        float d[8];
+        Conv<T>::diff(av[i], m_deq, d);
         const float s = group_max_any(abs_max8(d), st.lanes_per_group);
         uint4 noise = make_uint4(0, 0, 0, 0);                // the message's rounding; the store's stays deterministic
         if constexpr (STOCH) noise = chunk_noise(ea.seed, ea.epoch, stream_id, (uint32_t)c);
