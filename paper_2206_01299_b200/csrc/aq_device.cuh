@@ -25,7 +25,35 @@ struct LaunchPlan {
   int rows_per_cta;        // rows of one sample that a CTA walks; grid = (ceil(rows / rows_per_cta), n_batch)
   unsigned share;          // what a CTA adds to the arrival counter ...
   unsigned first_share;    // ... and what CTA (0,0) adds, so that the grid adds kCallQuantum in all
+  // Decode launches are one-dimensional and may taper: CTAs [0, ctas1) walk samples [0, n1), gx1 CTAs of
+  // rows_per_cta rows per sample; the CTAs behind them walk the last samples, gx2 CTAs of tail_rows rows each.
+  unsigned ctas1, gx1, gx2;
+  int n1, tail_rows;
 };
+
+// Which sample of the call, and which of its rows, a CTA of a one-dimensional (tapered) grid walks.
+struct CtaRows {
+  int y;       // sample of the call
+  int x;       // the CTA's place among those of the sample
+  int rows;    // rows per CTA in this part of the grid
+};
+__device__ __forceinline__ CtaRows locate_cta(const LaunchPlan& plan) {
+  unsigned b = blockIdx.x;
+  CtaRows c;
+  if (b < plan.ctas1) {
+    const unsigned q = b / plan.gx1;
+    c.y = (int)q;
+    c.x = (int)(b - q * plan.gx1);
+    c.rows = plan.rows_per_cta;
+  } else {
+    b -= plan.ctas1;
+    const unsigned q = b / plan.gx2;
+    c.y = plan.n1 + (int)q;
+    c.x = (int)(b - q * plan.gx2);
+    c.rows = plan.tail_rows;
+  }
+  return c;
+}
 
 // ------------------------------------------------------------------ 16-bit types
 
@@ -472,10 +500,13 @@ struct BufferLists {
 // missing or not 16-byte aligned makes the sample kModeNothing (nothing read or written for it).
 // raw_at: which of the lists holds the raw message of a first visit (-1: none); a null entry
 // there means "no raw message for this sample".
+// cta_x: the CTA's place among those of its sample, where the grid is not (CTAs of a sample, samples).
 __device__ __forceinline__ Sample open_sample(const State& st, const LaunchPlan& plan,
                                               const int32_t* __restrict__ ids, int y, bool need_raw,
                                               bool have_raw, uint8_t* first_flags,
-                                              const BufferLists* lists = nullptr, int raw_at = -1) {
+                                              const BufferLists* lists = nullptr, int raw_at = -1,
+                                              int cta_x = -1) {
+  if (cta_x < 0) cta_x = (int)blockIdx.x;       // two-dimensional grid: x counts the CTAs of a sample
   __shared__ Sample s_sample;
   if (threadIdx.x < 32) {
     const int lane = threadIdx.x;
@@ -528,7 +559,7 @@ __device__ __forceinline__ Sample open_sample(const State& st, const LaunchPlan&
       s_sample.row = st.slot_ids ? (unsigned)y : (unsigned)id;
 #pragma unroll
       for (int k = 0; k < 4; ++k) s_sample.buf[k] = buf[k];
-      if (blockIdx.x == 0) {                     // once per sample and call
+      if (cta_x == 0) {                          // once per sample and call
         if (why) atomicOr(st.status, why);
         if (first_flags) first_flags[y] = (uint8_t)(mode == kModeFirst);
         if (mode == kModeFirst) st.seen[id] = call;

@@ -195,16 +195,17 @@ template <typename T, int BITS, bool LISTS>
 __global__ void __launch_bounds__(kThreads, decode_ctas_per_sm<BITS>()) decode_kernel(const State st, const DecodeArgs a, const LaunchPlan plan) {
   const int tid = threadIdx.x;
   const int lane = tid & 31;
-  const int y = blockIdx.y;                                       // sample of the call
+  const CtaRows cta = locate_cta(plan);
+  const int y = cta.y;                                            // sample of the call
   let_dependents_launch();
-  int r = blockIdx.x * plan.rows_per_cta;                         // this CTA's rows of the sample: [r, r_end)
-  const int r_end = min(st.rows, r + plan.rows_per_cta);
+  int r = cta.x * cta.rows;                                       // this CTA's rows of the sample: [r, r_end)
+  const int r_end = min(st.rows, r + cta.rows);
   // the CTA's rows of m(xi) are asked for while the previous kernel of the stream is still draining
   if (st.l2_prefetch && tid == 32) prefetch_rows_of_m<T>(st, a.ids, y, r * kThreads, min(st.chunks, r_end * kThreads));
   wait_for_predecessor();
   const BufferLists lists = {{a.packed_list(), a.scales_list(), a.raw_list(), a.out_list()}, {true, true, false, true}};
   const Sample sample = open_sample(st, plan, a.ids, y, true, a.raw != nullptr, a.first_flags, LISTS ? &lists : nullptr,
-                                    a.raw != nullptr ? 2 : -1);
+                                    a.raw != nullptr ? 2 : -1, cta.x);
   const int mode = sample.mode;
   const unsigned elems = (unsigned)st.elems;
   // the sample's buffers: at a fixed stride from the call's base pointers, or (list form) fetched with the sample
@@ -567,10 +568,12 @@ cudaError_t launch_quant16(int lanes16, const void* grad, long long pairs, uint8
 
 inline unsigned grid_x(long long chunks) { return (unsigned)((chunks + kChunksPerCta - 1) / kChunksPerCta); }
 
-template <typename K, typename Args>
-cudaError_t launch_rows(K kernel, const State& st, const Args& a, cudaStream_t s) {
-  if (a.n_batch <= 0) return cudaSuccess;
-  const long long total = (long long)a.n_batch * st.rows;
+// Rows per CTA and CTAs per sample of an encode / decode launch.
+struct RowSplit {
+  long long per, gx;
+};
+inline RowSplit split_rows(const State& st, int n_batch) {
+  const long long total = (long long)n_batch * st.rows;
   long long per = st.rows_per_cta;
   if (per <= 0) {
     // a small call gets the fewest rows per CTA that still put the whole grid on the multiprocessors at once
@@ -582,17 +585,65 @@ cudaError_t launch_rows(K kernel, const State& st, const Args& a, cudaStream_t s
   }
   if (per > st.rows) per = st.rows;
   long long gx = (st.rows + per - 1) / per;
-  if (gx * a.n_batch > (long long)kCallQuantum) {            // keep every CTA's share of the quantum >= 1
-    gx = (long long)kCallQuantum / a.n_batch;
+  if (gx * n_batch > (long long)kCallQuantum) {            // keep every CTA's share of the quantum >= 1
+    gx = (long long)kCallQuantum / n_batch;
     per = (st.rows + gx - 1) / gx;
     gx = (st.rows + per - 1) / per;
   }
-  const unsigned long long ctas = (unsigned long long)gx * (unsigned long long)a.n_batch;
-  LaunchPlan plan;
-  plan.rows_per_cta = (int)per;
+  return {per, gx};
+}
+
+inline void set_shares(LaunchPlan& plan, unsigned long long ctas) {
   plan.share = (unsigned)(kCallQuantum / ctas);
   plan.first_share = (unsigned)(kCallQuantum - (unsigned long long)plan.share * (ctas - 1ull));
-  return launch_overlapped(kernel, dim3((unsigned)gx, (unsigned)a.n_batch), s, st, a, plan);
+}
+
+// Grid (CTAs of a sample, samples).
+template <typename K, typename Args>
+cudaError_t launch_rows(K kernel, const State& st, const Args& a, cudaStream_t s) {
+  if (a.n_batch <= 0) return cudaSuccess;
+  const RowSplit sp = split_rows(st, a.n_batch);
+  LaunchPlan plan = {};
+  plan.rows_per_cta = (int)sp.per;
+  set_shares(plan, (unsigned long long)sp.gx * (unsigned long long)a.n_batch);
+  return launch_overlapped(kernel, dim3((unsigned)sp.gx, (unsigned)a.n_batch), s, st, a, plan);
+}
+
+// One-dimensional grid in the same order (the CTAs of sample 0, then those of sample 1, ...) whose end tapers:
+// when a grid runs out of CTAs, every multiprocessor still has to finish the ones it holds, and how long that
+// takes is set by the rows a CTA walks.  On a call of several waves of full-size CTAs the last samples -- about
+// one wave of the resident CTA slots at half the rows -- are therefore walked by CTAs of half the rows.
+template <typename K, typename Args>
+cudaError_t launch_rows_tapered(K kernel, const State& st, const Args& a, cudaStream_t s) {
+  if (a.n_batch <= 0) return cudaSuccess;
+  const RowSplit sp = split_rows(st, a.n_batch);
+  const long long slots = (long long)st.sms * 6;
+  long long tail_rows = sp.per, gx2 = sp.gx;
+  int n2 = 0;
+  if (st.rows_per_cta <= 0 && sp.per == kRowsPerCta && sp.gx * a.n_batch >= 2 * slots) {
+    tail_rows = sp.per / 2;
+    gx2 = (st.rows + tail_rows - 1) / tail_rows;
+    n2 = (int)(slots * tail_rows / st.rows);
+    n2 = n2 < 1 ? 1 : n2;
+    if (n2 > a.n_batch / 2) n2 = a.n_batch / 2;
+  }
+  const int n1 = a.n_batch - n2;
+  const unsigned long long ctas = (unsigned long long)sp.gx * n1 + (unsigned long long)gx2 * n2;
+  LaunchPlan plan = {};
+  plan.rows_per_cta = (int)sp.per;
+  plan.ctas1 = (unsigned)(sp.gx * n1);
+  plan.gx1 = (unsigned)sp.gx;
+  plan.gx2 = (unsigned)gx2;
+  plan.n1 = n1;
+  plan.tail_rows = (int)tail_rows;
+  if (ctas > kCallQuantum) {                               // no taper: split_rows has bounded gx * n_batch
+    plan.ctas1 = (unsigned)(sp.gx * a.n_batch);
+    plan.n1 = a.n_batch;
+    set_shares(plan, plan.ctas1);
+    return launch_overlapped(kernel, dim3(plan.ctas1), s, st, a, plan);
+  }
+  set_shares(plan, ctas);
+  return launch_overlapped(kernel, dim3((unsigned)ctas), s, st, a, plan);
 }
 
 }  // namespace
@@ -614,7 +665,7 @@ cudaError_t launch_encode(int dtype, int bits, const State& st, const EncodeArgs
 }
 
 cudaError_t launch_decode(int dtype, int bits, const State& st, const DecodeArgs& a, cudaStream_t s) {
-#define AQ_CALL(T, B) return a.lists ? launch_rows(decode_kernel<T, B, true>, st, a, s) : launch_rows(decode_kernel<T, B, false>, st, a, s)
+#define AQ_CALL(T, B) return a.lists ? launch_rows_tapered(decode_kernel<T, B, true>, st, a, s) : launch_rows_tapered(decode_kernel<T, B, false>, st, a, s)
   AQ_DISPATCH(dtype, bits, AQ_CALL)
 #undef AQ_CALL
   return cudaErrorInvalidValue;

@@ -195,7 +195,7 @@ cudaError_t launch_lowbit(K kernel, const State& st, const EncodeArgs& ea, const
     gx = (st.rows + per - 1) / per;
   }
   const unsigned long long ctas = (unsigned long long)gx * (unsigned long long)n_batch;
-  LaunchPlan plan;
+  LaunchPlan plan = {};
   plan.rows_per_cta = (int)per;
   plan.share = (unsigned)(kCallQuantum / ctas);
   plan.first_share = (unsigned)(kCallQuantum - (unsigned long long)plan.share * (ctas - 1ull));

@@ -125,6 +125,16 @@ def test_every_bit_width_on_ragged_shapes(dtype, bits):
     run_boundary(cfg)
 
 
+@pytest.mark.parametrize("dtype,bits", [("fp16", 3), ("bf16", 4)])
+def test_call_large_enough_for_the_tapered_end_of_the_decode_grid(dtype, bits):
+    """128 samples of 57 rows (the last one ragged) in one call: more than two waves of four-row CTAs on
+    148 multiprocessors, so the receiver's grid walks its last samples with two-row CTAs; 57 is odd, so
+    either part of the grid ends each sample with a one-row CTA.  Every element is compared."""
+    cfg = synth.Boundary("taper", 128, 128, 57, 2040, dtype, bits, 8, 3, "outlier", 0.2, seed=70 + bits)
+    assert cfg.elems // 8 == 57 * 255 and (cfg.elems // 8) % 256 != 0
+    run_boundary(cfg)
+
+
 @pytest.mark.parametrize("group", [16, 32, 256])
 def test_other_group_sizes(group):
     cfg = synth.Boundary("groups", 4, 2, 5, 1024, "fp16", 4, group, 3, "outlier", 0.1, seed=group)
