@@ -86,7 +86,8 @@ enum {
                             independent random numbers need different values (for activations the epoch
                             or step number; for gradients any number unique to the call); default 0 */
   AQ_ROWS_PER_CTA = 6,   /* tuning: rows (256 chunks = 2048 elements each) that one CTA of aq_encode /
-                            aq_decode walks; 0 (default) = chosen from the size of the call (1..4) */
+                            aq_decode walks; 0 (default) = chosen from the size of the call (1..4; on
+                            large calls the CTAs that walk the last samples of aq_decode take half) */
   AQ_L2_PREFETCH = 10,   /* tuning: 1 (default for stores in device memory) = every CTA of aq_encode /
                             aq_decode asks for its rows of act and m, and every CTA of aq_quant_grad for its
                             piece of the gradient, to be brought into L2 ahead of its loads (bulk-prefetch
