@@ -5,7 +5,9 @@ between: bit width, type, group size, sequence length, hidden size, samples per 
 recipe are drawn from a fixed seed, so that a failure names a case that can be run again.  Three
 families: small calls (ragged rows, single chunks, calls that leave multiprocessors idle), calls
 around the size from which the receiver's grid ends in smaller CTAs (a few samples more or fewer than
-two waves of full-size CTAs, odd and ragged row counts), and gradients of random length."""
+two waves of full-size CTAs, odd and ragged row counts), and gradients of random length; the small shapes
+also go through the optional modes (stochastic rounding, low-precision and binary32 stores, the store in
+host memory with and without prefetch)."""
 import random
 
 import numpy as np
@@ -16,6 +18,7 @@ import oracle
 import paper_2206_01299_b200 as aq
 from codec_harness import DT, Guarded, bits16, check_guards, run_boundary
 from fixtures import synth
+from test_gpu_lowbit import run_lowbit
 
 pytestmark = pytest.mark.gpu
 
@@ -95,3 +98,19 @@ def test_random_gradient_lengths(i):
         assert aq.aq_status(h) == 0
     finally:
         aq.aq_destroy(h)
+
+
+@pytest.mark.parametrize("i", range(24))
+def test_small_random_shapes_through_the_optional_modes(i):
+    rng = random.Random(9900 + i)
+    cfg = _small_case(100 + i)
+    mode = i % 4
+    if mode == 0:                                    # unbiased stochastic rounding of the messages
+        run_boundary(cfg, stochastic_seed=rng.getrandbits(40))
+    elif mode == 1:                                  # previous messages kept in 2, 4, 8 bits or binary32
+        run_lowbit(cfg, rng.choice((2, 4, 8, 32)), stochastic_seed=rng.choice((None, 77)))
+    elif mode == 2:                                  # m in page-locked host memory; some calls prefetched
+        pattern = rng.getrandbits(16) | 1
+        run_boundary(cfg, hosted=True, prefetch=lambda k: (pattern >> (k % 16)) & 1 == 1)
+    else:                                            # low-precision store in host memory
+        run_lowbit(cfg, rng.choice((2, 4, 8)), hosted=True, prefetch=lambda k: k % 2 == 0)
