@@ -25,6 +25,9 @@ namespace {
 
 // ------------------------------------------------------------------ encode (sender)
 
+// rows that the plain-copy paths (first visit of a sample) move per loop iteration
+constexpr int kCopyRows = 4;
+
 // Delta visit of n rows starting at chunk c0 of one sample.  FULL: n == kRowsPerIter and every
 // chunk is inside the sample, so no bounds are checked.
 template <typename T, int BITS, int LPG, bool STOCH, bool FULL>
@@ -134,15 +137,28 @@ __global__ void __launch_bounds__(kThreads, STOCH ? (BITS <= 4 ? 6 : 4) : encode
     // first visit: the activation itself becomes m(xi); skipped sample: nothing is stored.
     // Either way the sample's codes and scales are zero.
     T* m = (mode == kModeFirst) ? reinterpret_cast<T*>(st.m) + (unsigned long long)sample.row * elems : nullptr;
-    for (; r < r_end; ++r) {
-      const int c = r * kThreads + tid;
-      const bool active = c < st.chunks;
-      if (active) {
-        if (m) st_stream(m + (size_t)c * kChunk, ld_stream(act + (size_t)c * kChunk));
-        if ((lane & (st.lanes_per_group - 1)) == 0) scales[c >> st.lg_shift] = 0.0f;
+    // kCopyRows rows at a time, their loads in flight together before the first store
+    for (; r < r_end; r += kCopyRows) {
+      uint4 v[kCopyRows];
+#pragma unroll
+      for (int i = 0; i < kCopyRows; ++i) {
+        const int c = (r + i) * kThreads + tid;
+        v[i] = make_uint4(0, 0, 0, 0);
+        if (m && r + i < r_end && c < st.chunks) v[i] = ld_stream(act + (size_t)c * kChunk);
       }
-      const bool warp_words = words_ok && (c - lane + 32 <= st.chunks);
-      store_codes<BITS>(stream, c, lane, active, warp_words, 0ull);
+#pragma unroll
+      for (int i = 0; i < kCopyRows; ++i) {
+        if (r + i < r_end) {                          // uniform over the CTA
+          const int c = (r + i) * kThreads + tid;
+          const bool active = c < st.chunks;
+          if (active) {
+            if (m) st_stream(m + (size_t)c * kChunk, v[i]);
+            if ((lane & (st.lanes_per_group - 1)) == 0) scales[c >> st.lg_shift] = 0.0f;
+          }
+          const bool warp_words = words_ok && (c - lane + 32 <= st.chunks);
+          store_codes<BITS>(stream, c, lane, active, warp_words, 0ull);
+        }
+      }
     }
   }
 }
@@ -234,15 +250,21 @@ __global__ void __launch_bounds__(kThreads, decode_ctas_per_sm<BITS>()) decode_k
     // first visit: the raw message becomes m(xi) and the activation; skipped sample: zeros out.
     const bool first = mode == kModeFirst;
     T* m = first ? reinterpret_cast<T*>(st.m) + (unsigned long long)sample.row * elems : nullptr;
-    for (; r < r_end; ++r) {
-      const int c = r * kThreads + tid;
-      if (c < st.chunks) {
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (first) {
-          v = ld_stream(raw + (size_t)c * kChunk);
-          st_stream(m + (size_t)c * kChunk, v);
+    for (; r < r_end; r += kCopyRows) {
+      uint4 v[kCopyRows];
+#pragma unroll
+      for (int i = 0; i < kCopyRows; ++i) {
+        const int c = (r + i) * kThreads + tid;
+        v[i] = make_uint4(0, 0, 0, 0);
+        if (first && r + i < r_end && c < st.chunks) v[i] = ld_stream(raw + (size_t)c * kChunk);
+      }
+#pragma unroll
+      for (int i = 0; i < kCopyRows; ++i) {
+        const int c = (r + i) * kThreads + tid;
+        if (r + i < r_end && c < st.chunks) {
+          if (first) st_stream(m + (size_t)c * kChunk, v[i]);
+          st_stream(out + (size_t)c * kChunk, v[i]);
         }
-        st_stream(out + (size_t)c * kChunk, v);
       }
     }
   }
