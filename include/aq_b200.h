@@ -128,11 +128,15 @@ enum {
  * Initialisation step of Algorithm 1: allocates m (n_samples*seq*hidden*2 bytes of device
  * memory on the current device) filled with zeros, and an empty "seen before"
  * set.  bits in 1..8 is b of the forward quantizer; group (a multiple of 8, so that a group
- * is a whole number of 16-byte pieces and group*bits/8 whole bytes) must divide hidden.  Kernels
- * exist for groups of 8, 16, 32, 64, 128 and 256 elements -- the lanes that share a group's
- * maximum are a power of two inside one warp; any other multiple of 8 (24, 40, 48, 96 ...) is a
- * valid setting of the quantizer that this build refuses with AQ_EUNSUPPORTED.  Returns NULL on
- * failure; aq_last_error(NULL) and aq_last_error_code(NULL) say why.
+ * is a whole number of 16-byte pieces and group*bits/8 whole bytes) must divide hidden, up to
+ * group == hidden (one step per token).  The tuned kernels are those for groups of 8, 16, 32, 64, 128
+ * and 256 elements -- the lanes that share a group's maximum are a power of two inside one warp;
+ * any other multiple of 8 (24, 40, 48, 96, 320, 512 ...) runs on plainer kernels of its own: same
+ * results by the same definition, not measured.  Those group sizes are offered by aq_create and
+ * aq_create_hosted (base-pointer and host-buffer forms of the calls, aq_quant_grad / aq_dequant_grad,
+ * either rounding mode); the low-precision and binary32 stores and the list forms answer
+ * AQ_EUNSUPPORTED for them.  Returns NULL on failure; aq_last_error(NULL) and aq_last_error_code(NULL)
+ * say why.
  */
 aq_handle* aq_create(int64_t n_samples, int seq, int hidden, int bits, int group);
 
@@ -189,7 +193,8 @@ int aq_prefetch(aq_handle* h, const int32_t* sample_ids_host, int n);
  * applies to the message (Q_b) only: the store's own re-quantization always takes the interval
  * number, so that the receiver, which never learns the rounding mode, ends with the same store.
  * aq_state_checksum_noalloc answers AQ_EUNSUPPORTED on such a handle.  aq_state_checksum covers
- * the code bytes (as 32-bit words), then the steps, then the seen-set.
+ * the code bytes (as 32-bit words), then the steps, then the seen-set.  group must be 8, 16, 32, 64,
+ * 128 or 256 (AQ_EUNSUPPORTED for the other multiples of 8).
  */
 aq_handle* aq_create_lowbit(int64_t n_samples, int seq, int hidden, int bits, int group, int m_bits);
 
@@ -245,8 +250,8 @@ int aq_decode(aq_handle* h, const void* packed, const float* scales, const int32
  * AQ_RAW_LIST.  Every pointer must be 16-byte aligned; the kernels check (the host cannot see the
  * arrays): a null or misaligned entry skips that sample altogether and sets AQ_ST_BAD_PTR.  Same
  * kernels, same results as the base-pointer forms on the same samples.  The arrays are read when the
- * kernel runs and must stay unchanged until then.  16-bit stores only (aq_create, aq_create_hosted);
- * AQ_EUNSUPPORTED otherwise.
+ * kernel runs and must stay unchanged until then.  16-bit stores only (aq_create, aq_create_hosted),
+ * groups of 8, 16, 32, 64, 128 or 256 elements; AQ_EUNSUPPORTED otherwise.
  */
 int aq_encode_list(aq_handle* h, const void* const* act_list, const int32_t* sample_ids,
                    void* const* packed_list, float* const* scales_list);

@@ -5,7 +5,7 @@ import sys
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
-SOURCES = [os.path.join(CSRC, f) for f in ("aq_api.cu", "aq_kernels.cu", "aq_lowbit.cu", "aq_noalloc.cu")]
+SOURCES = [os.path.join(CSRC, f) for f in ("aq_api.cu", "aq_kernels.cu", "aq_lowbit.cu", "aq_anygroup.cu", "aq_noalloc.cu")]
 HEADERS = [os.path.join(CSRC, "aq_internal.h"), os.path.join(CSRC, "aq_device.cuh"),
            os.path.join(os.path.dirname(HERE), "include", "aq_b200.h")]
 OBJ_DIR = os.path.join(HERE, "_build")

@@ -270,10 +270,10 @@ static aq_handle* create_handle(int64_t n_samples, int seq, int hidden, int bits
   if (bits < 1 || bits > 8) { fail(nullptr, AQ_EINVAL, "bits must be in 1..8 (got %d)", bits); return nullptr; }
   if (group <= 0 || group % 8) { fail(nullptr, AQ_EINVAL, "group must be a positive multiple of 8 (got %d)", group); return nullptr; }
   if (hidden % group) { fail(nullptr, AQ_EINVAL, "group %d does not divide hidden %d", group, hidden); return nullptr; }
-  if (!lanes) {
-    // a valid quantizer setting that no kernel is built for: the lanes that share a group's maximum must be
-    // a power of two within one warp
-    fail(nullptr, AQ_EUNSUPPORTED, "group %d: this build has kernels for groups of 8, 16, 32, 64, 128 and 256 elements only", group);
+  if (!lanes && m_bits) {
+    // a valid quantizer setting that the kernels of the low-precision and binary32 stores are not built for:
+    // there the lanes that share a group's maximum must be a power of two within one warp
+    fail(nullptr, AQ_EUNSUPPORTED, "group %d: the low-precision and binary32 stores have kernels for groups of 8, 16, 32, 64, 128 and 256 elements only", group);
     return nullptr;
   }
   aq_handle* h = new (std::nothrow) aq_handle();
@@ -286,8 +286,9 @@ static aq_handle* create_handle(int64_t n_samples, int seq, int hidden, int bits
   st.rows = (st.chunks + aq::kThreads - 1) / aq::kThreads;
   st.packed_bytes = st.elems * bits / 8;
   st.groups = st.elems / group;
-  st.lanes_per_group = lanes;
-  st.lg_shift = __builtin_ctz((unsigned)lanes);
+  // any other multiple of 8 runs on the kernels of aq_anygroup.cu (lg_shift < 0 marks it)
+  st.lanes_per_group = lanes ? lanes : group / aq::kChunk;
+  st.lg_shift = lanes ? __builtin_ctz((unsigned)lanes) : -1;
   st.l2_prefetch = hosted ? 0 : h->l2_prefetch;     // rows in mapped host memory are not brought into L2
   cudaError_t e = cudaGetDevice(&h->device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&st.sms, cudaDevAttrMultiProcessorCount, h->device);
@@ -424,25 +425,30 @@ int aq_configure(aq_handle* h, int key, int64_t value) {
   }
 }
 
+// The kernels of a call: the low-precision stores have their own, and so have the group sizes whose lanes
+// are not a power of two within a warp.
+static cudaError_t run_encode(aq_handle* h, const aq::State& st, const aq::EncodeArgs& a) {
+  if (st.m_bits) return aq::launch_encode_lowbit(h->dtype, h->bits, st, a, h->stream);
+  if (st.lg_shift < 0) return aq::launch_encode_anygroup(h->dtype, h->bits, st, a, h->stream);
+  return aq::launch_encode(h->dtype, h->bits, st, a, h->stream);
+}
+static cudaError_t run_decode(aq_handle* h, const aq::State& st, const aq::DecodeArgs& a) {
+  if (st.m_bits) return aq::launch_decode_lowbit(h->dtype, h->bits, st, a, h->stream);
+  if (st.lg_shift < 0) return aq::launch_decode_anygroup(h->dtype, h->bits, st, a, h->stream);
+  return aq::launch_decode(h->dtype, h->bits, st, a, h->stream);
+}
+
 static int launch_encode_call(aq_handle* h, const aq::EncodeArgs& a) {
   AQ_CUDA(h, settle(h));
   h->inplace_since_fetch = true;
-  if (h->st.m_bits) {
-    AQ_CUDA(h, aq::launch_encode_lowbit(h->dtype, h->bits, h->st, a, h->stream));
-    return AQ_OK;
-  }
-  AQ_CUDA(h, aq::launch_encode(h->dtype, h->bits, h->st, a, h->stream));
+  AQ_CUDA(h, run_encode(h, h->st, a));
   return AQ_OK;
 }
 
 static int launch_decode_call(aq_handle* h, const aq::DecodeArgs& a) {
   AQ_CUDA(h, settle(h));
   h->inplace_since_fetch = true;
-  if (h->st.m_bits) {
-    AQ_CUDA(h, aq::launch_decode_lowbit(h->dtype, h->bits, h->st, a, h->stream));
-    return AQ_OK;
-  }
-  AQ_CUDA(h, aq::launch_decode(h->dtype, h->bits, h->st, a, h->stream));
+  AQ_CUDA(h, run_decode(h, h->st, a));
   return AQ_OK;
 }
 
@@ -454,14 +460,13 @@ static int encode_call(aq_handle* h, const void* act, const int32_t* sample_ids,
   if (!lists && (!aligned16(act) || !aligned16(packed) || !aligned16(scales)))
     return fail(h, AQ_EINVAL, "%s: act, packed and scales must be 16-byte aligned", who);
   if (lists && h->st.m_bits) return fail(h, AQ_EUNSUPPORTED, "%s: the list form is built for the 16-bit store only", who);
+  if (lists && h->st.lg_shift < 0)
+    return fail(h, AQ_EUNSUPPORTED, "%s: the list form is built for groups of 8, 16, 32, 64, 128 and 256 elements only", who);
   DeviceGuard g(h->device);
   aq::EncodeArgs a{act, sample_ids, static_cast<uint8_t*>(packed), scales, h->first_flags, h->n_batch,
                    h->rounding == AQ_ROUND_STOCHASTIC, h->seed, h->epoch, lists};
   if (h->pending_stage >= 0)
-    return run_staged(h, [&](const aq::State& st) {
-      return h->st.m_bits ? aq::launch_encode_lowbit(h->dtype, h->bits, st, a, h->stream)
-                          : aq::launch_encode(h->dtype, h->bits, st, a, h->stream);
-    });
+    return run_staged(h, [&](const aq::State& st) { return run_encode(h, st, a); });
   return launch_encode_call(h, a);
 }
 
@@ -483,14 +488,13 @@ static int decode_call(aq_handle* h, const void* packed, const float* scales, co
   if (!lists && (!aligned16(packed) || !aligned16(scales) || !aligned16(out)))
     return fail(h, AQ_EINVAL, "%s: packed, scales and out must be 16-byte aligned", who);
   if (lists && h->st.m_bits) return fail(h, AQ_EUNSUPPORTED, "%s: the list form is built for the 16-bit store only", who);
+  if (lists && h->st.lg_shift < 0)
+    return fail(h, AQ_EUNSUPPORTED, "%s: the list form is built for groups of 8, 16, 32, 64, 128 and 256 elements only", who);
   DeviceGuard g(h->device);
   aq::DecodeArgs a{static_cast<const uint8_t*>(packed), scales, lists ? static_cast<const void*>(h->raw_list) : h->raw, sample_ids,
                    out, h->first_flags, h->n_batch, lists};
   if (h->pending_stage >= 0)
-    return run_staged(h, [&](const aq::State& st) {
-      return h->st.m_bits ? aq::launch_decode_lowbit(h->dtype, h->bits, st, a, h->stream)
-                          : aq::launch_decode(h->dtype, h->bits, st, a, h->stream);
-    });
+    return run_staged(h, [&](const aq::State& st) { return run_decode(h, st, a); });
   return launch_decode_call(h, a);
 }
 
@@ -521,6 +525,11 @@ int aq_quant_grad(aq_handle* h, const void* grad, int64_t n_elems, int bits, voi
   const bool stochastic = h->rounding == AQ_ROUND_STOCHASTIC;
   if (stochastic && n_elems / aq::kChunk > 0xFFFFFFFFll)
     return fail(h, AQ_EINVAL, "aq_quant_grad: stochastic rounding numbers chunks with 32 bits (n_elems < 2^35)");
+  if (h->st.lg_shift < 0) {
+    AQ_CUDA(h, aq::launch_quant_grad_anygroup(h->dtype, bits, h->st.lanes_per_group, grad, n_elems, static_cast<uint8_t*>(packed),
+                                              scales, stochastic, h->seed, h->epoch, h->stream));
+    return AQ_OK;
+  }
   AQ_CUDA(h, aq::launch_quant_grad(h->dtype, bits, h->st.lanes_per_group, grad, n_elems,
                                    static_cast<uint8_t*>(packed), scales, stochastic, h->seed, h->epoch, h->l2_prefetch,
                                    h->stream));
@@ -531,6 +540,11 @@ int aq_dequant_grad(aq_handle* h, const void* packed, const float* scales, int64
   const int rc = check_grad_args(h, packed, scales, out, n_elems, bits);
   if (rc != AQ_OK || n_elems == 0) return rc;
   DeviceGuard g(h->device);
+  if (h->st.lg_shift < 0) {
+    AQ_CUDA(h, aq::launch_dequant_grad_anygroup(h->dtype, bits, h->st.lanes_per_group, static_cast<const uint8_t*>(packed), scales,
+                                                n_elems, out, h->stream));
+    return AQ_OK;
+  }
   AQ_CUDA(h, aq::launch_dequant_grad(h->dtype, bits, h->st.lanes_per_group, static_cast<const uint8_t*>(packed),
                                      scales, n_elems, out, h->stream));
   return AQ_OK;

@@ -35,8 +35,8 @@ struct State {
   long long groups;               // per sample
   int chunks;                     // elems / 8
   int rows;                       // ceil(chunks / kThreads): rows per sample
-  int lanes_per_group;            // group / 8, a power of two <= 32
-  int lg_shift;                   // log2(lanes_per_group)
+  int lanes_per_group;            // group / 8: a power of two <= 32 for the kernels of aq_kernels.cu and aq_lowbit.cu
+  int lg_shift;                   // log2(lanes_per_group); -1: any other lane count (kernels of aq_anygroup.cu)
   int sms;                        // multiprocessors of the handle's device
   int rows_per_cta;               // 0 = chosen by the launch layer (default); > 0 = fixed rows per CTA
   int l2_prefetch;                // 1: encode / decode ask for a CTA's rows to be brought into L2 ahead of its loads
@@ -85,6 +85,14 @@ cudaError_t launch_quant_grad(int dtype, int bits, int lanes_per_group, const vo
                               unsigned long long seed, unsigned long long epoch, int l2_prefetch, cudaStream_t s);
 cudaError_t launch_dequant_grad(int dtype, int bits, int lanes_per_group, const uint8_t* packed,
                                 const float* scales, long long n_elems, void* out, cudaStream_t s);
+// The same four for groups whose lane count is not a power of two up to 32 (aq_anygroup.cu; 16-bit store, base-pointer form).
+cudaError_t launch_encode_anygroup(int dtype, int bits, const State& st, const EncodeArgs& a, cudaStream_t s);
+cudaError_t launch_decode_anygroup(int dtype, int bits, const State& st, const DecodeArgs& a, cudaStream_t s);
+cudaError_t launch_quant_grad_anygroup(int dtype, int bits, int lanes_per_group, const void* grad, long long n_elems,
+                                       uint8_t* packed, float* scales, bool stochastic, unsigned long long seed,
+                                       unsigned long long epoch, cudaStream_t s);
+cudaError_t launch_dequant_grad_anygroup(int dtype, int bits, int lanes_per_group, const uint8_t* packed, const float* scales,
+                                         long long n_elems, void* out, cudaStream_t s);
 // Rows of `row_bytes` bytes moved by one kernel (in 16-, 4- or 1-byte pieces, as the size and the bases allow): gather: dst row y <- src row
 // ids[y]; scatter: dst row ids[y] <- src row y; entries with ids[y] < 0 are left out.
 cudaError_t launch_copy_rows(const void* src, void* dst, const int32_t* ids, int n, long long row_bytes, bool gather,

@@ -210,7 +210,7 @@ def test_host_side_argument_errors():
     with pytest.raises(aq.AqError):
         aq.aq_create(4, 2, 100, 4, 64)          # group does not divide hidden
     with pytest.raises(aq.AqError) as e:
-        aq.aq_create(4, 2, 96, 4, 24)           # a valid group that no kernel is built for
+        aq.aq_create_lowbit(4, 2, 96, 4, 24, 8)  # a valid group that the low-precision store has no kernel for
     assert e.value.code == aq.AQ_EUNSUPPORTED and "24" in str(e.value)
     with pytest.raises(aq.AqError) as e:
         aq.aq_create(4, 2, 96, 4, 12)           # not a whole number of 16-byte pieces
