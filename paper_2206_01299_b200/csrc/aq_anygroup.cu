@@ -224,9 +224,10 @@ __global__ void __launch_bounds__(kThreads) dequant_grad_anygroup_kernel(const u
 template <typename K, typename Args, typename... Extra>
 cudaError_t launch_per_sample(K kernel, const State& st, const Args& a, long long per_cta, cudaStream_t s, Extra... extra) {
   if (a.n_batch <= 0) return cudaSuccess;
+  // every CTA's share of the call quantum must be at least 1: very large calls get longer CTAs
+  while ((st.groups + per_cta - 1) / per_cta * a.n_batch > (long long)kCallQuantum) per_cta *= 2;
   const long long gx = (st.groups + per_cta - 1) / per_cta;
   const unsigned long long ctas = (unsigned long long)gx * (unsigned long long)a.n_batch;
-  if (ctas > kCallQuantum || gx > 0x7FFFFFFFll) return cudaErrorInvalidConfiguration;
   LaunchPlan plan = {};
   plan.rows_per_cta = 0;
   plan.share = (unsigned)(kCallQuantum / ctas);
