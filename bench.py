@@ -50,7 +50,7 @@ FALLBACK_HBM_GBS = 6650.0
 # per element, by workload; reported as roofline.traffic only while the kernel sources still hash to the
 # value recorded with the capture (`python bench.py --kernel-hash` prints the current one).
 NCU_TRAFFIC = {
-    "gpt2": {"kernel_hash": "50563dbbfa9c6103", "encode_bytes_per_element": (209778176 + 78859264) / 52428800,
+    "gpt2": {"kernel_hash": "cd123e3688cfb3ef", "encode_bytes_per_element": (209772800 + 77900544) / 52428800,
              "capture": "ncu --set full, encode_kernel<__half,4,8,0>, one launch of 32 sequences on the 128-id case"},
 }
 

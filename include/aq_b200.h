@@ -133,9 +133,8 @@ enum {
  * and 256 elements -- the lanes that share a group's maximum are a power of two inside one warp;
  * any other multiple of 8 (24, 40, 48, 96, 320, 512 ...) runs on plainer kernels of its own: same
  * results by the same definition, at roughly 0.6 of the rate.  Those group sizes are offered by aq_create and
- * aq_create_hosted (base-pointer and host-buffer forms of the calls, aq_quant_grad / aq_dequant_grad,
- * either rounding mode); the low-precision and binary32 stores and the list forms answer
- * AQ_EUNSUPPORTED for them.  Returns NULL on failure; aq_last_error(NULL) and aq_last_error_code(NULL)
+ * aq_create_hosted (every form of the calls, aq_quant_grad / aq_dequant_grad, either rounding mode);
+ * the low-precision and binary32 stores answer AQ_EUNSUPPORTED for them.  Returns NULL on failure; aq_last_error(NULL) and aq_last_error_code(NULL)
  * say why.
  */
 aq_handle* aq_create(int64_t n_samples, int seq, int hidden, int bits, int group);
@@ -250,8 +249,8 @@ int aq_decode(aq_handle* h, const void* packed, const float* scales, const int32
  * AQ_RAW_LIST.  Every pointer must be 16-byte aligned; the kernels check (the host cannot see the
  * arrays): a null or misaligned entry skips that sample altogether and sets AQ_ST_BAD_PTR.  Same
  * kernels, same results as the base-pointer forms on the same samples.  The arrays are read when the
- * kernel runs and must stay unchanged until then.  16-bit stores only (aq_create, aq_create_hosted),
- * groups of 8, 16, 32, 64, 128 or 256 elements; AQ_EUNSUPPORTED otherwise.
+ * kernel runs and must stay unchanged until then.  16-bit stores only (aq_create, aq_create_hosted);
+ * AQ_EUNSUPPORTED otherwise.
  */
 int aq_encode_list(aq_handle* h, const void* const* act_list, const int32_t* sample_ids,
                    void* const* packed_list, float* const* scales_list);

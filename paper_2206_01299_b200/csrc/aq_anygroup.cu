@@ -128,11 +128,19 @@ __global__ void __launch_bounds__(kThreads) encode_anygroup_kernel(const State s
                                                                    const Tiling tl, const long long per_cta) {
   const int y = blockIdx.y;
   overlap_with_neighbours();
-  const Sample sample = open_sample(st, plan, a.ids, y, false, false, a.first_flags);
+  const BufferLists lists = {{a.act_list(), a.packed_list(), a.scales_list(), nullptr}, {true, true, true, false}};
+  const Sample sample = open_sample(st, plan, a.ids, y, false, false, a.first_flags, a.lists ? &lists : nullptr);
   const unsigned long long elems = (unsigned long long)st.elems;
+  // the sample's buffers: at a fixed stride from the call's base pointers, or (list form) fetched with the sample
   const T* act = reinterpret_cast<const T*>(a.act) + (unsigned long long)(unsigned)y * elems;
   uint8_t* stream = a.packed + (unsigned long long)(unsigned)y * (unsigned long long)st.packed_bytes;
   float* scales = a.scales + (unsigned long long)(unsigned)y * (unsigned long long)st.groups;
+  if (a.lists) {
+    if (sample.mode == kModeNothing) return;
+    act = static_cast<const T*>(sample.buf[0]);
+    stream = static_cast<uint8_t*>(const_cast<void*>(sample.buf[1]));
+    scales = static_cast<float*>(const_cast<void*>(sample.buf[2]));
+  }
   const long long g_lo = (long long)blockIdx.x * per_cta;
   const long long g_hi = g_lo + per_cta < st.groups ? g_lo + per_cta : st.groups;
   if (sample.mode == kModeDelta) {
@@ -157,11 +165,21 @@ __global__ void __launch_bounds__(kThreads) decode_anygroup_kernel(const State s
   const int y = blockIdx.y;
   const int lane = threadIdx.x & 31;
   overlap_with_neighbours();
-  const Sample sample = open_sample(st, plan, a.ids, y, true, a.raw != nullptr, a.first_flags);
+  const BufferLists lists = {{a.packed_list(), a.scales_list(), a.raw_list(), a.out_list()}, {true, true, false, true}};
+  const Sample sample = open_sample(st, plan, a.ids, y, true, a.raw != nullptr, a.first_flags, a.lists ? &lists : nullptr,
+                                    a.raw != nullptr ? 2 : -1);
   const unsigned long long elems = (unsigned long long)st.elems;
   T* out = reinterpret_cast<T*>(a.out) + (unsigned long long)(unsigned)y * elems;
   const uint8_t* stream = a.packed + (unsigned long long)(unsigned)y * (unsigned long long)st.packed_bytes;
   const float* scales = a.scales + (unsigned long long)(unsigned)y * (unsigned long long)st.groups;
+  const T* raw = a.raw ? reinterpret_cast<const T*>(a.raw) + (unsigned long long)(unsigned)y * elems : nullptr;
+  if (a.lists) {
+    if (sample.mode == kModeNothing) return;
+    stream = static_cast<const uint8_t*>(sample.buf[0]);
+    scales = static_cast<const float*>(sample.buf[1]);
+    raw = static_cast<const T*>(sample.buf[2]);
+    out = static_cast<T*>(const_cast<void*>(sample.buf[3]));
+  }
   const long long g_lo = (long long)blockIdx.x * per_cta;
   const long long g_hi = g_lo + per_cta < st.groups ? g_lo + per_cta : st.groups;
   const long long c_lo = g_lo * lanes_per_group, c_hi = g_hi * lanes_per_group;
@@ -184,7 +202,6 @@ __global__ void __launch_bounds__(kThreads) decode_anygroup_kernel(const State s
     // first visit: the raw message becomes m(xi) and the activation; skipped sample: zeros out
     const bool first = sample.mode == kModeFirst;
     T* m = first ? reinterpret_cast<T*>(st.m) + (unsigned long long)sample.row * elems : nullptr;
-    const T* raw = a.raw ? reinterpret_cast<const T*>(a.raw) + (unsigned long long)(unsigned)y * elems : nullptr;
     for (long long c = c_lo + threadIdx.x; c < c_hi; c += kThreads) {
       uint4 v = make_uint4(0, 0, 0, 0);
       if (first) {

@@ -460,8 +460,6 @@ static int encode_call(aq_handle* h, const void* act, const int32_t* sample_ids,
   if (!lists && (!aligned16(act) || !aligned16(packed) || !aligned16(scales)))
     return fail(h, AQ_EINVAL, "%s: act, packed and scales must be 16-byte aligned", who);
   if (lists && h->st.m_bits) return fail(h, AQ_EUNSUPPORTED, "%s: the list form is built for the 16-bit store only", who);
-  if (lists && h->st.lg_shift < 0)
-    return fail(h, AQ_EUNSUPPORTED, "%s: the list form is built for groups of 8, 16, 32, 64, 128 and 256 elements only", who);
   DeviceGuard g(h->device);
   aq::EncodeArgs a{act, sample_ids, static_cast<uint8_t*>(packed), scales, h->first_flags, h->n_batch,
                    h->rounding == AQ_ROUND_STOCHASTIC, h->seed, h->epoch, lists};
@@ -488,8 +486,6 @@ static int decode_call(aq_handle* h, const void* packed, const float* scales, co
   if (!lists && (!aligned16(packed) || !aligned16(scales) || !aligned16(out)))
     return fail(h, AQ_EINVAL, "%s: packed, scales and out must be 16-byte aligned", who);
   if (lists && h->st.m_bits) return fail(h, AQ_EUNSUPPORTED, "%s: the list form is built for the 16-bit store only", who);
-  if (lists && h->st.lg_shift < 0)
-    return fail(h, AQ_EUNSUPPORTED, "%s: the list form is built for groups of 8, 16, 32, 64, 128 and 256 elements only", who);
   DeviceGuard g(h->device);
   aq::DecodeArgs a{static_cast<const uint8_t*>(packed), scales, lists ? static_cast<const void*>(h->raw_list) : h->raw, sample_ids,
                    out, h->first_flags, h->n_batch, lists};

@@ -85,7 +85,7 @@ cudaError_t launch_quant_grad(int dtype, int bits, int lanes_per_group, const vo
                               unsigned long long seed, unsigned long long epoch, int l2_prefetch, cudaStream_t s);
 cudaError_t launch_dequant_grad(int dtype, int bits, int lanes_per_group, const uint8_t* packed,
                                 const float* scales, long long n_elems, void* out, cudaStream_t s);
-// The same four for groups whose lane count is not a power of two up to 32 (aq_anygroup.cu; 16-bit store, base-pointer form).
+// The same four for groups whose lane count is not a power of two up to 32 (aq_anygroup.cu; 16-bit store).
 cudaError_t launch_encode_anygroup(int dtype, int bits, const State& st, const EncodeArgs& a, cudaStream_t s);
 cudaError_t launch_decode_anygroup(int dtype, int bits, const State& st, const DecodeArgs& a, cudaStream_t s);
 cudaError_t launch_quant_grad_anygroup(int dtype, int bits, int lanes_per_group, const void* grad, long long n_elems,

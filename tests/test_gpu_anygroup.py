@@ -75,23 +75,10 @@ def test_gradients_with_other_group_sizes(group, dtype, bits):
 
 
 def test_what_other_group_sizes_do_not_offer():
-    """The low-precision and binary32 stores and the list forms have kernels for groups of 8 to 256
-    elements in powers of two only, and say so."""
+    """The low-precision and binary32 stores have kernels for groups of 8 to 256 elements in powers of
+    two only, and say so."""
     for create in (lambda: aq.aq_create_lowbit(4, 2, 96, 4, 24, 4), lambda: aq.aq_create_fp32(4, 2, 96, 4, 24),
                    lambda: aq.aq_create_hosted_lowbit(4, 2, 96, 4, 24, 8)):
         with pytest.raises(aq.AqError) as e:
             create()
         assert e.value.code == aq.AQ_EUNSUPPORTED
-    h = aq.aq_create(4, 2, 96, 4, 24)
-    try:
-        aq.aq_configure(h, aq.AQ_BATCH, 2)
-        ptrs = torch.zeros(2, dtype=torch.int64, device="cuda")
-        ids = torch.zeros(2, dtype=torch.int32, device="cuda")
-        with pytest.raises(aq.AqError) as e:
-            aq.aq_encode_list(h, ptrs, ids, ptrs, ptrs)
-        assert e.value.code == aq.AQ_EUNSUPPORTED
-        with pytest.raises(aq.AqError) as e:
-            aq.aq_decode_list(h, ptrs, ptrs, ids, ptrs)
-        assert e.value.code == aq.AQ_EUNSUPPORTED
-    finally:
-        aq.aq_destroy(h)

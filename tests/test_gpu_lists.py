@@ -38,6 +38,8 @@ class Scattered:
     (synth.shrink(synth.DEBERTA_XXL, 16, seq=24), 8),
     (synth.shrink(synth.SWEEP_FWD, 6, seq=16), 3),
     (synth.Boundary("list-ragged", 6, 3, 37, 136, "bf16", 5, 8, 3, "outlier", 0.3, seed=71), 3),
+    (synth.Boundary("list-group-40", 6, 3, 11, 640, "fp16", 3, 40, 3, "outlier", 0.3, seed=72), 3),
+    (synth.Boundary("list-group-row", 4, 2, 9, 1600, "bf16", 4, 1600, 3, "normal", 0.3, seed=73), 2),
 ])
 def test_list_forms_match_the_oracle(cfg, nb):
     gs, gr = GpuSide(cfg, nb), GpuSide(cfg, nb)
